@@ -1,0 +1,332 @@
+"""Float64 CPU oracle for the two-stage IPGS visual-token compression of TokenCarve.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+path computes, written from the paper's equations.  It is imported by the tests,
+by the smoke check and by the benchmark's CPU-baseline leg, and by nothing else:
+the CUDA library never calls it and shares no code, table or constant with it.
+
+Everything is float64 numpy.  Library primitives are used only as single steps
+the paper itself names (an SVD, a matrix product, a sort); there is no blocking,
+fusion or reordering.  A LAPACK-free one-sided Jacobi SVD (`svd_jacobi`) is kept
+beside the LAPACK call so each can check the other.
+
+Paper passages followed (TokenCarve, Sec. 3.3):
+  Sec. 3.3.1  Z = U Sigma V^T; row expansion Eq. 3-5; information contribution
+              score Eq. 3-6; attention score Eq. 3-7; combined score Eq. 3-8;
+              Stage I keeps L_vc (1 + rho) tokens.
+  Sec. 3.3.2  Set A / Set B split of the survivors by descending score Eq. 3-9;
+              cosine similarity of normalised attention-output rows Eq. 3-10;
+              the L_vc * rho Set-B tokens with the highest similarity are merged
+              into their Set-A match with ToMe's average; the rest stay intact;
+              L_vc tokens result.
+  Conclusion  surviving tokens keep their original positional relationships.
+
+Readings taken where the paper is silent (each is a parameter or a stated rule):
+  * r in Eq. 3-5/3-6 is the numerical rank  #{sigma_i > rank_tol * sigma_1};
+    rank_tol = 0 sums every min(N, d) term.
+  * Eq. 3-8 is applied to the raw C and S ("none"), or to C / sum(C) and
+    S / sum(S) ("sum1") as an opt-in variant.
+  * M = floor(L_vc * rho) clamped to [0, N - L_vc];  P = L_vc + M survivors;
+    Set A gets floor(P / 2), Set B the rest.
+  * All ties are broken towards the lower original token index.
+  * Decisions (orderings, arg-max) are taken on float32-rounded scores /
+    similarities, the precision in which the library stores them.
+  * "Norm" in Eq. 3-10 is the L2 row normalisation  x / max(|x|_2, 1e-12).
+  * The merged token is the unweighted mean of the destination and every source
+    that chose it; K and V get the same map per head (an extension: the paper
+    merges tokens, it does not say K/V).
+  * Output rows are in ascending original index; that index list is returned.
+
+Parity status: every function below is pinned by tests against closed forms,
+invariants, brute force or an independent routine, except `carve` as a whole
+against the paper's own end-task numbers: the paper prints no intermediate
+values, so end-to-end agreement with the authors' run is "parity unpinned".
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# counts
+# --------------------------------------------------------------------------
+def resolve_counts(n_tokens: int, keep: int, rho: float = 0.5,
+                   n_merge: int = -1) -> Tuple[int, int, int, int]:
+    """(M, P, nA, nB): merged count, Stage-I survivors, |Set A|, |Set B|.
+
+    Stage I keeps L_vc (1 + rho) tokens (Sec. 3.3.1, last paragraph); Stage II
+    merges L_vc * rho of them (Sec. 3.3.2, last paragraph); Eq. 3-9 cuts the
+    sorted survivors at half.
+    """
+    if not (1 <= keep <= n_tokens):
+        raise ValueError("keep out of range")
+    if n_merge < 0:
+        if not (0.0 <= rho <= 1.0):
+            raise ValueError("rho out of range")
+        M = int(np.floor(F64(keep) * F64(np.float32(rho))))
+    else:
+        M = int(n_merge)
+    M = max(0, min(M, n_tokens - keep))
+    P = keep + M
+    nA = P // 2
+    nB = P - nA
+    if M > nB:
+        raise ValueError("n_merge exceeds |Set B|")
+    return M, P, nA, nB
+
+
+# --------------------------------------------------------------------------
+# SVD (Sec. 3.3.1) -- two independent routes
+# --------------------------------------------------------------------------
+def svd_lapack(O: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """U [N, q], sigma [q] (descending), q = min(N, d): the thin SVD as a library step."""
+    U, s, _ = np.linalg.svd(np.asarray(O, F64), full_matrices=False)
+    return U, s
+
+
+def svd_jacobi(O: np.ndarray, max_sweeps: int = 60, tol: float = 1e-15
+               ) -> Tuple[np.ndarray, np.ndarray]:
+    """One-sided (Hestenes) Jacobi SVD written out with plain loops.
+
+    Works on M = O^T when N <= d (so the N columns of M are the tokens) and
+    orthogonalises the columns of M J; the accumulated J is then U and the
+    column norms are sigma.  For N > d it works on O's columns and recovers U
+    from the rotated matrix.  Small inputs only (O(N^2 d) per sweep in Python).
+    """
+    O = np.asarray(O, F64)
+    N, d = O.shape
+    if N <= d:
+        M = O.T.copy()                 # d x N, columns = tokens
+        J = np.eye(N)
+        n = N
+    else:
+        M = O.copy()                   # N x d, columns = features
+        J = None
+        n = d
+    for _ in range(max_sweeps):
+        rotated = False
+        for p in range(n - 1):
+            for q in range(p + 1, n):
+                a = M[:, p] @ M[:, p]
+                b = M[:, q] @ M[:, q]
+                g = M[:, p] @ M[:, q]
+                if abs(g) <= tol * np.sqrt(a * b) or g == 0.0:
+                    continue
+                rotated = True
+                zeta = (b - a) / (2.0 * g)
+                t = np.sign(zeta) / (abs(zeta) + np.sqrt(1.0 + zeta * zeta)) if zeta != 0 else 1.0
+                c = 1.0 / np.sqrt(1.0 + t * t)
+                s = c * t
+                mp = M[:, p].copy()
+                M[:, p] = c * mp - s * M[:, q]
+                M[:, q] = s * mp + c * M[:, q]
+                if J is not None:
+                    jp = J[:, p].copy()
+                    J[:, p] = c * jp - s * J[:, q]
+                    J[:, q] = s * jp + c * J[:, q]
+        if not rotated:
+            break
+    sig = np.sqrt(np.sum(M * M, axis=0))
+    order = np.argsort(-sig, kind="stable")
+    sig = sig[order]
+    if J is not None:
+        U = J[:, order]
+    else:
+        U = np.zeros((N, n))
+        for k, j in enumerate(order):
+            U[:, k] = M[:, j] / sig[k] if sig[k] > 0 else 0.0
+    return U, sig
+
+
+def numerical_rank(sigma: np.ndarray, rank_tol: float) -> int:
+    """r = #{ sigma_i > rank_tol * sigma_1 } (upper limit of the sums in Eq. 3-5 / 3-6)."""
+    if sigma.size == 0 or sigma[0] <= 0.0:
+        return 0
+    return int(np.sum(sigma > F64(np.float32(rank_tol)) * sigma[0]))
+
+
+# --------------------------------------------------------------------------
+# scores (Sec. 3.3.1)
+# --------------------------------------------------------------------------
+def information_contribution(O: np.ndarray, rank_tol: float = 0.0, method: str = "lapack"
+                             ) -> Tuple[np.ndarray, np.ndarray, int]:
+    """C(x) = sum_{i<=r} |u_xi sigma_i|  (Eq. 3-6).  Returns (C [N], sigma [q], r)."""
+    U, sigma = svd_lapack(O) if method == "lapack" else svd_jacobi(O)
+    r = numerical_rank(sigma, rank_tol)
+    C = np.zeros(U.shape[0])
+    for i in range(r):
+        C += np.abs(U[:, i] * sigma[i])
+    return C, sigma, r
+
+
+def attention_score(A: np.ndarray) -> np.ndarray:
+    """S(x) = mean over heads and query rows of A[:, :, x]  (Eq. 3-7).  A is [H, T, N]."""
+    A = np.asarray(A, F64)
+    H, T, N = A.shape
+    S = np.zeros(N)
+    for h in range(H):
+        for t in range(T):
+            S += A[h, t]
+    return S / (H * T)
+
+
+def combined_score(C: np.ndarray, S: np.ndarray, lam: float, score_norm: str = "none"
+                   ) -> np.ndarray:
+    """E(x) = (1 - lambda) C(x) + lambda S(x)  (Eq. 3-8), on raw or sum-normalised terms."""
+    lam = F64(np.float32(lam))
+    if not (0.0 <= lam <= 1.0):
+        raise ValueError("lambda out of range")
+    C = np.asarray(C, F64)
+    S = np.asarray(S, F64)
+    if score_norm == "sum1":
+        cs, ss = C.sum(), S.sum()
+        C = C / cs if cs > 0 else C
+        S = S / ss if ss > 0 else S
+    elif score_norm != "none":
+        raise ValueError("score_norm")
+    return (1.0 - lam) * C + lam * S
+
+
+def score(O: np.ndarray, A: np.ndarray, lam: float = 0.5, rank_tol: float = 0.0,
+          score_norm: str = "none", method: str = "lapack") -> Dict[str, np.ndarray]:
+    C, sigma, r = information_contribution(O, rank_tol, method)
+    S = attention_score(A)
+    E = combined_score(C, S, lam, score_norm)
+    return {"E": E, "C": C, "S": S, "sigma": sigma, "rank": r}
+
+
+# --------------------------------------------------------------------------
+# Stage I prune + Set A / Set B (Sec. 3.3.1 end, Eq. 3-9)
+# --------------------------------------------------------------------------
+def descending_order(values: np.ndarray) -> List[int]:
+    """Indices by (value descending, index ascending); value compared in float32."""
+    v = np.asarray(values, F64).astype(np.float32)
+    idx = list(range(len(v)))
+    idx.sort(key=lambda i: (-float(v[i]), i))
+    return idx
+
+
+def prune_split(E: np.ndarray, P: int, nA: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Survivors = the P best tokens; Set A = the first nA of them, Set B = the rest
+    (Eq. 3-9: IndexSort is the descending-score order of the IPGS scores)."""
+    order = descending_order(E)
+    setA = np.array(order[:nA], dtype=np.int32)
+    setB = np.array(order[nA:P], dtype=np.int32)
+    return setA, setB
+
+
+# --------------------------------------------------------------------------
+# Stage II similarity, matching, merge selection (Eq. 3-10 and the paragraph after it)
+# --------------------------------------------------------------------------
+def normalise_rows(O: np.ndarray) -> np.ndarray:
+    O = np.asarray(O, F64)
+    out = np.empty_like(O)
+    for x in range(O.shape[0]):
+        nrm = np.sqrt(np.sum(O[x] * O[x]))
+        out[x] = O[x] / max(nrm, 1e-12)
+    return out
+
+
+def similarity(O: np.ndarray, setA: Sequence[int], setB: Sequence[int]) -> np.ndarray:
+    """Simi_AB [nB, nA] = Norm(Z)[Set B] x Norm(Z)[Set A]^T  (Eq. 3-10)."""
+    Zn = normalise_rows(O)
+    return Zn[np.asarray(setB, int)] @ Zn[np.asarray(setA, int)].T
+
+
+def match_and_select(sim: np.ndarray, setA: Sequence[int], setB: Sequence[int], M: int
+                     ) -> Tuple[np.ndarray, np.ndarray]:
+    """Each Set-B token's best Set-A partner, then the M Set-B tokens with the highest
+    best-similarity.  Returns (merge_src [M], merge_dst [M]) as original token indices,
+    in selection order (best first).  Ties: lower original index."""
+    setA = [int(a) for a in setA]
+    setB = [int(b) for b in setB]
+    sim32 = np.asarray(sim, F64).astype(np.float32)
+    best_val = []
+    best_dst = []
+    for j, b in enumerate(setB):
+        bv, ba = None, None
+        for i, a in enumerate(setA):
+            v = float(sim32[j, i])
+            if bv is None or v > bv or (v == bv and a < ba):
+                bv, ba = v, a
+        best_val.append(bv)
+        best_dst.append(ba)
+    cand = list(range(len(setB)))
+    cand.sort(key=lambda j: (-best_val[j], setB[j]))
+    chosen = cand[:M]
+    src = np.array([setB[j] for j in chosen], dtype=np.int32)
+    dst = np.array([best_dst[j] for j in chosen], dtype=np.int32)
+    return src, dst
+
+
+def merge(O: np.ndarray, setA: Sequence[int], setB: Sequence[int], M: int
+          ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """(merge_src, merge_dst, kept_idx) for given sets; kept = Set A ∪ unmerged Set B, ascending."""
+    if M > 0 and len(setA) > 0:
+        sim = similarity(O, setA, setB)
+        src, dst = match_and_select(sim, setA, setB, M)
+    else:
+        src = np.zeros(0, np.int32)
+        dst = np.zeros(0, np.int32)
+    merged = set(int(s) for s in src)
+    kept = sorted([int(a) for a in setA] + [int(b) for b in setB if int(b) not in merged])
+    return src, dst, np.array(kept, dtype=np.int32)
+
+
+# --------------------------------------------------------------------------
+# merge + compaction of X, K, V
+# --------------------------------------------------------------------------
+def compact_rows(R: np.ndarray, kept_idx: Sequence[int], merge_src: Sequence[int],
+                 merge_dst: Sequence[int], out_dtype) -> np.ndarray:
+    """Rows `kept_idx` of R [N, w]; a kept row that is a merge destination becomes the
+    plain mean of itself and all its sources (ToMe average with unit sizes), computed
+    in float64 and rounded once (to nearest even) to the storage dtype."""
+    R = np.asarray(R, F64)
+    out = np.empty((len(kept_idx), R.shape[1]), F64)
+    for j, a in enumerate(kept_idx):
+        acc = R[int(a)].copy()
+        cnt = 1
+        for s, t in zip(merge_src, merge_dst):
+            if int(t) == int(a):
+                acc += R[int(s)]
+                cnt += 1
+        out[j] = acc / cnt
+    return out.astype(out_dtype)
+
+
+def compact(X: np.ndarray, K: Optional[np.ndarray], V: Optional[np.ndarray],
+            kept_idx: Sequence[int], merge_src: Sequence[int], merge_dst: Sequence[int],
+            out_dtype) -> Dict[str, Optional[np.ndarray]]:
+    """X' [keep, d], K' / V' [H, keep, dh] under one merge map."""
+    res: Dict[str, Optional[np.ndarray]] = {
+        "X": compact_rows(X, kept_idx, merge_src, merge_dst, out_dtype), "K": None, "V": None}
+    for name, T in (("K", K), ("V", V)):
+        if T is not None:
+            res[name] = np.stack([compact_rows(T[h], kept_idx, merge_src, merge_dst, out_dtype)
+                                  for h in range(T.shape[0])], axis=0)
+    return res
+
+
+# --------------------------------------------------------------------------
+# the whole path for one image
+# --------------------------------------------------------------------------
+def carve(O: np.ndarray, A: np.ndarray, X: np.ndarray, K: Optional[np.ndarray],
+          V: Optional[np.ndarray], keep: int, rho: float = 0.5, lam: float = 0.5,
+          rank_tol: float = 0.0, score_norm: str = "none", n_merge: int = -1,
+          method: str = "lapack") -> Dict[str, object]:
+    """score -> prune -> split -> similarity -> match/select -> merge -> compact, one image.
+
+    Inputs are taken as given (already rounded to their storage dtype); outputs X', K', V'
+    are rounded to X's dtype."""
+    N = O.shape[0]
+    M, P, nA, nB = resolve_counts(N, keep, rho, n_merge)
+    sc = score(O, A, lam, rank_tol, score_norm, method)
+    setA, setB = prune_split(sc["E"], P, nA)
+    src, dst, kept = merge(O, setA, setB, M)
+    out = compact(X, K, V, kept, src, dst, X.dtype)
+    return {**sc, "M": M, "P": P, "setA": setA, "setB": setB, "merge_src": src,
+            "merge_dst": dst, "kept_idx": kept, "Xo": out["X"], "Ko": out["K"], "Vo": out["V"]}
