@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Throughput of the IPGS carve path (TokenCarve Sec. 3.3) on synthetic LLaVA-1.5-shaped inputs.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one tc_carve over a batch of images (score -> prune -> match -> merge -> gather).
+For N > 1 launch under torch.distributed.run; every rank carves its own batch (images are
+independent, so there is no collective on the path) and rank 0 prints one JSON line.
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_10501_b200 import inputs  # noqa: E402
+
+METRIC = "IPGS carve images/s (N=576,d=4096,fp16,keep 128)"
+UNIT = "images/s"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            m = json.load(f)
+        return {"hbm_gbs": float(m["hbm_gbs"]), "bf16_tflops": float(m["bf16_tflops"]),
+                "bf16_tflops_sustained": float(m.get("bf16_tflops_sustained", m["bf16_tflops"])),
+                "sm_max_mhz": float(m.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+def workload(args, rank=0):
+    cfg = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=args.batch, n_query=args.n_query,
+                                                 keep=args.keep)
+    name = f"cfg5_sweep_f16 B={cfg.batch} N={cfg.n_tokens} d={cfg.d_model} T={cfg.n_query} keep={cfg.keep}"
+    return cfg, name
+
+
+def algorithmic_bytes_per_image(cfg, P):
+    """O and A read once; P rows of X, K, V read and keep rows written."""
+    e = 2 if cfg.dtype == "f16" else 4
+    N, d, H, dh, T = cfg.n_tokens, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.n_query
+    row = (d + 2 * H * dh) * e
+    return N * d * e + H * T * N * e + (P + cfg.keep) * row
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+def time_oracle(cfg, n_images, first_image=0):
+    """Seconds per image of the float64 oracle as it stands, and the BLAS threads it may use."""
+    from oracle import ipgs_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    ims = [inputs.make_image(cfg, first_image + b) for b in range(n_images)]
+    t0 = time.perf_counter()
+    for im in ims:
+        orc.carve(im["O"].astype(np.float64), im["A"].astype(np.float64), im["X"], im["K"], im["V"],
+                  cfg.keep, cfg.rho, cfg.lam, cfg.rank_tol, "none")
+    dt = time.perf_counter() - t0
+    return dt / n_images, threads
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, name = workload(args)
+    n = args.cpu_images
+    for _ in range(max(0, min(args.warmup, 1))):
+        time_oracle(cfg, 1)
+    per = []
+    for s in range(args.steps):
+        sec, threads = time_oracle(cfg, n, first_image=s * n)
+        per.append(sec)
+    sec = float(np.mean(per))
+    val = 1.0 / sec
+    sample = f"{n} images per step of the {cfg.batch}-image batch, float64 oracle (LAPACK SVD + loops)"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * n * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": name, "sample_images_per_step": n},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.stop = threading.Event()
+        self.th = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self.stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                      "--format=csv,noheader,nounits"], capture_output=True,
+                                     text=True, timeout=5).stdout.strip()
+                if out:
+                    self.rows.append([c.strip() for c in out.split(",")])
+            except Exception:
+                pass
+            self.stop.wait(0.2)
+
+    def __enter__(self):
+        self.th.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        self.th.join(timeout=6)
+
+    def summary(self):
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names)
+                   if any(len(r) > 3 + i and r[3 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2503_10501_b200 import binding as tcb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the carve path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    tcb.lib()
+
+    cfg, name = workload(args)
+    M, P, nA, nB = 0, 0, 0, 0
+    p = tcb.Params(batch=cfg.batch, n_tokens=cfg.n_tokens, d_model=cfg.d_model, n_heads=cfg.n_heads,
+                   head_dim=cfg.head_dim, n_query=cfg.n_query, keep=cfg.keep, rho=cfg.rho,
+                   lam=cfg.lam, rank_tol=cfg.rank_tol, dtype=cfg.dtype, rank_cap=cfg.rank_cap)
+    M, P, nA, nB = tcb.tc_counts(p)
+    # each rank carves its own images (weak scaling): image numbers rank*B .. rank*B + B - 1
+    batch = inputs.make_batch(cfg, images=range(rank * cfg.batch, (rank + 1) * cfg.batch))
+    hostin = {k: torch.from_numpy(v).pin_memory() for k, v in batch.items()}
+    devin = {k: v.cuda(non_blocking=True) for k, v in hostin.items()}
+    dt = p.torch_dtype
+    mk = lambda *s, dtype=dt: torch.empty(*s, dtype=dtype, device="cuda")
+    out = (mk(p.batch, p.keep, p.d_model), mk(p.batch, p.n_heads, p.keep, p.head_dim),
+           mk(p.batch, p.n_heads, p.keep, p.head_dim), mk(p.batch, p.keep, dtype=torch.int32),
+           mk(p.batch, dtype=torch.int32))
+    hout = tuple(torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in out)
+    ws = tcb.workspace(p, host=True)
+    torch.cuda.synchronize()
+
+    def step():
+        tcb.tc_carve(p, devin["O"], devin["A"], devin["X"], devin["K"], devin["V"], ws, out)
+
+    def step_host():
+        tcb.tc_carve_host(p, hostin["O"], hostin["A"], hostin["X"], hostin["K"], hostin["V"], hout, ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    status = out[4].cpu().numpy()
+    if status.any():
+        raise SystemExit(f"carve reported per-image status {status.tolist()}")
+
+    launches0 = tcb.tc_launch_count()
+    with ClockSampler(local) as cs:
+        ms = timed(step, args.steps)
+    launches = tcb.tc_launch_count() - launches0
+    clocks = cs.summary()
+
+    # per-kernel-class device time (CUDA events on the launching stream), same steps again
+    tcb.tc_profile_begin()
+    for _ in range(args.steps):
+        step()
+    prof = tcb.tc_profile_end()
+
+    # end to end through the host-buffer entry point
+    for _ in range(min(args.warmup, 2)):
+        step_host()
+    ms_host = timed(step_host, args.steps)
+
+    images = cfg.batch * world * args.steps
+    value = images / (ms * 1e-3)
+    e2e = images / (ms_host * 1e-3)
+    nbytes = lambda ts: int(sum(t.numel() * t.element_size() for t in ts))
+    pk = peaks()
+
+    # roofline of the kernel class that takes the most device time
+    top = max(prof.items(), key=lambda kv: kv[1][0])
+    top_name, (top_ms, top_launches) = top
+    per_launch_s = top_ms * 1e-3 / max(top_launches, 1)
+    k = p.rank_cap if p.rank_cap else p.n_tokens
+    alg_bytes_img = algorithmic_bytes_per_image(cfg, P)
+    if top_name == "jacobi":
+        # one-sided Jacobi with accumulated rotations: 18 k flops per column pair, k(k-1)/2 pairs
+        # per sweep, 8 sweeps nominal
+        flops = cfg.batch * 8 * 18.0 * k * (k * (k - 1) / 2)
+        peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+        roof = {"kernel": top_name, "bound": "alu", "achieved": flops / per_launch_s / 1e12,
+                "peak": peak, "unit": "TFLOP/s", "traffic": None}
+    elif top_name in ("gram",):
+        flops = cfg.batch * 2.0 * cfg.n_tokens ** 2 * cfg.d_model
+        roof = {"kernel": top_name, "bound": "tensor", "achieved": flops / per_launch_s / 1e12,
+                "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "traffic": None}
+    elif top_name == "gemm_f32":
+        N = cfg.n_tokens
+        flops = cfg.batch * (2 * 2.0 * N * N * k + 8 * 2.0 * N * k * k + 5 * 2.0 * N * k * k) / max(top_launches / args.steps, 1)
+        peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+        roof = {"kernel": top_name, "bound": "alu", "achieved": flops / per_launch_s / 1e12,
+                "peak": peak, "unit": "TFLOP/s", "traffic": None}
+    else:
+        e = 2
+        per = {"attn_colsum": cfg.n_heads * cfg.n_query * cfg.n_tokens * e,
+               "compact": (P + cfg.keep) * (cfg.d_model + 2 * cfg.n_heads * cfg.head_dim) * e,
+               "sketch": cfg.n_tokens * cfg.d_model * e}.get(top_name, alg_bytes_img)
+        roof = {"kernel": top_name, "bound": "hbm", "achieved": cfg.batch * per / per_launch_s / 1e9,
+                "peak": pk["hbm_gbs"], "unit": "GB/s", "traffic": None}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["peak_source"] = pk["source"]
+    # the whole path against the slower of its HBM bytes and its Gram flops
+    t_hbm = alg_bytes_img / (pk["hbm_gbs"] * 1e9)
+    t_tensor = 2.0 * cfg.n_tokens ** 2 * cfg.d_model / (pk["bf16_tflops_sustained"] * 1e12)
+    t_roof = max(t_hbm, t_tensor)
+    us_img = ms * 1e3 / (cfg.batch * args.steps)
+    path = {"roofline_us_per_image": t_roof * 1e6, "achieved_us_per_image": us_img,
+            "frac": t_roof * 1e6 / us_img, "bound": "hbm" if t_hbm >= t_tensor else "tensor",
+            "algorithmic_bytes_per_image": alg_bytes_img}
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and args.cpu_images > 0:
+            sec, threads = time_oracle(cfg, args.cpu_images)
+            cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
+                   "sample": f"{args.cpu_images} images of the {cfg.batch}-image batch, "
+                             "float64 oracle (LAPACK SVD + loops)"}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": name, "images_per_gpu": cfg.batch, "rank_cap": p.rank_cap,
+                           "rank_tol": p.rank_tol, "lambda": p.lam, "rho": p.rho,
+                           "l2": "inputs (1.5 GB per step) exceed the 126 MB L2"},
+                "us_per_image": us_img,
+                "e2e": {"value": e2e, "unit": UNIT,
+                        "h2d_bytes_per_step": nbytes(hostin.values()),
+                        "d2h_bytes_per_step": nbytes(hout)},
+                "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
+                "path_roofline": path,
+                "kernel_ms_per_step": {k_: round(v[0] / args.steps, 4) for k_, v in prof.items() if v[1]},
+                "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=64, help="images per GPU per step")
+    ap.add_argument("--n-query", type=int, default=128)
+    ap.add_argument("--keep", type=int, default=128)
+    ap.add_argument("--cpu-images", type=int, default=12,
+                    help="images the CPU oracle is timed on (0 = skip)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

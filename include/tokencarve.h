@@ -1,0 +1,183 @@
+/*
+ * tokencarve.h -- C ABI of the IPGS carve library (TokenCarve, Sec. 3.3).
+ *
+ * The library runs the two-stage Information-Preservation-Guided Selection that TokenCarve
+ * applies once per request at prefill, between LLM layers 2 and 3:
+ *
+ *   Stage I  (Sec. 3.3.1)  score every visual token  E(x) = (1-lambda) C(x) + lambda S(x)
+ *                          (Eq. 3-8), C from the SVD of the attention-output matrix (Eq. 3-5,
+ *                          3-6), S the mean attention the token receives (Eq. 3-7); keep the
+ *                          L_vc (1 + rho) best.
+ *   Stage II (Sec. 3.3.2)  split the survivors by score into Set A / Set B (Eq. 3-9), match
+ *                          every Set-B token to its most cosine-similar Set-A token
+ *                          (Eq. 3-10), merge the L_vc * rho best-matched Set-B tokens into
+ *                          their match by a plain average, keep the rest; L_vc tokens result,
+ *                          in their original order (Sec. 5).
+ *
+ * Conventions for every entry point
+ *   - Every data pointer is DEVICE memory owned by the caller (the *_host entry point is the
+ *     one exception and says so), contiguous, row-major, 16-byte aligned.  The library
+ *     allocates nothing: all scratch is carved out of the caller's workspace `ws`, whose
+ *     size tc_workspace_bytes() reports for a given tc_params.
+ *   - Layouts:  O, X [B, N, d];  A [B, H, T, N];  K, V [B, H, N, dh];
+ *     outputs   Xo [B, keep, d];  Ko, Vo [B, H, keep, dh];  kept_idx [B, keep].
+ *     Element type is tc_params.dtype for O, A, X, K, V and the outputs; scores, singular
+ *     values and similarities are float32; indices are int32 token numbers in [0, N).
+ *   - Calls only enqueue work on `stream` and never synchronise.  Errors the host can see
+ *     (bad sizes, NULL pointers, short workspace) return a status immediately and enqueue
+ *     nothing.  Conditions only the device can see are written per image to `img_status`
+ *     (TC_OK when fine) and never trap; they are valid once the stream has been synchronised.
+ *   - Index lists are in ascending token order.  Every tie (equal scores, equal
+ *     similarities) goes to the lower token index.
+ */
+#ifndef TOKENCARVE_H
+#define TOKENCARVE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TC_OK = 0,
+  TC_ERR_INVALID_ARG = 1,   /* NULL pointer, size or parameter out of range                 */
+  TC_ERR_UNSUPPORTED = 2,   /* shape outside what the kernels handle                         */
+  TC_ERR_WORKSPACE = 3,     /* ws_bytes smaller than tc_workspace_bytes()                    */
+  TC_ERR_NOT_CONVERGED = 4, /* img_status: Jacobi hit max_sweeps before its tolerance        */
+  TC_ERR_CUDA = 5,          /* a CUDA runtime call failed                                    */
+  TC_ERR_RANK_CAP = 6,      /* img_status: numerical rank reached rank_cap; rerun that image
+                               with a larger rank_cap or with rank_cap = 0                   */
+  TC_ERR_BREAKDOWN = 7      /* img_status: a Cholesky pivot was not positive                 */
+} tc_status;
+
+typedef enum { TC_F16 = 0, TC_F32 = 1 } tc_dtype;
+
+/* How Eq. 3-8 combines the two terms: on the raw C and S (the equation as printed), or on
+ * C / sum(C) and S / sum(S) so that both terms have the same scale. */
+typedef enum { TC_NORM_NONE = 0, TC_NORM_SUM1 = 1 } tc_score_norm;
+
+typedef struct tc_params {
+  int32_t batch;      /* B   images                                                          */
+  int32_t n_tokens;   /* N = L_v  visual tokens per image                                    */
+  int32_t d_model;    /* d   width of O and X                                                */
+  int32_t n_heads;    /* H                                                                   */
+  int32_t head_dim;   /* dh                                                                  */
+  int32_t n_query;    /* T   query rows in the attention slice A                             */
+  int32_t keep;       /* L_vc, 1..N                                                          */
+  int32_t n_merge;    /* M;  -1 => floor(keep * rho), clamped to [0, N - keep]               */
+  float   rho;        /* merge proportion of Sec. 3.3.1/3.3.2, in [0, 1]                     */
+  float   lambda;     /* weight of Eq. 3-8, in [0, 1]                                        */
+  float   rank_tol;   /* r of Eq. 3-5/3-6 = #{ sigma_i > rank_tol * sigma_1 }; 0 => all      */
+  int32_t dtype;      /* tc_dtype of O, A, X, K, V and of Xo, Ko, Vo                         */
+  int32_t score_norm; /* tc_score_norm                                                       */
+  int32_t max_sweeps; /* bound on Jacobi sweeps (<= 0 => 30)                                 */
+  int32_t rank_cap;   /* 0 => full N x N eigen-decomposition of the Gram matrix.
+                         k > 0 (k < N) => the caller states that the numerical rank r is
+                         below k: only a k-dimensional dominant subspace is decomposed.  The
+                         device checks r <= k - 8 and reports TC_ERR_RANK_CAP otherwise.
+                         Singular values beyond the k-th are then reported as 0.             */
+  uint32_t flags;     /* reserved, 0                                                         */
+} tc_params;
+
+/* Counts derived from the parameters (Sec. 3.3.1 last paragraph, Eq. 3-9):
+ * M merged tokens, P = keep + M Stage-I survivors, nA = floor(P / 2), nB = P - nA. */
+tc_status tc_counts(const tc_params* p, int32_t* M, int32_t* P, int32_t* nA, int32_t* nB);
+
+/* Bytes of device workspace any of the calls below needs for these parameters. */
+tc_status tc_workspace_bytes(const tc_params* p, size_t* bytes);
+
+/*
+ * Stage I scores (Sec. 3.3.1, Eq. 3-5 ... 3-8).
+ *   O [B,N,d], A [B,H,T,N] in;  E [B,N] out (required);
+ *   optional outs (NULL to skip): C [B,N] Eq. 3-6, S [B,N] Eq. 3-7,
+ *   sigma [B, min(N,d)] singular values, descending, rank [B] the r used in Eq. 3-6.
+ *   img_status [B] int32 (required).
+ */
+tc_status tc_score(const tc_params* p, const void* O, const void* A, float* E, float* C,
+                   float* S, float* sigma, int32_t* rank, int32_t* img_status, void* ws,
+                   size_t ws_bytes, void* stream);
+
+/*
+ * Stage I prune and the Set A / Set B split (Sec. 3.3.1 last paragraph, Eq. 3-9).
+ *   E [B,N] in;  setA [B,nA], setB [B,nB] out: Set A holds the nA best-scored tokens, Set B
+ *   the next nB; each list in ascending token index.
+ */
+tc_status tc_prune(const tc_params* p, const float* E, int32_t* setA, int32_t* setB, void* ws,
+                   size_t ws_bytes, void* stream);
+
+/*
+ * Stage II matching (Eq. 3-10 and the paragraph after it).
+ *   O [B,N,d], setA, setB in.  Cosine similarity of the L2-normalised rows of O between every
+ *   Set-B and Set-A token; each Set-B token's best Set-A match; the M Set-B tokens with the
+ *   highest best-similarity are merged.
+ *   merge_src [B,M] (ascending), merge_dst [B,M] (the match of merge_src[i]),
+ *   kept_idx [B,keep] = Set A plus the unmerged Set-B tokens, ascending.
+ */
+tc_status tc_merge(const tc_params* p, const void* O, const int32_t* setA, const int32_t* setB,
+                   int32_t* merge_src, int32_t* merge_dst, int32_t* kept_idx, void* ws,
+                   size_t ws_bytes, void* stream);
+
+/*
+ * Merge and gather (Sec. 3.3.2 last paragraph: ToMe's average; Sec. 5: original order).
+ *   Row j of the output is row kept_idx[j] of the input, or, when that token is a merge
+ *   destination, the plain mean of it and all tokens merged into it (float32 accumulate,
+ *   one rounding to the storage type).  The same map is applied to X and to every head of
+ *   K and V.  K, V, Ko, Vo may all be NULL (then only X is compacted).
+ */
+tc_status tc_compact(const tc_params* p, const void* X, const void* K, const void* V,
+                     const int32_t* kept_idx, const int32_t* merge_src,
+                     const int32_t* merge_dst, void* Xo, void* Ko, void* Vo, void* ws,
+                     size_t ws_bytes, void* stream);
+
+/*
+ * The whole path (Sec. 3.3): score -> prune -> split -> match -> merge -> gather, one
+ * enqueue, no host synchronisation inside.
+ */
+tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void* X,
+                   const void* K, const void* V, void* Xo, void* Ko, void* Vo,
+                   int32_t* kept_idx, int32_t* img_status, void* ws, size_t ws_bytes,
+                   void* stream);
+
+/*
+ * tc_carve for callers whose tensors live in HOST memory (pinned for the copies to be
+ * asynchronous).  O, A, X, K, V, Xo, Ko, Vo, kept_idx and img_status are host pointers; the
+ * inputs are copied to the device, carved, and the results copied back, all on `stream`.
+ * `ws` is device memory of at least tc_workspace_bytes_host() bytes (staging + scratch).
+ */
+tc_status tc_workspace_bytes_host(const tc_params* p, size_t* bytes);
+tc_status tc_carve_host(const tc_params* p, const void* O, const void* A, const void* X,
+                        const void* K, const void* V, void* Xo, void* Ko, void* Vo,
+                        int32_t* kept_idx, int32_t* img_status, void* ws, size_t ws_bytes,
+                        void* stream);
+
+/*
+ * The Gram matrix behind the SVD of Sec. 3.3.1 (O O^T = U Sigma^2 U^T) and the similarity of
+ * Eq. 3-10, exposed for inspection: G [B,N,N] float32 out.
+ */
+tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream);
+
+/*
+ * Optional event profile (diagnostics; the paper has no counterpart).  Between
+ * tc_profile_begin() and tc_profile_end() every kernel launch of the library is bracketed by
+ * CUDA events on its stream.  tc_profile_end() waits for those events and returns, per kernel
+ * class (0 .. TC_N_KERNEL_CLASSES-1, named by tc_kernel_class_name), the summed device time in
+ * milliseconds and the number of launches, in the HOST arrays ms[n], launches[n]
+ * (n >= TC_N_KERNEL_CLASSES).  Not thread-safe against concurrent carve calls.
+ */
+#define TC_N_KERNEL_CLASSES 13
+int32_t tc_profile_begin(void);
+int32_t tc_profile_end(double* ms, int64_t* launches, int32_t n);
+const char* tc_kernel_class_name(int32_t cls);
+
+/* Number of kernels the library has launched in this process so far (diagnostics). */
+int64_t tc_launch_count(void);
+
+const char* tc_status_string(int32_t status);
+int32_t tc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOKENCARVE_H */

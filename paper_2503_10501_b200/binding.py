@@ -1,0 +1,289 @@
+"""ctypes binding of ``libtokencarve.so``: argument marshalling only.
+
+Every function takes torch CUDA tensors (used purely as device memory) and enqueues the
+library call of the same name on the current CUDA stream.  There is no fallback: if the
+shared library cannot be built or loaded, importing the entry points raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Dict, Optional, Tuple
+
+import torch
+
+from . import build as _build
+
+TC_OK = 0
+TC_F16, TC_F32 = 0, 1
+TC_NORM_NONE, TC_NORM_SUM1 = 0, 1
+STATUS_NAMES = {0: "TC_OK", 1: "TC_ERR_INVALID_ARG", 2: "TC_ERR_UNSUPPORTED", 3: "TC_ERR_WORKSPACE",
+                4: "TC_ERR_NOT_CONVERGED", 5: "TC_ERR_CUDA", 6: "TC_ERR_RANK_CAP",
+                7: "TC_ERR_BREAKDOWN"}
+
+# every symbol include/tokencarve.h declares
+EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge", "tc_compact",
+           "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
+           "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
+           "tc_kernel_class_name")
+
+
+class TcParams(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_tokens", C.c_int32), ("d_model", C.c_int32),
+                ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("n_query", C.c_int32),
+                ("keep", C.c_int32), ("n_merge", C.c_int32), ("rho", C.c_float),
+                ("lambda_", C.c_float), ("rank_tol", C.c_float), ("dtype", C.c_int32),
+                ("score_norm", C.c_int32), ("max_sweeps", C.c_int32), ("rank_cap", C.c_int32),
+                ("flags", C.c_uint32)]
+
+
+class TokenCarveError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        super().__init__(f"{fn} returned {STATUS_NAMES.get(status, status)}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load (building first if needed) the shared library; raises if that is impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not _build.up_to_date():
+            try:
+                path = _build.build()
+            except Exception:
+                if not os.path.exists(path):
+                    raise
+        L = C.CDLL(path)
+        vp, sz = C.c_void_p, C.c_size_t
+        pp = C.POINTER(TcParams)
+        L.tc_counts.argtypes = [pp] + [C.POINTER(C.c_int32)] * 4
+        L.tc_workspace_bytes.argtypes = [pp, C.POINTER(sz)]
+        L.tc_workspace_bytes_host.argtypes = [pp, C.POINTER(sz)]
+        L.tc_score.argtypes = [pp] + [vp] * 8 + [vp, sz, vp]
+        L.tc_prune.argtypes = [pp, vp, vp, vp, vp, sz, vp]
+        L.tc_merge.argtypes = [pp] + [vp] * 6 + [vp, sz, vp]
+        L.tc_compact.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
+        L.tc_carve.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
+        L.tc_carve_host.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
+        L.tc_gram.argtypes = [pp, vp, vp, vp]
+        L.tc_status_string.argtypes = [C.c_int32]
+        L.tc_status_string.restype = C.c_char_p
+        L.tc_kernel_class_name.argtypes = [C.c_int32]
+        L.tc_kernel_class_name.restype = C.c_char_p
+        L.tc_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int32]
+        for name in EXPORTS:
+            if name not in ("tc_status_string", "tc_kernel_class_name"):
+                getattr(L, name).restype = C.c_int32
+        L.tc_launch_count.restype = C.c_int64
+        _lib = L
+    return _lib
+
+
+@dataclass
+class Params:
+    """Python mirror of ``tc_params`` (see include/tokencarve.h for the meaning of each field)."""
+    batch: int
+    n_tokens: int
+    d_model: int
+    n_heads: int
+    head_dim: int
+    n_query: int
+    keep: int
+    n_merge: int = -1
+    rho: float = 0.5
+    lam: float = 0.5
+    rank_tol: float = 0.0
+    dtype: str = "f16"
+    score_norm: str = "none"
+    max_sweeps: int = 30
+    rank_cap: int = 0
+
+    def c(self) -> TcParams:
+        return TcParams(self.batch, self.n_tokens, self.d_model, self.n_heads, self.head_dim,
+                        self.n_query, self.keep, self.n_merge, self.rho, self.lam, self.rank_tol,
+                        TC_F16 if self.dtype == "f16" else TC_F32,
+                        TC_NORM_SUM1 if self.score_norm == "sum1" else TC_NORM_NONE,
+                        self.max_sweeps, self.rank_cap, 0)
+
+    @property
+    def torch_dtype(self):
+        return torch.float16 if self.dtype == "f16" else torch.float32
+
+
+def _check(fn: str, status: int) -> None:
+    if status != TC_OK:
+        raise TokenCarveError(fn, status)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device, contiguous tensors only"
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def tc_counts(p: Params) -> Tuple[int, int, int, int]:
+    v = [C.c_int32() for _ in range(4)]
+    cp = p.c()
+    _check("tc_counts", lib().tc_counts(C.byref(cp), *[C.byref(x) for x in v]))
+    return tuple(x.value for x in v)
+
+
+def tc_workspace_bytes(p: Params) -> int:
+    n = C.c_size_t()
+    cp = p.c()
+    _check("tc_workspace_bytes", lib().tc_workspace_bytes(C.byref(cp), C.byref(n)))
+    return n.value
+
+
+def tc_workspace_bytes_host(p: Params) -> int:
+    n = C.c_size_t()
+    cp = p.c()
+    _check("tc_workspace_bytes_host", lib().tc_workspace_bytes_host(C.byref(cp), C.byref(n)))
+    return n.value
+
+
+def workspace(p: Params, device="cuda", host: bool = False) -> torch.Tensor:
+    n = tc_workspace_bytes_host(p) if host else tc_workspace_bytes(p)
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def tc_gram(p: Params, O: torch.Tensor) -> torch.Tensor:
+    G = torch.empty(p.batch, p.n_tokens, p.n_tokens, dtype=torch.float32, device=O.device)
+    cp = p.c()
+    _check("tc_gram", lib().tc_gram(C.byref(cp), _ptr(O), _ptr(G), _stream()))
+    return G
+
+
+def tc_score(p: Params, O, A, ws=None) -> Dict[str, torch.Tensor]:
+    dev = O.device
+    ws = ws if ws is not None else workspace(p, dev)
+    B, N = p.batch, p.n_tokens
+    q = min(N, p.d_model)
+    out = {"E": torch.empty(B, N, dtype=torch.float32, device=dev),
+           "C": torch.empty(B, N, dtype=torch.float32, device=dev),
+           "S": torch.empty(B, N, dtype=torch.float32, device=dev),
+           "sigma": torch.empty(B, q, dtype=torch.float32, device=dev),
+           "rank": torch.empty(B, dtype=torch.int32, device=dev),
+           "img_status": torch.empty(B, dtype=torch.int32, device=dev)}
+    cp = p.c()
+    _check("tc_score", lib().tc_score(C.byref(cp), _ptr(O), _ptr(A), _ptr(out["E"]), _ptr(out["C"]),
+                                      _ptr(out["S"]), _ptr(out["sigma"]), _ptr(out["rank"]),
+                                      _ptr(out["img_status"]), _ptr(ws), ws.numel(), _stream()))
+    return out
+
+
+def tc_prune(p: Params, E, ws=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    dev = E.device
+    ws = ws if ws is not None else workspace(p, dev)
+    M, P, nA, nB = tc_counts(p)
+    setA = torch.empty(p.batch, nA, dtype=torch.int32, device=dev)
+    setB = torch.empty(p.batch, nB, dtype=torch.int32, device=dev)
+    cp = p.c()
+    _check("tc_prune", lib().tc_prune(C.byref(cp), _ptr(E), _ptr(setA) if nA else None, _ptr(setB),
+                                      _ptr(ws), ws.numel(), _stream()))
+    return setA, setB
+
+
+def tc_merge(p: Params, O, setA, setB, ws=None):
+    dev = O.device
+    ws = ws if ws is not None else workspace(p, dev)
+    M, P, nA, nB = tc_counts(p)
+    src = torch.empty(p.batch, M, dtype=torch.int32, device=dev)
+    dst = torch.empty(p.batch, M, dtype=torch.int32, device=dev)
+    kept = torch.empty(p.batch, p.keep, dtype=torch.int32, device=dev)
+    cp = p.c()
+    _check("tc_merge", lib().tc_merge(C.byref(cp), _ptr(O), _ptr(setA) if nA else None, _ptr(setB),
+                                      _ptr(src) if M else None, _ptr(dst) if M else None,
+                                      _ptr(kept), _ptr(ws), ws.numel(), _stream()))
+    return src, dst, kept
+
+
+def _outputs(p: Params, dev, with_kv: bool):
+    dt = p.torch_dtype
+    Xo = torch.empty(p.batch, p.keep, p.d_model, dtype=dt, device=dev)
+    Ko = Vo = None
+    if with_kv:
+        Ko = torch.empty(p.batch, p.n_heads, p.keep, p.head_dim, dtype=dt, device=dev)
+        Vo = torch.empty_like(Ko)
+    return Xo, Ko, Vo
+
+
+def tc_compact(p: Params, X, K, V, kept, src, dst, ws=None):
+    dev = X.device
+    ws = ws if ws is not None else workspace(p, dev)
+    M = tc_counts(p)[0]
+    Xo, Ko, Vo = _outputs(p, dev, K is not None)
+    cp = p.c()
+    _check("tc_compact", lib().tc_compact(C.byref(cp), _ptr(X), _ptr(K), _ptr(V), _ptr(kept),
+                                          _ptr(src) if M else None, _ptr(dst) if M else None,
+                                          _ptr(Xo), _ptr(Ko), _ptr(Vo), _ptr(ws), ws.numel(),
+                                          _stream()))
+    return Xo, Ko, Vo
+
+
+def tc_carve(p: Params, O, A, X, K=None, V=None, ws=None, out=None):
+    """Returns (Xo, Ko, Vo, kept_idx, img_status); `out` may supply those five tensors."""
+    dev = O.device
+    ws = ws if ws is not None else workspace(p, dev)
+    if out is None:
+        Xo, Ko, Vo = _outputs(p, dev, K is not None)
+        kept = torch.empty(p.batch, p.keep, dtype=torch.int32, device=dev)
+        status = torch.empty(p.batch, dtype=torch.int32, device=dev)
+    else:
+        Xo, Ko, Vo, kept, status = out
+    cp = p.c()
+    _check("tc_carve", lib().tc_carve(C.byref(cp), _ptr(O), _ptr(A), _ptr(X), _ptr(K), _ptr(V),
+                                      _ptr(Xo), _ptr(Ko), _ptr(Vo), _ptr(kept), _ptr(status),
+                                      _ptr(ws), ws.numel(), _stream()))
+    return Xo, Ko, Vo, kept, status
+
+
+def tc_carve_host(p: Params, O, A, X, K, V, out, ws):
+    """Host-memory variant: inputs and `out` = (Xo, Ko, Vo, kept_idx, img_status) are (pinned)
+    CPU tensors, `ws` a device workspace of tc_workspace_bytes_host() bytes."""
+    for t in (O, A, X, K, V) + tuple(out):
+        assert t is None or (not t.is_cuda and t.is_contiguous())
+    hp = lambda t: None if t is None else t.data_ptr()
+    Xo, Ko, Vo, kept, status = out
+    cp = p.c()
+    _check("tc_carve_host", lib().tc_carve_host(C.byref(cp), hp(O), hp(A), hp(X), hp(K), hp(V),
+                                                hp(Xo), hp(Ko), hp(Vo), hp(kept), hp(status),
+                                                _ptr(ws), ws.numel(), _stream()))
+    return out
+
+
+def tc_status_string(status: int) -> str:
+    return lib().tc_status_string(status).decode()
+
+
+def tc_version() -> int:
+    return lib().tc_version()
+
+
+def tc_launch_count() -> int:
+    return lib().tc_launch_count()
+
+
+N_KERNEL_CLASSES = 13
+
+
+def tc_profile_begin() -> None:
+    _check("tc_profile_begin", lib().tc_profile_begin())
+
+
+def tc_profile_end() -> Dict[str, Tuple[float, int]]:
+    """{kernel class name: (device milliseconds, launches)} since tc_profile_begin()."""
+    ms = (C.c_double * N_KERNEL_CLASSES)()
+    n = (C.c_int64 * N_KERNEL_CLASSES)()
+    _check("tc_profile_end", lib().tc_profile_end(ms, n, N_KERNEL_CLASSES))
+    return {lib().tc_kernel_class_name(i).decode(): (ms[i], n[i]) for i in range(N_KERNEL_CLASSES)}

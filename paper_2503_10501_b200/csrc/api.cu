@@ -1,0 +1,440 @@
+// C ABI of libtokencarve: argument checks, workspace planning, and the order in which the
+// kernels of each stage are enqueued.
+#include <math.h>
+#include <string.h>
+
+#include <atomic>
+#include <mutex>
+#include <vector>
+
+#include "tc_internal.cuh"
+
+namespace tc {
+
+static std::atomic<long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// ---- optional event profile ---------------------------------------------------------------
+struct Profiler {
+  std::mutex mu;
+  bool on = false;
+  std::vector<cudaEvent_t> ev;   // pairs (start, stop)
+  std::vector<int> cls;          // class of each pair
+  std::vector<long long> launches_at_open, launches_at_close;
+  size_t used = 0;               // pairs in use
+};
+static Profiler g_prof;
+
+Scope::Scope(int cls, cudaStream_t s) : slot(-1), st(s) {
+  if (!g_prof.on) return;
+  std::lock_guard<std::mutex> lk(g_prof.mu);
+  if (g_prof.used == g_prof.cls.size()) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+    g_prof.ev.push_back(a);
+    g_prof.ev.push_back(b);
+    g_prof.cls.push_back(cls);
+    g_prof.launches_at_open.push_back(0);
+    g_prof.launches_at_close.push_back(0);
+  }
+  slot = (int)g_prof.used++;
+  g_prof.cls[slot] = cls;
+  g_prof.launches_at_open[slot] = g_launches.load();
+  cudaEventRecord(g_prof.ev[2 * slot], st);
+}
+Scope::~Scope() {
+  if (slot < 0) return;
+  std::lock_guard<std::mutex> lk(g_prof.mu);
+  cudaEventRecord(g_prof.ev[2 * slot + 1], st);
+  g_prof.launches_at_close[slot] = g_launches.load();
+}
+
+tc_status launch_gram_simt(const Dims& D, const void* O, float* G, cudaStream_t st);
+void fill_i32(int32_t* p, int n, int v, cudaStream_t st);
+
+tc_status make_dims(const tc_params* p, Dims* out) {
+  if (p == nullptr || out == nullptr) return TC_ERR_INVALID_ARG;
+  Dims D;
+  memset(&D, 0, sizeof(D));
+  D.B = p->batch; D.N = p->n_tokens; D.d = p->d_model; D.H = p->n_heads; D.dh = p->head_dim;
+  D.T = p->n_query; D.keep = p->keep;
+  if (D.B < 1 || D.N < 1 || D.d < 1 || D.H < 1 || D.dh < 1 || D.T < 1) return TC_ERR_INVALID_ARG;
+  if (D.keep < 1 || D.keep > D.N) return TC_ERR_INVALID_ARG;
+  if (!(p->lambda >= 0.f && p->lambda <= 1.f)) return TC_ERR_INVALID_ARG;
+  if (!(p->rank_tol >= 0.f && p->rank_tol < 1.f)) return TC_ERR_INVALID_ARG;
+  if (p->dtype != TC_F16 && p->dtype != TC_F32) return TC_ERR_INVALID_ARG;
+  if (p->score_norm != TC_NORM_NONE && p->score_norm != TC_NORM_SUM1) return TC_ERR_INVALID_ARG;
+  if (p->flags != 0) return TC_ERR_INVALID_ARG;
+  // M = floor(L_vc * rho), P = L_vc + M (Sec. 3.3.1 / 3.3.2), Set A = first half (Eq. 3-9)
+  int M;
+  if (p->n_merge < 0) {
+    if (!(p->rho >= 0.f && p->rho <= 1.f)) return TC_ERR_INVALID_ARG;
+    M = (int)floor((double)D.keep * (double)p->rho);
+  } else {
+    M = p->n_merge;
+  }
+  if (M > D.N - D.keep) M = D.N - D.keep;
+  if (M < 0) M = 0;
+  D.M = M;
+  D.P = D.keep + M;
+  D.nA = D.P / 2;
+  D.nB = D.P - D.nA;
+  if (D.M > D.nB) return TC_ERR_INVALID_ARG;
+  D.f16 = (p->dtype == TC_F16);
+  D.esz = D.f16 ? 2 : 4;
+  // rows must be whole 16-byte vectors for the gather; selection kernels cover N <= 4096
+  if (((size_t)D.d * D.esz) % 16 != 0 || ((size_t)D.dh * D.esz) % 16 != 0) return TC_ERR_UNSUPPORTED;
+  if (D.N > 4096) return TC_ERR_UNSUPPORTED;
+  if (p->rank_cap < 0) return TC_ERR_INVALID_ARG;
+  D.full = (p->rank_cap == 0) || (p->rank_cap >= D.N);
+  D.k = D.full ? D.N : p->rank_cap;
+  if (D.k > 1024) return TC_ERR_UNSUPPORTED;  // Jacobi keeps at most 32 elements per lane
+  if (!D.full && D.k < 16) return TC_ERR_INVALID_ARG;
+  D.max_sweeps = p->max_sweeps > 0 ? p->max_sweeps : 30;
+  D.lambda = p->lambda;
+  D.rank_tol = p->rank_tol;
+  D.score_norm = p->score_norm;
+  // row chunks of the attention reduction: enough blocks to fill the GPU, at least 32 rows each
+  const int R = D.H * D.T;
+  int chunks = (4 * 148 + D.B - 1) / D.B;
+  if (chunks > R / 32) chunks = R / 32;
+  if (chunks > 64) chunks = 64;
+  if (chunks < 1) chunks = 1;
+  D.chunks = chunks;
+  *out = D;
+  return TC_OK;
+}
+
+Plan make_plan(const Dims& D) {
+  Plan P;
+  memset(&P, 0, sizeof(P));
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t B = D.B, N = D.N, k = D.k;
+  P.s_part = take(B * D.chunks * N * 4);
+  P.S = take(B * N * 4);
+  P.C = take(B * N * 4);
+  P.E = take(B * N * 4);
+  P.sigma = take(B * k * 4);
+  P.G = take(B * N * N * 4);
+  if (!D.full) {
+    P.Y0 = take(B * N * k * 4);
+    P.Y1 = take(B * N * k * 4);
+    P.Y2 = take(B * N * k * 4);
+    P.Sm = take(B * k * k * 4);
+    P.Rinv = take(B * k * k * 4);
+    P.Hm = take(B * k * k * 4);
+  }
+  P.W = take(B * k * k * 4);
+  P.ZT = take(B * k * k * 4);
+  P.setA = take(B * (size_t)(D.nA > 0 ? D.nA : 1) * 4);
+  P.setB = take(B * (size_t)D.nB * 4);
+  P.best_val = take(B * (size_t)D.nB * 4);
+  P.best_dst = take(B * (size_t)D.nB * 4);
+  P.msrc = take(B * (size_t)(D.M > 0 ? D.M : 1) * 4);
+  P.mdst = take(B * (size_t)(D.M > 0 ? D.M : 1) * 4);
+  P.kept = take(B * (size_t)D.keep * 4);
+  P.rank = take(B * 4);
+  P.flags = take(B * 4);
+  P.total = off;
+  return P;
+}
+
+tc_status launch_gram(const Dims& D, const void* O, float* G, cudaStream_t st) {
+  return launch_gram_simt(D, O, G, st);
+}
+
+static tc_status check_launch() {
+  return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
+}
+
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15u) != 0; }
+
+struct Ctx {
+  Dims D;
+  Plan P;
+  char* ws;
+  cudaStream_t st;
+};
+
+static tc_status open_ctx(const tc_params* p, void* ws, size_t ws_bytes, void* stream, Ctx* c) {
+  tc_status s = make_dims(p, &c->D);
+  if (s != TC_OK) return s;
+  c->P = make_plan(c->D);
+  if (ws == nullptr || misaligned(ws)) return TC_ERR_INVALID_ARG;
+  if (ws_bytes < c->P.total) return TC_ERR_WORKSPACE;
+  c->ws = (char*)ws;
+  c->st = (cudaStream_t)stream;
+  return TC_OK;
+}
+
+// score: S partial sums || Gram -> eigen-solve -> C -> E
+static void enqueue_score(const Ctx& c, const void* O, const void* A, float* E, float* C, float* S,
+                          float* sigma, int32_t* rank, int32_t* img_status) {
+  const Dims& D = c.D;
+  fill_i32(img_status, D.B, 0, c.st);
+  launch_attn_colsum(D, A, (float*)(c.ws + c.P.s_part), c.st);
+  launch_gram(D, O, (float*)(c.ws + c.P.G), c.st);
+  launch_ics(D, c.P, c.ws, O, C, sigma, rank, img_status, c.st);
+  launch_combine(D, (const float*)(c.ws + c.P.s_part), C, S, E, c.st);
+}
+
+}  // namespace tc
+
+using namespace tc;
+
+extern "C" {
+
+tc_status tc_counts(const tc_params* p, int32_t* M, int32_t* P, int32_t* nA, int32_t* nB) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  if (M) *M = D.M;
+  if (P) *P = D.P;
+  if (nA) *nA = D.nA;
+  if (nB) *nB = D.nB;
+  return TC_OK;
+}
+
+tc_status tc_workspace_bytes(const tc_params* p, size_t* bytes) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  if (bytes == nullptr) return TC_ERR_INVALID_ARG;
+  *bytes = make_plan(D).total;
+  return TC_OK;
+}
+
+tc_status tc_score(const tc_params* p, const void* O, const void* A, float* E, float* C, float* S,
+                   float* sigma, int32_t* rank, int32_t* img_status, void* ws, size_t ws_bytes,
+                   void* stream) {
+  Ctx c;
+  tc_status s = open_ctx(p, ws, ws_bytes, stream, &c);
+  if (s != TC_OK) return s;
+  if (!O || !A || !E || !img_status || misaligned(O) || misaligned(A)) return TC_ERR_INVALID_ARG;
+  float* Cw = C ? C : (float*)(c.ws + c.P.C);
+  float* Sw = S ? S : (float*)(c.ws + c.P.S);
+  enqueue_score(c, O, A, E, Cw, Sw, sigma, rank, img_status);
+  return check_launch();
+}
+
+tc_status tc_prune(const tc_params* p, const float* E, int32_t* setA, int32_t* setB, void* ws,
+                   size_t ws_bytes, void* stream) {
+  Ctx c;
+  tc_status s = open_ctx(p, ws, ws_bytes, stream, &c);
+  if (s != TC_OK) return s;
+  if (!E || !setB || (c.D.nA > 0 && !setA)) return TC_ERR_INVALID_ARG;
+  launch_prune(c.D, E, setA, setB, c.st);
+  return check_launch();
+}
+
+tc_status tc_merge(const tc_params* p, const void* O, const int32_t* setA, const int32_t* setB,
+                   int32_t* merge_src, int32_t* merge_dst, int32_t* kept_idx, void* ws,
+                   size_t ws_bytes, void* stream) {
+  Ctx c;
+  tc_status s = open_ctx(p, ws, ws_bytes, stream, &c);
+  if (s != TC_OK) return s;
+  const Dims& D = c.D;
+  if (!O || !setB || !kept_idx || (D.nA > 0 && !setA) || misaligned(O)) return TC_ERR_INVALID_ARG;
+  if (D.M > 0 && (!merge_src || !merge_dst)) return TC_ERR_INVALID_ARG;
+  if ((size_t)D.d * sizeof(float) > 48 * 1024) return TC_ERR_UNSUPPORTED;
+  float* bv = (float*)(c.ws + c.P.best_val);
+  int32_t* bd = (int32_t*)(c.ws + c.P.best_dst);
+  if (D.M > 0) launch_match_rows(D, O, setA, setB, bv, bd, c.st);
+  launch_merge_select(D, setA, setB, bv, bd, merge_src, merge_dst, kept_idx, c.st);
+  return check_launch();
+}
+
+tc_status tc_compact(const tc_params* p, const void* X, const void* K, const void* V,
+                     const int32_t* kept_idx, const int32_t* merge_src, const int32_t* merge_dst,
+                     void* Xo, void* Ko, void* Vo, void* ws, size_t ws_bytes, void* stream) {
+  Ctx c;
+  tc_status s = open_ctx(p, ws, ws_bytes, stream, &c);
+  if (s != TC_OK) return s;
+  const Dims& D = c.D;
+  if (!X || !Xo || !kept_idx || misaligned(X) || misaligned(Xo)) return TC_ERR_INVALID_ARG;
+  if (D.M > 0 && (!merge_src || !merge_dst)) return TC_ERR_INVALID_ARG;
+  const bool kv = (K != nullptr);
+  if (kv != (V != nullptr) || kv != (Ko != nullptr) || kv != (Vo != nullptr)) return TC_ERR_INVALID_ARG;
+  if (kv && (misaligned(K) || misaligned(V) || misaligned(Ko) || misaligned(Vo))) return TC_ERR_INVALID_ARG;
+  launch_compact(D, X, K, V, kept_idx, merge_src, merge_dst, Xo, Ko, Vo, c.st);
+  return check_launch();
+}
+
+tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void* X, const void* K,
+                   const void* V, void* Xo, void* Ko, void* Vo, int32_t* kept_idx,
+                   int32_t* img_status, void* ws, size_t ws_bytes, void* stream) {
+  Ctx c;
+  tc_status s = open_ctx(p, ws, ws_bytes, stream, &c);
+  if (s != TC_OK) return s;
+  const Dims& D = c.D;
+  if (!O || !A || !X || !Xo || !kept_idx || !img_status) return TC_ERR_INVALID_ARG;
+  if (misaligned(O) || misaligned(A) || misaligned(X) || misaligned(Xo)) return TC_ERR_INVALID_ARG;
+  const bool kv = (K != nullptr);
+  if (kv != (V != nullptr) || kv != (Ko != nullptr) || kv != (Vo != nullptr)) return TC_ERR_INVALID_ARG;
+  if (kv && (misaligned(K) || misaligned(V) || misaligned(Ko) || misaligned(Vo))) return TC_ERR_INVALID_ARG;
+  float* E = (float*)(c.ws + c.P.E);
+  float* C = (float*)(c.ws + c.P.C);
+  float* S = (float*)(c.ws + c.P.S);
+  int32_t* setA = (int32_t*)(c.ws + c.P.setA);
+  int32_t* setB = (int32_t*)(c.ws + c.P.setB);
+  float* bv = (float*)(c.ws + c.P.best_val);
+  int32_t* bd = (int32_t*)(c.ws + c.P.best_dst);
+  int32_t* msrc = (int32_t*)(c.ws + c.P.msrc);
+  int32_t* mdst = (int32_t*)(c.ws + c.P.mdst);
+  enqueue_score(c, O, A, E, C, S, nullptr, nullptr, img_status);
+  launch_prune(D, E, setA, setB, c.st);
+  if (D.M > 0) launch_match_gram(D, (const float*)(c.ws + c.P.G), setA, setB, bv, bd, c.st);
+  launch_merge_select(D, setA, setB, bv, bd, msrc, mdst, kept_idx, c.st);
+  launch_compact(D, X, K, V, kept_idx, msrc, mdst, Xo, Ko, Vo, c.st);
+  return check_launch();
+}
+
+// ---- host-buffer variant: device staging lives at the front of the workspace ---------------
+struct HostPlan {
+  size_t O, A, X, K, V, Xo, Ko, Vo, kept, status, scratch, total;
+};
+
+static HostPlan make_host_plan(const Dims& D, size_t scratch_bytes) {
+  HostPlan h;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t B = D.B, e = D.esz;
+  h.O = take(B * D.N * D.d * e);
+  h.A = take(B * D.H * D.T * (size_t)D.N * e);
+  h.X = take(B * D.N * D.d * e);
+  h.K = take(B * D.H * D.N * (size_t)D.dh * e);
+  h.V = take(B * D.H * D.N * (size_t)D.dh * e);
+  h.Xo = take(B * D.keep * (size_t)D.d * e);
+  h.Ko = take(B * D.H * D.keep * (size_t)D.dh * e);
+  h.Vo = take(B * D.H * D.keep * (size_t)D.dh * e);
+  h.kept = take(B * D.keep * 4);
+  h.status = take(B * 4);
+  h.scratch = off;
+  h.total = off + scratch_bytes;
+  return h;
+}
+
+tc_status tc_workspace_bytes_host(const tc_params* p, size_t* bytes) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  if (bytes == nullptr) return TC_ERR_INVALID_ARG;
+  *bytes = make_host_plan(D, make_plan(D).total).total;
+  return TC_OK;
+}
+
+tc_status tc_carve_host(const tc_params* p, const void* O, const void* A, const void* X,
+                        const void* K, const void* V, void* Xo, void* Ko, void* Vo,
+                        int32_t* kept_idx, int32_t* img_status, void* ws, size_t ws_bytes,
+                        void* stream) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  const size_t scratch = make_plan(D).total;
+  HostPlan h = make_host_plan(D, scratch);
+  if (ws == nullptr || misaligned(ws)) return TC_ERR_INVALID_ARG;
+  if (ws_bytes < h.total) return TC_ERR_WORKSPACE;
+  if (!O || !A || !X || !Xo || !kept_idx || !img_status) return TC_ERR_INVALID_ARG;
+  const bool kv = (K != nullptr);
+  if (kv != (V != nullptr) || kv != (Ko != nullptr) || kv != (Vo != nullptr)) return TC_ERR_INVALID_ARG;
+  char* w = (char*)ws;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t B = D.B, e = D.esz;
+  const size_t bO = B * D.N * D.d * e, bA = B * D.H * D.T * (size_t)D.N * e;
+  const size_t bKV = B * D.H * D.N * (size_t)D.dh * e;
+  const size_t bXo = B * D.keep * (size_t)D.d * e, bKVo = B * D.H * D.keep * (size_t)D.dh * e;
+  bool ok = true;
+  ok &= cudaMemcpyAsync(w + h.O, O, bO, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(w + h.A, A, bA, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(w + h.X, X, bO, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (kv) {
+    ok &= cudaMemcpyAsync(w + h.K, K, bKV, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(w + h.V, V, bKV, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  if (!ok) return TC_ERR_CUDA;
+  s = tc_carve(p, w + h.O, w + h.A, w + h.X, kv ? w + h.K : nullptr, kv ? w + h.V : nullptr,
+               w + h.Xo, kv ? w + h.Ko : nullptr, kv ? w + h.Vo : nullptr,
+               (int32_t*)(w + h.kept), (int32_t*)(w + h.status), w + h.scratch, scratch, stream);
+  if (s != TC_OK) return s;
+  ok &= cudaMemcpyAsync(Xo, w + h.Xo, bXo, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (kv) {
+    ok &= cudaMemcpyAsync(Ko, w + h.Ko, bKVo, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(Vo, w + h.Vo, bKVo, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  }
+  ok &= cudaMemcpyAsync(kept_idx, w + h.kept, B * D.keep * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(img_status, w + h.status, B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  return ok ? TC_OK : TC_ERR_CUDA;
+}
+
+tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  if (!O || !G || misaligned(O) || misaligned(G)) return TC_ERR_INVALID_ARG;
+  s = launch_gram(D, O, G, (cudaStream_t)stream);
+  if (s != TC_OK) return s;
+  return check_launch();
+}
+
+const char* tc_status_string(int32_t status) {
+  switch (status) {
+    case TC_OK: return "ok";
+    case TC_ERR_INVALID_ARG: return "invalid argument";
+    case TC_ERR_UNSUPPORTED: return "unsupported shape";
+    case TC_ERR_WORKSPACE: return "workspace too small";
+    case TC_ERR_NOT_CONVERGED: return "eigen-solver did not converge within max_sweeps";
+    case TC_ERR_CUDA: return "CUDA runtime error";
+    case TC_ERR_RANK_CAP: return "numerical rank reached rank_cap";
+    case TC_ERR_BREAKDOWN: return "Cholesky breakdown";
+    default: return "unknown status";
+  }
+}
+
+int32_t tc_version(void) { return 100; }
+
+int32_t tc_profile_begin(void) {
+  std::lock_guard<std::mutex> lk(tc::g_prof.mu);
+  tc::g_prof.used = 0;
+  tc::g_prof.on = true;
+  return TC_OK;
+}
+
+int32_t tc_profile_end(double* ms, int64_t* launches, int32_t n) {
+  std::lock_guard<std::mutex> lk(tc::g_prof.mu);
+  tc::g_prof.on = false;
+  if (!ms || !launches || n < (int)tc::KC_COUNT) return TC_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    ms[i] = 0.0;
+    launches[i] = 0;
+  }
+  for (size_t s = 0; s < tc::g_prof.used; ++s) {
+    if (cudaEventSynchronize(tc::g_prof.ev[2 * s + 1]) != cudaSuccess) return TC_ERR_CUDA;
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, tc::g_prof.ev[2 * s], tc::g_prof.ev[2 * s + 1]) != cudaSuccess)
+      return TC_ERR_CUDA;
+    ms[tc::g_prof.cls[s]] += t;
+    launches[tc::g_prof.cls[s]] += tc::g_prof.launches_at_close[s] - tc::g_prof.launches_at_open[s];
+  }
+  tc::g_prof.used = 0;
+  return TC_OK;
+}
+
+const char* tc_kernel_class_name(int32_t cls) {
+  static const char* names[] = {"fill", "attn_colsum", "gram", "sketch", "gemm_f32", "chol_inv",
+                                "jacobi", "ics", "combine", "prune", "match", "merge_select",
+                                "compact"};
+  return (cls >= 0 && cls < (int)tc::KC_COUNT) ? names[cls] : "?";
+}
+
+int64_t tc_launch_count(void) { return (int64_t)tc::g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,564 @@
+// Dense linear algebra behind Eq. 3-5 / 3-6: the eigen-decomposition of the Gram matrix
+// G = O O^T = U Sigma^2 U^T, which yields the singular values and the rows of U Sigma that the
+// information contribution score sums.
+//
+// Two routes, chosen by rank_cap:
+//   full      one-sided Jacobi on the N x N matrix (columns of W = G J are orthogonalised; the
+//             accumulated rotations J are the eigenvectors, the column norms the eigenvalues).
+//   subspace  when the caller bounds the numerical rank by k < N: a k-dimensional dominant
+//             subspace is built (sign sketch of O, one multiplication by G, Cholesky-QR
+//             orthonormalisation), G is projected onto it (Rayleigh-Ritz) and only the k x k
+//             projection goes through Jacobi, inside shared memory.
+// All arithmetic is float32 with a fixed summation order.
+#include "tc_internal.cuh"
+
+namespace tc {
+
+// ==========================================================================================
+// Batched float32 GEMM on the plain ALUs:  C[m][n] = sum_k opA[m][k] * opB[k][n].
+//   opA[m][k] = TRA ? A[k * lda + m] : A[m * lda + k]
+//   opB[k][n] = TRB ? B[n * ldb + k] : B[k * ldb + n]
+// 64 x 64 tile per block, 16-deep slices, 4 x 4 outputs per thread.  blockIdx.z = batch.
+// ==========================================================================================
+__device__ inline float ld_f32(const float* p) { return __ldg(p); }
+__device__ inline float ld_f32(const __half* p) { return __half2float(__ldg(p)); }
+
+template <typename TA, typename TB, bool TRA, bool TRB>
+__global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
+                                                  const TB* __restrict__ B, float* __restrict__ C,
+                                                  int M, int N, int K, int lda, int ldb, int ldc,
+                                                  size_t sA, size_t sB, size_t sC) {
+  constexpr int BM = 64, BN = 64, BK = 16;
+  __shared__ float As[BK][BM + 4];
+  __shared__ float Bs[BK][BN + 4];
+  A += (size_t)blockIdx.z * sA;
+  B += (size_t)blockIdx.z * sB;
+  C += (size_t)blockIdx.z * sC;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < K; k0 += BK) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int e = tid + i * 256;
+      int m, k;
+      if (TRA) {
+        m = e & 63;
+        k = e >> 6;
+      } else {
+        k = e & 15;
+        m = e >> 4;
+      }
+      const int gm = m0 + m, gk = k0 + k;
+      float v = 0.f;
+      if (gm < M && gk < K) v = TRA ? ld_f32(A + (size_t)gk * lda + gm) : ld_f32(A + (size_t)gm * lda + gk);
+      As[k][m] = v;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int e = tid + i * 256;
+      int n, k;
+      if (TRB) {
+        k = e & 15;
+        n = e >> 4;
+      } else {
+        n = e & 63;
+        k = e >> 6;
+      }
+      const int gn = n0 + n, gk = k0 + k;
+      float v = 0.f;
+      if (gn < N && gk < K) v = TRB ? ld_f32(B + (size_t)gn * ldb + gk) : ld_f32(B + (size_t)gk * ldb + gn);
+      Bs[k][n] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[4], bb[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bb[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int gm = m0 + ty * 4 + i;
+    if (gm >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int gn = n0 + tx * 4 + j;
+      if (gn < N) C[(size_t)gm * ldc + gn] = acc[i][j];
+    }
+  }
+}
+
+template <typename TA, typename TB, bool TRA, bool TRB>
+static void gemm(const TA* A, const TB* B, float* C, int M, int N, int K, int lda, int ldb,
+                 int ldc, size_t sA, size_t sB, size_t sC, int batch, cudaStream_t st,
+                 int cls = KC_GEMM) {
+  Scope scope_(cls, st);
+  dim3 grid((N + 63) / 64, (M + 63) / 64, batch);
+  { gemm_kernel<TA, TB, TRA, TRB><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC); note_launch(); }
+}
+
+// G = O O^T for float32 inputs (and, until the tensor-core kernel takes over, float16 ones).
+tc_status launch_gram_simt(const Dims& D, const void* O, float* G, cudaStream_t st) {
+  const size_t sO = (size_t)D.N * D.d, sG = (size_t)D.N * D.N;
+  if (D.f16)
+    gemm<__half, __half, false, true>((const __half*)O, (const __half*)O, G, D.N, D.N, D.d, D.d,
+                                      D.d, D.N, sO, sO, sG, D.B, st, KC_GRAM);
+  else
+    gemm<float, float, false, true>((const float*)O, (const float*)O, G, D.N, D.N, D.d, D.d, D.d,
+                                    D.N, sO, sO, sG, D.B, st, KC_GRAM);
+  return TC_OK;
+}
+
+// ==========================================================================================
+// Sign sketch of O:  Y[x][j] = sum over columns c == j (mod k) of s(c) O[x][c],  s(c) = +-1
+// from a fixed integer hash.  grid (N, B), block k.  It only has to capture the dominant
+// column space of O; the steps after it correct it against G itself.
+// ==========================================================================================
+__device__ inline float hash_sign(uint32_t c) {
+  uint32_t h = c * 2654435761u;
+  h ^= h >> 15;
+  h *= 2246822519u;
+  h ^= h >> 13;
+  return (h & 1u) ? 1.f : -1.f;
+}
+
+template <typename T>
+__global__ void sketch_kernel(const T* __restrict__ O, float* __restrict__ Y, int N, int d, int k) {
+  const int x = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
+  if (j >= k) return;
+  const T* row = O + ((size_t)b * N + x) * d;
+  float acc = 0.f;
+  for (int c = j; c < d; c += k) acc += hash_sign((uint32_t)c) * ld_f32(row + c);
+  Y[((size_t)b * N + x) * k + j] = acc;
+}
+
+// ==========================================================================================
+// Cholesky factor of S (+ shift) and its inverse.  One block per image.
+//   S [k][k] symmetric in;  RinvT [k][k] out, RinvT[c][m] = (R^{-1})[m][c] for m <= c, else 0,
+//   where R^T R = S + shift_rel * max_i S_ii * I.  Then  Y R^{-1}  has (nearly) orthonormal
+//   columns: one pass of Cholesky-QR.  The shift keeps the factorisation alive when S is
+//   numerically singular; a later unshifted pass removes its effect.
+// The k x k work arrays live in shared memory when they fit, else in global memory.
+// ==========================================================================================
+__global__ void __launch_bounds__(512) chol_inv_kernel(const float* __restrict__ S,
+                                                      float* __restrict__ RinvT,
+                                                      float* __restrict__ Rwork, int k,
+                                                      float shift_rel, int use_smem,
+                                                      int32_t* __restrict__ status) {
+  extern __shared__ float sm[];
+  __shared__ float s_red[16];
+  __shared__ float s_piv;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const size_t kk = (size_t)k * k;
+  const float* Sb = S + b * kk;
+  float* R = use_smem ? sm : Rwork + b * kk;        // upper triangle used
+  float* XT = use_smem ? sm + kk : RinvT + b * kk;  // XT[c][m]
+  float* out = RinvT + b * kk;
+
+  float md = 0.f;
+  for (int i = tid; i < k; i += 512) md = fmaxf(md, Sb[(size_t)i * k + i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, o));
+  if (lane == 0) s_red[warp] = md;
+  __syncthreads();
+  md = s_red[0];
+  for (int w = 1; w < 16; ++w) md = fmaxf(md, s_red[w]);
+  const float shift = shift_rel * md;
+  for (size_t e = tid; e < kk; e += 512) {
+    const int r = (int)(e / k), c = (int)(e % k);
+    float v = Sb[e];
+    if (r == c) v += shift;
+    R[e] = v;
+  }
+  __syncthreads();
+
+  bool bad = false;
+  for (int j = 0; j < k; ++j) {
+    if (tid == 0) {
+      float p = R[(size_t)j * k + j];
+      if (!(p > 0.f)) {
+        p = fmaxf(md, 1e-30f) * 1e-12f;
+        bad = true;
+      }
+      s_piv = sqrtf(p);
+    }
+    __syncthreads();
+    const float dj = s_piv, inv = 1.0f / dj;
+    for (int c = j + tid; c < k; c += 512) R[(size_t)j * k + c] = (c == j) ? dj : R[(size_t)j * k + c] * inv;
+    __syncthreads();
+    for (int r = j + 1 + warp; r < k; r += 16) {
+      const float f = R[(size_t)j * k + r];
+      for (int c = r + lane; c < k; c += 32) R[(size_t)r * k + c] = fmaf(-f, R[(size_t)j * k + c], R[(size_t)r * k + c]);
+    }
+    __syncthreads();
+  }
+  if (tid == 0 && bad) atomicMax(&status[b], (int)TC_ERR_BREAKDOWN);
+
+  // inverse, one warp per column c of R^{-1}:  R x = e_c by back substitution
+  for (int c = warp; c < k; c += 16) {
+    float* x = XT + (size_t)c * k;
+    if (lane == 0) x[c] = 1.0f / R[(size_t)c * k + c];
+    __syncwarp();
+    for (int i = c - 1; i >= 0; --i) {
+      float s = 0.f;
+      for (int m = i + 1 + lane; m <= c; m += 32) s = fmaf(R[(size_t)i * k + m], x[m], s);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) x[i] = -s / R[(size_t)i * k + i];
+      __syncwarp();
+    }
+    for (int m = c + 1 + lane; m < k; m += 32) x[m] = 0.f;
+  }
+  __syncthreads();
+  if (use_smem)
+    for (size_t e = tid; e < kk; e += 512) out[e] = XT[e];
+}
+
+// ==========================================================================================
+// One-sided Jacobi eigen-solver for a symmetric positive semi-definite n x n matrix.
+// One block (16 warps) per image.  W (column-major) starts as the matrix, J as the identity;
+// each pair step rotates columns p, q of both so that the W columns become orthogonal.  At
+// convergence  W = Z Theta  and  J = Z  (eigenvectors), column norms = eigenvalues.
+// Pairs follow a round-robin tournament: n/2 disjoint pairs per round, one warp per pair,
+// a block barrier between rounds.  R = elements of a column each lane keeps in registers.
+// ==========================================================================================
+template <int R>
+__device__ inline int jacobi_pair(float* __restrict__ W, float* __restrict__ J, int n, int p,
+                                  int q, int lane, float tol, float floor2) {
+  float wp[R], wq[R];
+  float a = 0.f, bq = 0.f, g = 0.f;
+  float* Wp = W + (size_t)p * n;
+  float* Wq = W + (size_t)q * n;
+#pragma unroll
+  for (int i = 0; i < R; ++i) {
+    const int r = lane + 32 * i;
+    wp[i] = (r < n) ? Wp[r] : 0.f;
+    wq[i] = (r < n) ? Wq[r] : 0.f;
+    a = fmaf(wp[i], wp[i], a);
+    bq = fmaf(wq[i], wq[i], bq);
+    g = fmaf(wp[i], wq[i], g);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a += __shfl_xor_sync(0xffffffffu, a, o);
+    bq += __shfl_xor_sync(0xffffffffu, bq, o);
+    g += __shfl_xor_sync(0xffffffffu, g, o);
+  }
+  const float nn = sqrtf(a) * sqrtf(bq);
+  if (!(fabsf(g) > tol * nn) || !(nn > floor2)) return 0;
+  const float zeta = (bq - a) / (2.0f * g);
+  const float t = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
+  const float c = rsqrtf(fmaf(t, t, 1.0f));
+  const float s = c * t;
+#pragma unroll
+  for (int i = 0; i < R; ++i) {
+    const int r = lane + 32 * i;
+    if (r < n) {
+      Wp[r] = c * wp[i] - s * wq[i];
+      Wq[r] = fmaf(s, wp[i], c * wq[i]);
+    }
+  }
+  float* Jp = J + (size_t)p * n;
+  float* Jq = J + (size_t)q * n;
+#pragma unroll
+  for (int i = 0; i < R; ++i) {
+    const int r = lane + 32 * i;
+    if (r < n) {
+      const float jp = Jp[r], jq = Jq[r];
+      Jp[r] = c * jp - s * jq;
+      Jq[r] = fmaf(s, jp, c * jq);
+    }
+  }
+  return 1;
+}
+
+template <int R>
+__global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ Hin,
+                                                    float* __restrict__ Wg, float* __restrict__ ZTg,
+                                                    float* __restrict__ theta, int n,
+                                                    int max_sweeps, float tol, int use_smem,
+                                                    int32_t* __restrict__ status) {
+  extern __shared__ float sm[];
+  __shared__ int s_rot;
+  __shared__ float s_red[16];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const size_t nn = (size_t)n * n;
+  const float* Hb = Hin + b * nn;
+  float* W = use_smem ? sm : Wg + b * nn;
+  float* J = use_smem ? sm + nn : ZTg + b * nn;
+
+  // W = (H + H^T) / 2 (column-major == row-major for a symmetric matrix), J = I
+  float md = 0.f;
+  for (size_t e = tid; e < nn; e += 512) {
+    const int p = (int)(e / n), i = (int)(e % n);
+    const float v = 0.5f * (Hb[e] + Hb[(size_t)i * n + p]);
+    W[e] = v;
+    J[e] = (p == i) ? 1.f : 0.f;
+    if (p == i) md = fmaxf(md, fabsf(v));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, o));
+  if (lane == 0) s_red[warp] = md;
+  if (tid == 0) s_rot = 0;
+  __syncthreads();
+  md = s_red[0];
+  for (int w = 1; w < 16; ++w) md = fmaxf(md, s_red[w]);
+  // column pairs whose norms are both at the rounding floor of the largest one are left alone
+  const float floor1 = 4e-7f * md;
+  const float floor2 = floor1 * floor1;
+
+  const int ne = (n + 1) & ~1;  // even number of players; index n (if any) is a bye
+  const int m = ne - 1;
+  const int half = ne / 2;
+  int sweep = 0;
+  bool converged = false;
+  for (; sweep < max_sweeps; ++sweep) {
+    int rot = 0;
+    for (int round = 0; round < m; ++round) {
+      for (int slot = warp; slot < half; slot += 16) {
+        int u, v;
+        if (slot == 0) {
+          u = round;
+          v = m;
+        } else {
+          u = round + slot;
+          if (u >= m) u -= m;
+          v = round - slot;
+          if (v < 0) v += m;
+        }
+        if (u >= n || v >= n) continue;
+        const int p = min(u, v), q = max(u, v);
+        rot += jacobi_pair<R>(W, J, n, p, q, lane, tol, floor2);
+      }
+      __syncthreads();
+    }
+    if (lane == 0 && rot) atomicAdd(&s_rot, rot);
+    __syncthreads();
+    const int total = s_rot;
+    __syncthreads();
+    if (tid == 0) s_rot = 0;
+    if (total == 0) {
+      converged = true;
+      break;
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && !converged) atomicMax(&status[b], (int)TC_ERR_NOT_CONVERGED);
+
+  // eigenvalues = column norms of W;  eigenvectors = columns of J, written as ZT[p][i]
+  for (int p = warp; p < n; p += 16) {
+    float a = 0.f;
+    for (int r = lane; r < n; r += 32) {
+      const float v = W[(size_t)p * n + r];
+      a = fmaf(v, v, a);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) theta[(size_t)b * n + p] = sqrtf(a);
+  }
+  if (use_smem) {
+    float* out = ZTg + b * nn;
+    for (size_t e = tid; e < nn; e += 512) out[e] = J[e];
+  }
+}
+
+typedef void (*jacobi_fn)(const float*, float*, float*, float*, int, int, float, int, int32_t*);
+
+static jacobi_fn pick_jacobi(int n) {
+  const int r = (n + 31) / 32;
+  if (r <= 1) return jacobi_kernel<1>;
+  if (r <= 2) return jacobi_kernel<2>;
+  if (r <= 3) return jacobi_kernel<3>;
+  if (r <= 4) return jacobi_kernel<4>;
+  if (r <= 5) return jacobi_kernel<5>;
+  if (r <= 6) return jacobi_kernel<6>;
+  if (r <= 8) return jacobi_kernel<8>;
+  if (r <= 10) return jacobi_kernel<10>;
+  if (r <= 14) return jacobi_kernel<14>;
+  if (r <= 18) return jacobi_kernel<18>;
+  if (r <= 24) return jacobi_kernel<24>;
+  if (r <= 32) return jacobi_kernel<32>;
+  return nullptr;
+}
+
+constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared variables
+
+static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
+                          int max_sweeps, int32_t* status, cudaStream_t st) {
+  Scope scope_(KC_JACOBI, st);
+  jacobi_fn fn = pick_jacobi(n);
+  const size_t need = 2 * (size_t)n * n * sizeof(float);
+  const int use_smem = need <= SMEM_LIMIT;
+  const size_t smem = use_smem ? need : 0;
+  if (use_smem) cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const float tol = n <= 256 ? 1e-6f : 2e-6f;
+  { fn<<<batch, 512, smem, st>>>(H, W, ZT, theta, n, max_sweeps, tol, use_smem, status); note_launch(); }
+}
+
+static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
+                            float shift_rel, int32_t* status, cudaStream_t st) {
+  Scope scope_(KC_CHOL, st);
+  const size_t need = 2 * (size_t)k * k * sizeof(float);
+  const int use_smem = need <= SMEM_LIMIT;
+  const size_t smem = use_smem ? need : 0;
+  if (use_smem)
+    cudaFuncSetAttribute((const void*)chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  { chol_inv_kernel<<<batch, 512, smem, st>>>(S, RinvT, Rwork, k, shift_rel, use_smem, status); note_launch(); }
+}
+
+// ==========================================================================================
+// Eq. 3-6 and the outputs that go with it.  One block per image.
+//   theta [k]   eigenvalues of G (unsorted);  sigma_i = sqrt(theta_i)
+//   PT [k][N]   PT[p][x] = component of token x along eigenvector p (u_xp)
+//   C(x) = sum over p with sigma_p > rank_tol * sigma_max of |u_xp| sigma_p
+// ==========================================================================================
+__global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ theta,
+                                                 const float* __restrict__ PT, float* __restrict__ C,
+                                                 float* __restrict__ sigma_sorted,
+                                                 int32_t* __restrict__ rank_out,
+                                                 int32_t* __restrict__ status, int N, int k, int q,
+                                                 float rank_tol, int full) {
+  extern __shared__ float sig[];  // [k] sigma, then [k] weights (sigma or 0)
+  float* wgt = sig + k;
+  __shared__ float s_red[256];
+  __shared__ int s_cnt[256];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  float mx = 0.f;
+  for (int p = tid; p < k; p += 256) {
+    const float s = sqrtf(fmaxf(theta[(size_t)b * k + p], 0.f));
+    sig[p] = s;
+    mx = fmaxf(mx, s);
+  }
+  s_red[tid] = mx;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (tid < s) s_red[tid] = fmaxf(s_red[tid], s_red[tid + s]);
+    __syncthreads();
+  }
+  const float smax = s_red[0];
+  const float cut = rank_tol * smax;
+  int cnt = 0;
+  for (int p = tid; p < k; p += 256) {
+    const bool on = sig[p] > cut;
+    wgt[p] = on ? sig[p] : 0.f;
+    cnt += on;
+  }
+  s_cnt[tid] = cnt;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (tid < s) s_cnt[tid] += s_cnt[tid + s];
+    __syncthreads();
+  }
+  const int r = s_cnt[0];
+  if (tid == 0) {
+    if (rank_out) rank_out[b] = r;
+    if (!full && r > k - 8) atomicMax(&status[b], (int)TC_ERR_RANK_CAP);
+  }
+  const float* PTb = PT + (size_t)b * k * N;
+  for (int x = tid; x < N; x += 256) {
+    float acc = 0.f;
+    for (int p = 0; p < k; ++p) {
+      const float w = wgt[p];
+      if (w != 0.f) acc = fmaf(fabsf(PTb[(size_t)p * N + x]), w, acc);
+    }
+    C[(size_t)b * N + x] = acc;
+  }
+  if (sigma_sorted) {
+    for (int p = tid; p < k; p += 256) {
+      const float s = sig[p];
+      int pos = 0;
+      for (int o = 0; o < k; ++o) pos += (sig[o] > s) || (sig[o] == s && o < p);
+      if (pos < q) sigma_sorted[(size_t)b * q + pos] = s;
+    }
+    for (int p = k + tid; p < q; p += 256) sigma_sorted[(size_t)b * q + p] = 0.f;
+  }
+}
+
+__global__ void fill_i32_kernel(int32_t* p, int n, int v) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
+
+void fill_i32(int32_t* p, int n, int v, cudaStream_t st) {
+  Scope scope_(KC_FILL, st);
+  { fill_i32_kernel<<<(n + 255) / 256, 256, 0, st>>>(p, n, v); note_launch(); }
+}
+
+// ==========================================================================================
+// The whole of Eq. 3-5 / 3-6 for a batch, given G in the workspace.
+// ==========================================================================================
+void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_out,
+                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st) {
+  const int B = D.B, N = D.N, k = D.k;
+  float* G = (float*)(ws + P.G);
+  float* W = (float*)(ws + P.W);
+  float* ZT = (float*)(ws + P.ZT);
+  float* theta = (float*)(ws + P.sigma);
+  const int q = min(D.N, D.d);
+  const size_t sG = (size_t)N * N, sY = (size_t)N * k, sK = (size_t)k * k;
+
+  if (D.full) {
+    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, img_status, st);
+    Scope scope_(KC_ICS, st);
+    { ics_kernel<<<B, 256, 2 * (size_t)N * sizeof(float), st>>>(theta, ZT, C_out, sigma_out, rank_out,
+                                                             img_status, N, N, q, D.rank_tol, 1); note_launch(); }
+    return;
+  }
+  float* Y0 = (float*)(ws + P.Y0);
+  float* Y1 = (float*)(ws + P.Y1);
+  float* Y2 = (float*)(ws + P.Y2);
+  float* Sm = (float*)(ws + P.Sm);
+  float* Rinv = (float*)(ws + P.Rinv);
+  float* Hm = (float*)(ws + P.Hm);
+
+  // 1. sketch of the column space of O
+  {
+    Scope scope_(KC_SKETCH, st);
+    dim3 grid(N, B);
+    const int threads = (k + 31) / 32 * 32;
+    if (D.f16)
+      { sketch_kernel<__half><<<grid, threads, 0, st>>>((const __half*)O, Y0, N, D.d, k); note_launch(); }
+    else
+      { sketch_kernel<float><<<grid, threads, 0, st>>>((const float*)O, Y0, N, D.d, k); note_launch(); }
+  }
+  // one Cholesky-QR pass: dst = src R^{-1},  R^T R = src^T src (+ shift)
+  auto cholqr_pass = [&](const float* src, float* dst, float shift_rel) {
+    gemm<float, float, true, false>(src, src, Sm, k, k, N, k, k, k, sY, sY, sK, B, st);
+    launch_chol_inv(Sm, Rinv, W, k, B, shift_rel, img_status, st);
+    gemm<float, float, false, true>(src, Rinv, dst, N, k, k, k, k, k, sY, sK, sY, B, st);
+  };
+  const float kShift = 1e-6f;
+  // 2. orthonormal basis Q0 of the sketch
+  cholqr_pass(Y0, Y1, kShift);
+  cholqr_pass(Y1, Y0, 0.f);  // Q0 in Y0
+  // 3. one multiplication by G sharpens the subspace:  Y1 = G Q0, then orthonormalise
+  gemm<float, float, false, false>(G, Y0, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);
+  cholqr_pass(Y1, Y2, kShift);
+  cholqr_pass(Y2, Y1, kShift);
+  cholqr_pass(Y1, Y2, 0.f);  // Q1 in Y2
+  // 4. Rayleigh-Ritz:  H = Q1^T G Q1
+  gemm<float, float, false, false>(G, Y2, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);   // T = G Q1
+  gemm<float, float, true, false>(Y2, Y1, Hm, k, k, N, k, k, k, sY, sY, sK, B, st);   // H = Q1^T T
+  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, img_status, st);
+  // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]
+  gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
+  Scope scope_(KC_ICS, st);
+  { ics_kernel<<<B, 256, 2 * (size_t)k * sizeof(float), st>>>(theta, Y0, C_out, sigma_out, rank_out,
+                                                           img_status, N, k, q, D.rank_tol, 0); note_launch(); }
+}
+
+}  // namespace tc

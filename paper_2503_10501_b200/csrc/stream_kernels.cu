@@ -1,0 +1,293 @@
+// HBM-streaming kernels of the carve path: attention column sums (Eq. 3-7), score combination
+// (Eq. 3-8) and the merge + gather of X, K, V (Sec. 3.3.2, last paragraph).
+#include "tc_internal.cuh"
+
+namespace tc {
+
+// ------------------------------------------------------------------------------------------
+// 16-byte vector helpers: a vector holds 8 halves or 4 floats.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+struct Vec16;
+template <>
+struct Vec16<__half> {
+  static constexpr int L = 8;
+  __device__ static void unpack(const uint4& v, float* f) {
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 t = __half22float2(h[i]);
+      f[2 * i] = t.x;
+      f[2 * i + 1] = t.y;
+    }
+  }
+  __device__ static uint4 pack(const float* f) {
+    uint4 v;
+    __half2* h = reinterpret_cast<__half2*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
+    return v;
+  }
+};
+template <>
+struct Vec16<float> {
+  static constexpr int L = 4;
+  __device__ static void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x);
+    f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z);
+    f[3] = __uint_as_float(v.w);
+  }
+  __device__ static uint4 pack(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                      __float_as_uint(f[3]));
+  }
+};
+
+__device__ inline float to_f32(__half v) { return __half2float(v); }
+__device__ inline float to_f32(float v) { return v; }
+
+// ------------------------------------------------------------------------------------------
+// Eq. 3-7, first half: per image and per chunk of the H*T attention rows, the column sums.
+// grid (chunks, B); block (bx, by): x walks 16-byte column groups, y walks rows.
+// part[b][chunk][x] is written by exactly one block, in a fixed summation order.
+// ------------------------------------------------------------------------------------------
+template <typename T, bool VECTOR>
+__global__ void attn_colsum_kernel(const T* __restrict__ A, float* __restrict__ part, int R,
+                                   int N, int rows_per_chunk) {
+  constexpr int L = VECTOR ? Vec16<T>::L : 1;
+  extern __shared__ float red[];  // [by][bx * L]
+  const int b = blockIdx.y, chunk = blockIdx.x;
+  const int bx = blockDim.x, by = blockDim.y;
+  const int ncg = N / L;
+  const int r_begin = chunk * rows_per_chunk;
+  const int r_end = min(R, r_begin + rows_per_chunk);
+  const T* Ab = A + (size_t)b * R * N;
+  float* out = part + ((size_t)b * gridDim.x + chunk) * N;
+
+  for (int cg0 = 0; cg0 < ncg; cg0 += bx) {
+    const int cg = cg0 + threadIdx.x;
+    float acc[L];
+#pragma unroll
+    for (int i = 0; i < L; ++i) acc[i] = 0.f;
+    if (cg < ncg) {
+      int r = r_begin + threadIdx.y;
+      if (VECTOR) {
+        // four independent 16-byte loads in flight per thread
+        for (; r + 3 * by < r_end; r += 4 * by) {
+          uint4 v[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            v[u] = __ldg(reinterpret_cast<const uint4*>(Ab + (size_t)(r + u * by) * N) + cg);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float f[8];
+            Vec16<T>::unpack(v[u], f);
+#pragma unroll
+            for (int i = 0; i < L; ++i) acc[i] += f[i];
+          }
+        }
+        for (; r < r_end; r += by) {
+          uint4 v = __ldg(reinterpret_cast<const uint4*>(Ab + (size_t)r * N) + cg);
+          float f[8];
+          Vec16<T>::unpack(v, f);
+#pragma unroll
+          for (int i = 0; i < L; ++i) acc[i] += f[i];
+        }
+      } else {
+        for (; r < r_end; r += by) acc[0] += to_f32(Ab[(size_t)r * N + cg]);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < L; ++i) red[(threadIdx.y * bx + threadIdx.x) * L + i] = acc[i];
+    __syncthreads();
+    if (threadIdx.y == 0 && cg < ncg) {
+#pragma unroll
+      for (int i = 0; i < L; ++i) {
+        float s = 0.f;
+        for (int y = 0; y < by; ++y) s += red[(y * bx + threadIdx.x) * L + i];
+        out[cg * L + i] = s;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+void launch_attn_colsum(const Dims& D, const void* A, float* s_part, cudaStream_t st) {
+  Scope scope_(KC_ATTN, st);
+  const int R = D.H * D.T;
+  const int L = D.f16 ? 8 : 4;
+  const bool vec = (D.N % L) == 0;
+  const int ncg = vec ? D.N / L : D.N;
+  int bx = min(ncg, 128);
+  bx = (bx + 31) / 32 * 32;
+  int by = max(1, 256 / bx);
+  const int rpc = (R + D.chunks - 1) / D.chunks;
+  dim3 grid(D.chunks, D.B), block(bx, by);
+  size_t smem = (size_t)bx * by * (vec ? L : 1) * sizeof(float);
+  if (D.f16) {
+    if (vec)
+      { attn_colsum_kernel<__half, true><<<grid, block, smem, st>>>((const __half*)A, s_part, R, D.N, rpc); note_launch(); }
+    else
+      { attn_colsum_kernel<__half, false><<<grid, block, smem, st>>>((const __half*)A, s_part, R, D.N, rpc); note_launch(); }
+  } else {
+    if (vec)
+      { attn_colsum_kernel<float, true><<<grid, block, smem, st>>>((const float*)A, s_part, R, D.N, rpc); note_launch(); }
+    else
+      { attn_colsum_kernel<float, false><<<grid, block, smem, st>>>((const float*)A, s_part, R, D.N, rpc); note_launch(); }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Eq. 3-7 second half and Eq. 3-8: S = colsum / (H T);  E = (1 - lambda) C~ + lambda S~.
+// One block per image; all reductions run in a fixed order.
+// ------------------------------------------------------------------------------------------
+__device__ float block_sum_256(float v, float* sh) {
+  const int t = threadIdx.x;
+  sh[t] = v;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (t < s) sh[t] += sh[t + s];
+    __syncthreads();
+  }
+  float r = sh[0];
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ part,
+                                                     const float* __restrict__ C,
+                                                     float* __restrict__ S, float* __restrict__ E,
+                                                     int N, int chunks, float inv_rows,
+                                                     float lambda, int sum1) {
+  __shared__ float sh[256];
+  const int b = blockIdx.x;
+  const float* pb = part + (size_t)b * chunks * N;
+  float ls = 0.f, lc = 0.f;
+  for (int x = threadIdx.x; x < N; x += 256) {
+    float s = 0.f;
+    for (int c = 0; c < chunks; ++c) s += pb[(size_t)c * N + x];
+    s *= inv_rows;
+    S[(size_t)b * N + x] = s;
+    ls += s;
+    lc += C[(size_t)b * N + x];
+  }
+  float cs = 1.f, ss = 1.f;
+  if (sum1) {
+    ss = block_sum_256(ls, sh);
+    cs = block_sum_256(lc, sh);
+    if (!(ss > 0.f)) ss = 1.f;
+    if (!(cs > 0.f)) cs = 1.f;
+  }
+  __syncthreads();
+  for (int x = threadIdx.x; x < N; x += 256) {
+    float c = C[(size_t)b * N + x], s = S[(size_t)b * N + x];
+    if (sum1) {
+      c = c / cs;
+      s = s / ss;
+    }
+    E[(size_t)b * N + x] = (1.f - lambda) * c + lambda * s;
+  }
+}
+
+void launch_combine(const Dims& D, const float* s_part, const float* C, float* S, float* E,
+                    cudaStream_t st) {
+  Scope scope_(KC_COMBINE, st);
+  const float inv_rows = 1.0f / (float)(D.H * D.T);
+  { combine_kernel<<<D.B, 256, 0, st>>>(s_part, C, S, E, D.N, D.chunks, inv_rows, D.lambda,
+                                      D.score_norm == TC_NORM_SUM1 ? 1 : 0); note_launch(); }
+}
+
+// ------------------------------------------------------------------------------------------
+// Merge + gather.  grid (keep, B), block 256.  Block (j, b) produces output row j of image b
+// for X and for every head of K and V: the mean of token a = kept[j] and of every token whose
+// merge destination is a, or a bit-exact copy when nothing merges into a.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__device__ inline void merge_row(const T* __restrict__ base, size_t row_stride, int a,
+                                 const int* srcs, int cnt, T* __restrict__ out, int nvec,
+                                 int v0, int vstep) {
+  constexpr int L = Vec16<T>::L;
+  const uint4* pa = reinterpret_cast<const uint4*>(base + (size_t)a * row_stride);
+  uint4* po = reinterpret_cast<uint4*>(out);
+  for (int v = v0; v < nvec; v += vstep) {
+    uint4 va = __ldg(pa + v);
+    if (cnt == 0) {
+      po[v] = va;
+      continue;
+    }
+    float acc[8], f[8];
+    Vec16<T>::unpack(va, acc);
+    for (int s = 0; s < cnt; ++s) {
+      uint4 vs = __ldg(reinterpret_cast<const uint4*>(base + (size_t)srcs[s] * row_stride) + v);
+      Vec16<T>::unpack(vs, f);
+#pragma unroll
+      for (int i = 0; i < L; ++i) acc[i] += f[i];
+    }
+    const float den = (float)(cnt + 1);
+#pragma unroll
+    for (int i = 0; i < L; ++i) acc[i] = acc[i] / den;
+    po[v] = Vec16<T>::pack(acc);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) compact_kernel(
+    const T* __restrict__ X, const T* __restrict__ K, const T* __restrict__ V,
+    const int32_t* __restrict__ kept, const int32_t* __restrict__ msrc,
+    const int32_t* __restrict__ mdst, T* __restrict__ Xo, T* __restrict__ Ko,
+    T* __restrict__ Vo, int N, int d, int H, int dh, int keep, int M) {
+  extern __shared__ int srcs[];  // [M]
+  __shared__ int s_cnt;
+  constexpr int L = Vec16<T>::L;
+  const int b = blockIdx.y, j = blockIdx.x;
+  const int a = kept[(size_t)b * keep + j];
+  // ordered list of the sources merged into a (first warp, ballot compaction)
+  if (threadIdx.x < 32) {
+    int cnt = 0;
+    for (int m0 = 0; m0 < M; m0 += 32) {
+      const int m = m0 + threadIdx.x;
+      const bool hit = (m < M) && (mdst[(size_t)b * M + m] == a);
+      const unsigned mask = __ballot_sync(0xffffffffu, hit);
+      if (hit) srcs[cnt + __popc(mask & ((1u << threadIdx.x) - 1u))] = msrc[(size_t)b * M + m];
+      cnt += __popc(mask);
+    }
+    if (threadIdx.x == 0) s_cnt = cnt;
+  }
+  __syncthreads();
+  const int cnt = s_cnt;
+
+  // X row
+  merge_row<T>(X + (size_t)b * N * d, d, a, srcs, cnt, Xo + ((size_t)b * keep + j) * d, d / L,
+               threadIdx.x, 256);
+  // K, V rows of every head
+  if (K != nullptr) {
+    const int vpr = dh / L;
+    for (int idx = threadIdx.x; idx < H * vpr; idx += 256) {
+      const int h = idx / vpr, v = idx - h * vpr;
+      const size_t in_off = ((size_t)b * H + h) * N * dh;
+      const size_t out_off = (((size_t)b * H + h) * keep + j) * dh;
+      merge_row<T>(K + in_off, dh, a, srcs, cnt, Ko + out_off, v + 1, v, vpr + 1);
+      merge_row<T>(V + in_off, dh, a, srcs, cnt, Vo + out_off, v + 1, v, vpr + 1);
+    }
+  }
+}
+
+void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
+                    const int32_t* kept, const int32_t* msrc, const int32_t* mdst, void* Xo,
+                    void* Ko, void* Vo, cudaStream_t st) {
+  Scope scope_(KC_COMPACT, st);
+  dim3 grid(D.keep, D.B);
+  size_t smem = (size_t)max(D.M, 1) * sizeof(int);
+  if (D.f16)
+    { compact_kernel<__half><<<grid, 256, smem, st>>>(
+        (const __half*)X, (const __half*)K, (const __half*)V, kept, msrc, mdst, (__half*)Xo,
+        (__half*)Ko, (__half*)Vo, D.N, D.d, D.H, D.dh, D.keep, D.M); note_launch(); }
+  else
+    { compact_kernel<float><<<grid, 256, smem, st>>>((const float*)X, (const float*)K,
+                                                    (const float*)V, kept, msrc, mdst,
+                                                    (float*)Xo, (float*)Ko, (float*)Vo, D.N, D.d,
+                                                    D.H, D.dh, D.keep, D.M); note_launch(); }
+}
+
+}  // namespace tc

@@ -1,0 +1,93 @@
+// Internal declarations shared by the translation units of libtokencarve.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "tokencarve.h"
+
+namespace tc {
+
+// Counts of Sec. 3.3.1 / Eq. 3-9 plus everything the launchers derive from tc_params.
+struct Dims {
+  int B, N, d, H, dh, T;
+  int keep, M, P, nA, nB;
+  int k;          // dimension of the decomposed subspace: rank_cap, or N for the full solve
+  bool full;      // rank_cap == 0
+  int esz;        // bytes per element of O, A, X, K, V
+  bool f16;
+  int chunks;     // row chunks of the attention column-mean
+  int max_sweeps;
+  float lambda, rank_tol;
+  int score_norm;
+};
+
+tc_status make_dims(const tc_params* p, Dims* out);
+
+// Offsets (bytes) of every scratch array inside the caller's workspace.
+struct Plan {
+  size_t s_part;   // [B, chunks, N] f32   partial column sums of A
+  size_t S, C, E;  // [B, N] f32 each
+  size_t sigma;    // [B, k] f32 (unsorted eigenvalue norms theta)
+  size_t G;        // [B, N, N] f32
+  size_t Y0, Y1, Y2;  // [B, N, k] f32 each (subspace solve only)
+  size_t Sm, Rinv, Hm;  // [B, k, k] f32 each (subspace solve only)
+  size_t W, ZT;    // [B, k, k] f32: Jacobi work matrix and accumulated rotations (column-major)
+  size_t setA, setB, best_val, best_dst, msrc, mdst, kept;  // int32 / f32 lists
+  size_t rank;     // [B] int32
+  size_t flags;    // [B] int32 device status scratch
+  size_t total;
+};
+
+Plan make_plan(const Dims& D);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Running count of kernels this library has launched (host side, all streams).
+void note_launch(int n = 1);
+
+// Kernel classes for the optional event profile (tc_profile_begin / tc_profile_end).
+enum KernelClass {
+  KC_FILL = 0, KC_ATTN, KC_GRAM, KC_SKETCH, KC_GEMM, KC_CHOL, KC_JACOBI, KC_ICS, KC_COMBINE,
+  KC_PRUNE, KC_MATCH, KC_MSEL, KC_COMPACT, KC_COUNT
+};
+// While a profile is open, brackets the launches made in its lifetime with two CUDA events
+// on `st`; otherwise does nothing.
+struct Scope {
+  int slot;
+  cudaStream_t st;
+  Scope(int cls, cudaStream_t st);
+  ~Scope();
+};
+
+// ---- launchers (each only enqueues on `st`) ---------------------------------------------
+// Eq. 3-7: column means of A over heads and query rows.
+void launch_attn_colsum(const Dims& D, const void* A, float* s_part, cudaStream_t st);
+// Eq. 3-8 (+ the 1/(H T) of Eq. 3-7): S and E from the partial sums and C.
+void launch_combine(const Dims& D, const float* s_part, const float* C, float* S, float* E,
+                    cudaStream_t st);
+// Stage I prune + Eq. 3-9 split.
+void launch_prune(const Dims& D, const float* E, int32_t* setA, int32_t* setB, cudaStream_t st);
+// Eq. 3-10 best match per Set-B token, from the Gram matrix or from the rows of O.
+void launch_match_gram(const Dims& D, const float* G, const int32_t* setA, const int32_t* setB,
+                       float* best_val, int32_t* best_dst, cudaStream_t st);
+void launch_match_rows(const Dims& D, const void* O, const int32_t* setA, const int32_t* setB,
+                       float* best_val, int32_t* best_dst, cudaStream_t st);
+// top-M of the best similarities, merge lists, kept list.
+void launch_merge_select(const Dims& D, const int32_t* setA, const int32_t* setB,
+                         const float* best_val, const int32_t* best_dst, int32_t* msrc,
+                         int32_t* mdst, int32_t* kept, cudaStream_t st);
+// merge + gather of X, K, V.
+void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
+                    const int32_t* kept, const int32_t* msrc, const int32_t* mdst, void* Xo,
+                    void* Ko, void* Vo, cudaStream_t st);
+
+// G = O O^T (float32 out).
+tc_status launch_gram(const Dims& D, const void* O, float* G, cudaStream_t st);
+
+// Eigen-decomposition of G and Eq. 3-6:  C, theta (unsorted), then sorted sigma / rank.
+void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_out,
+                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st);
+
+}  // namespace tc

@@ -54,6 +54,7 @@ class CarveConfig:
     rho: float = 0.5
     lam: float = 0.5
     rank_tol: float = 2e-3
+    rank_cap: int = 0      # bound on the numerical rank handed to the solver (0 = full solve)
     dup_frac: float = 0.0
     near_frac: float = 0.0
     near_cos: float = 0.98
@@ -68,18 +69,19 @@ class CarveConfig:
 # The five workloads the benchmark description names (index 0 is the small one).
 CONFIGS: Dict[str, CarveConfig] = {
     "cfg1_single_f32": CarveConfig("cfg1_single_f32", 1, 576, 4096, 32, 128, 32, "f32",
-                                   rank=96, noise=0.01, tau=1.5, keep=192, seed=0),
+                                   rank=96, noise=0.01, tau=1.5, keep=192, rank_cap=128, seed=0),
     "cfg2_llava7b_f16": CarveConfig("cfg2_llava7b_f16", 16, 576, 4096, 32, 128, 64, "f16",
                                     rank=128, noise=0.01, tau=2.0, keep=128,
-                                    dup_frac=0.05, seed=2),
+                                    rank_cap=160, dup_frac=0.05, seed=2),
     "cfg3_llava13b_f16": CarveConfig("cfg3_llava13b_f16", 16, 576, 5120, 40, 128, 64, "f16",
                                      rank=160, noise=0.02, tau=2.0, keep=64,
-                                     hot=8, hot_bias=4.0, seed=3),
+                                     rank_cap=192, hot=8, hot_bias=4.0, seed=3),
     "cfg4_anyres_f16": CarveConfig("cfg4_anyres_f16", 4, 2880, 4096, 32, 128, 128, "f16",
                                    rank=384, noise=0.01, tau=2.0, keep=640,
-                                   near_frac=0.10, seed=4),
+                                   rank_cap=448, near_frac=0.10, seed=4),
     "cfg5_sweep_f16": CarveConfig("cfg5_sweep_f16", 64, 576, 4096, 32, 128, 128, "f16",
-                                  rank=128, noise=0.01, tau=2.0, keep=128, seed=5),
+                                  rank=128, noise=0.01, tau=2.0, keep=128, rank_cap=160,
+                                  seed=5),
 }
 
 

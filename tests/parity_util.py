@@ -1,0 +1,155 @@
+"""Comparison of the CUDA path with the float64 oracle, stage by stage, on one image.
+
+Rules (written out here so the tolerances are visible in the tests):
+  * S, C, E, sigma_i (i <= r): relative error <= 1e-3; sigma beyond r: within 1e-3 * sigma_1.
+  * Index results are compared exactly, except for tokens inside a band the floating-point
+    scores cannot resolve: a token may sit on either side of a cut (Stage-I cut, A/B cut) only
+    if its oracle score is within 1e-3 relative of the score at that cut; a Set-B token may be
+    in or out of the merge set only if its best similarity is within 1e-4 of the similarity at
+    the merge cut; its destination may differ only among Set-A tokens whose similarity is
+    within 1e-4 of the best.  Every later stage is then checked against the oracle run on the
+    CUDA path's own earlier decision, so one allowed flip cannot hide a later error.
+  * X', K', V': absolute error <= 2e-2 in the storage type, and exact where nothing merges.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import numpy as np
+
+from oracle import ipgs_oracle as orc
+
+REL_SCORE = 1e-3
+SIM_BAND = 1e-4
+ABS_OUT = 2e-2
+
+
+def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+    ref = np.asarray(ref, np.float64)
+    got = np.asarray(got, np.float64)
+    den = np.maximum(np.abs(ref), 1e-300)
+    return float(np.max(np.abs(got - ref) / den)) if ref.size else 0.0
+
+
+def check_scores(g: Dict[str, np.ndarray], o: Dict[str, np.ndarray], rank_tol: float) -> None:
+    """g: CUDA outputs of one image (E, C, S, sigma, rank); o: oracle.score() result."""
+    assert rel_err(g["S"], o["S"]) <= REL_SCORE, ("S", rel_err(g["S"], o["S"]))
+    r = int(o["rank"])
+    assert int(g["rank"]) == r, ("rank", int(g["rank"]), r)
+    sig_o = o["sigma"]
+    assert rel_err(g["sigma"][:r], sig_o[:r]) <= REL_SCORE, ("sigma", rel_err(g["sigma"][:r], sig_o[:r]))
+    if len(sig_o) > r:
+        assert np.max(np.abs(g["sigma"][r:len(sig_o)] - sig_o[r:])) <= REL_SCORE * sig_o[0], "sigma tail"
+    assert rel_err(g["C"], o["C"]) <= REL_SCORE, ("C", rel_err(g["C"], o["C"]))
+    assert rel_err(g["E"], o["E"]) <= REL_SCORE, ("E", rel_err(g["E"], o["E"]))
+
+
+def check_sets(E_or: np.ndarray, setA_g, setB_g, P: int, nA: int) -> int:
+    """Exact agreement outside the unresolvable band; returns the number of in-band flips."""
+    N = len(E_or)
+    E32 = np.asarray(E_or, np.float64).astype(np.float32).astype(np.float64)
+    order = orc.descending_order(E_or)
+    cls_o = np.zeros(N, np.int8)
+    cls_o[order[:nA]] = 1
+    cls_o[order[nA:P]] = 2
+    cls_g = np.zeros(N, np.int8)
+    setA_g = np.asarray(setA_g)
+    setB_g = np.asarray(setB_g)
+    assert len(setA_g) == nA and len(setB_g) == P - nA
+    assert np.all(np.diff(setA_g) > 0) and np.all(np.diff(setB_g) > 0), "lists must ascend"
+    assert len(set(setA_g.tolist()) & set(setB_g.tolist())) == 0
+    cls_g[setA_g] = 1
+    cls_g[setB_g] = 2
+    cuts = []
+    for c in (nA, P):
+        if 0 < c < N:
+            cuts.append(0.5 * (E32[order[c - 1]] + E32[order[c]]))
+    flips = 0
+    for x in np.nonzero(cls_o != cls_g)[0]:
+        ok = any(abs(E32[x] - v) <= REL_SCORE * abs(v) for v in cuts)
+        assert ok, f"token {x}: oracle class {cls_o[x]}, CUDA class {cls_g[x]}, E={E32[x]}, cuts={cuts}"
+        flips += 1
+    return flips
+
+
+def check_merge(O: np.ndarray, setA, setB, M: int, src_g, dst_g, kept_g, keep: int) -> int:
+    """Oracle matching on the given sets against the CUDA lists; returns in-band flips."""
+    setA = [int(a) for a in setA]
+    setB = [int(b) for b in setB]
+    src_g = np.asarray(src_g)
+    dst_g = np.asarray(dst_g)
+    kept_g = np.asarray(kept_g)
+    assert len(src_g) == M and len(dst_g) == M and len(kept_g) == keep
+    flips = 0
+    if M > 0:
+        assert np.all(np.diff(src_g) > 0), "merge_src must ascend"
+        sim = orc.similarity(O, setA, setB)
+        best = sim.max(axis=1)
+        src_o, dst_o = orc.match_and_select(sim, setA, setB, M)
+        order = sorted(range(len(setB)), key=lambda j: (-float(np.float32(best[j])), setB[j]))
+        cut = 0.5 * (best[order[M - 1]] + best[order[M]]) if M < len(setB) else -np.inf
+        pos = {b: j for j, b in enumerate(setB)}
+        for b in set(src_o.tolist()) ^ set(src_g.tolist()):
+            assert b in pos and abs(best[pos[b]] - cut) <= SIM_BAND, f"merge set differs at token {b}"
+            flips += 1
+        dmap_o = dict(zip(src_o.tolist(), dst_o.tolist()))
+        colA = {a: i for i, a in enumerate(setA)}
+        for b, a in zip(src_g.tolist(), dst_g.tolist()):
+            assert b in pos and a in colA, "merge pair outside the sets"
+            row = sim[pos[b]]
+            if dmap_o.get(b, None) != a:
+                assert row.max() - row[colA[a]] <= SIM_BAND, f"destination of {b}: {a} is not a best match"
+                # a bit-identical alternative must respect the lower-index rule
+                exact = [x for x in setA if row[colA[x]] == row[colA[a]] and np.array_equal(O[x], O[a])]
+                assert a == min(exact), f"tie among identical rows must go to the lower index ({b}->{a})"
+                flips += 1
+    expect_kept = sorted(set(setA) | (set(setB) - set(src_g.tolist())))
+    assert kept_g.tolist() == expect_kept, "kept_idx != Set A + unmerged Set B, ascending"
+    return flips
+
+
+def check_compact(X, K, V, kept, src, dst, Xo_g, Ko_g, Vo_g) -> None:
+    ref = orc.compact(X, K, V, kept, src, dst, X.dtype)
+    dests = set(int(t) for t in dst)
+    plain = np.array([int(a) not in dests for a in kept])
+    for name, got, want in (("X", Xo_g, ref["X"]), ("K", Ko_g, ref["K"]), ("V", Vo_g, ref["V"])):
+        if want is None:
+            assert got is None
+            continue
+        got = np.asarray(got)
+        assert got.shape == want.shape and got.dtype == want.dtype, name
+        err = np.max(np.abs(got.astype(np.float64) - want.astype(np.float64))) if got.size else 0.0
+        assert err <= ABS_OUT, (name, err)
+        # rows nothing merges into are copies
+        if name == "X":
+            assert np.array_equal(got[plain], want[plain]), "unmerged rows must be bit-exact copies"
+        else:
+            assert np.array_equal(got[:, plain], want[:, plain]), "unmerged rows must be bit-exact copies"
+        # a merged row is at most one unit in the last place of the storage type away
+        # (float32 storage: the float32 accumulation of a few terms adds a few more)
+        n_ulp = 1.0 if want.dtype == np.float16 else 4.0
+        ulp = np.spacing(np.abs(want).astype(want.dtype)).astype(np.float64)
+        assert np.all(np.abs(got.astype(np.float64) - want.astype(np.float64)) <= n_ulp * ulp + 1e-30), name
+
+
+def oracle_scores(cfgp, O, A) -> Dict[str, np.ndarray]:
+    return orc.score(O.astype(np.float64), A.astype(np.float64), cfgp["lam"], cfgp["rank_tol"],
+                     cfgp["score_norm"])
+
+
+def check_image(cfgp: dict, im: Dict[str, np.ndarray], g: Dict[str, np.ndarray],
+                with_scores: bool = True) -> Dict[str, int]:
+    """Full staged comparison of one image.  cfgp: keep, rho, n_merge, lam, rank_tol, score_norm.
+    im: O, A, X, K, V (storage dtype).  g: CUDA results of that image: E, C, S, sigma, rank, setA,
+    setB, src, dst, kept, Xo, Ko, Vo."""
+    N = im["O"].shape[0]
+    M, P, nA, nB = orc.resolve_counts(N, cfgp["keep"], cfgp["rho"], cfgp.get("n_merge", -1))
+    o = oracle_scores(cfgp, im["O"], im["A"])
+    if with_scores:
+        check_scores(g, o, cfgp["rank_tol"])
+    flips_sets = check_sets(o["E"], g["setA"], g["setB"], P, nA)
+    flips_merge = check_merge(im["O"].astype(np.float64), g["setA"], g["setB"], M, g["src"],
+                              g["dst"], g["kept"], cfgp["keep"])
+    check_compact(im["X"], im.get("K"), im.get("V"), g["kept"], g["src"], g["dst"], g["Xo"],
+                  g.get("Ko"), g.get("Vo"))
+    return {"flips_sets": flips_sets, "flips_merge": flips_merge}

@@ -1,0 +1,185 @@
+"""CUDA path against the float64 oracle, through the C ABI, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ipgs_oracle as orc
+from paper_2503_10501_b200 import binding as tcb
+from paper_2503_10501_b200 import inputs
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def dev(a):
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def host(t):
+    return None if t is None else t.cpu().numpy()
+
+
+def params_of(cfg, **over):
+    kw = dict(batch=cfg.batch, n_tokens=cfg.n_tokens, d_model=cfg.d_model, n_heads=cfg.n_heads,
+              head_dim=cfg.head_dim, n_query=cfg.n_query, keep=cfg.keep, rho=cfg.rho, lam=cfg.lam,
+              rank_tol=cfg.rank_tol, dtype=cfg.dtype, rank_cap=cfg.rank_cap)
+    kw.update(over)
+    return tcb.Params(**kw)
+
+
+def run_staged(p, batch, with_kv=True):
+    """Every stage through its own entry point, each fed with the previous stage's CUDA output."""
+    O, A, X = dev(batch["O"]), dev(batch["A"]), dev(batch["X"])
+    K = dev(batch["K"]) if with_kv else None
+    V = dev(batch["V"]) if with_kv else None
+    ws = tcb.workspace(p)
+    sc = tcb.tc_score(p, O, A, ws)
+    setA, setB = tcb.tc_prune(p, sc["E"], ws)
+    src, dst, kept = tcb.tc_merge(p, O, setA, setB, ws)
+    Xo, Ko, Vo = tcb.tc_compact(p, X, K, V, kept, src, dst, ws)
+    cX, cK, cV, ckept, cstatus = tcb.tc_carve(p, O, A, X, K, V, ws)
+    torch.cuda.synchronize()
+    res = {k: host(v) for k, v in sc.items()}
+    res.update(setA=host(setA), setB=host(setB), src=host(src), dst=host(dst), kept=host(kept),
+               Xo=host(Xo), Ko=host(Ko), Vo=host(Vo), cX=host(cX), cK=host(cK), cV=host(cV),
+               ckept=host(ckept), cstatus=host(cstatus))
+    return res
+
+
+def image_slice(res, b, with_kv=True):
+    g = {k: res[k][b] for k in ("E", "C", "S", "sigma", "rank", "setA", "setB", "src", "dst",
+                                "kept", "Xo")}
+    g["Ko"] = res["Ko"][b] if with_kv else None
+    g["Vo"] = res["Vo"][b] if with_kv else None
+    return g
+
+
+def cfgp_of(p):
+    return dict(keep=p.keep, rho=p.rho, n_merge=p.n_merge, lam=p.lam, rank_tol=p.rank_tol,
+                score_norm=p.score_norm)
+
+
+def check_config(cfg, images, with_kv=True, **over):
+    p = params_of(cfg, **over)
+    batch = inputs.make_batch(cfg)
+    res = run_staged(p, batch, with_kv)
+    assert np.all(res["img_status"] == 0), res["img_status"]
+    assert np.all(res["cstatus"] == 0), res["cstatus"]
+    # the fused call must reproduce the staged calls
+    assert np.array_equal(res["ckept"], res["kept"])
+    assert np.array_equal(res["cX"], res["Xo"])
+    if with_kv:
+        assert np.array_equal(res["cK"], res["Ko"]) and np.array_equal(res["cV"], res["Vo"])
+    flips = {"flips_sets": 0, "flips_merge": 0}
+    for b in images:
+        im = {k: batch[k][b] for k in batch}
+        if not with_kv:
+            im.pop("K"), im.pop("V")
+        f = pu.check_image(cfgp_of(p), im, image_slice(res, b, with_kv))
+        for k in f:
+            flips[k] += f[k]
+    return flips
+
+
+# ------------------------------------------------------------------ tiny shapes, full solve
+@pytest.mark.parametrize("N,d,keep,rho,lam,norm,dtype", [
+    (12, 16, 4, 0.5, 0.5, "none", "f32"),
+    (16, 32, 7, 0.5, 0.0, "none", "f32"),
+    (24, 16, 9, 0.3, 1.0, "none", "f32"),      # N > d: rank <= d
+    (33, 64, 11, 1.0, 0.5, "sum1", "f32"),     # odd N (bye column in the tournament)
+    (64, 128, 20, 0.5, 0.5, "sum1", "f16"),
+    (40, 64, 40, 0.5, 0.5, "none", "f16"),     # keep = N: nothing pruned or merged
+    (40, 64, 1, 0.0, 0.5, "none", "f16"),      # keep = 1, rho = 0: Set A empty
+    (40, 64, 1, 1.0, 0.5, "none", "f16"),
+    (50, 64, 10, 0.0, 0.5, "none", "f16"),     # rho = 0: pure gather
+])
+def test_tiny_full_solve(N, d, keep, rho, lam, norm, dtype):
+    cfg = inputs.tiny_config(n_tokens=N, d_model=d, n_heads=2, head_dim=8, n_query=5, keep=keep,
+                             rank=min(N, d) // 2, dtype=dtype, batch=3, seed=17 + N, noise=0.3,
+                             rho=rho, lam=lam, rank_tol=0.0)
+    check_config(cfg, range(3), score_norm=norm)
+
+
+def test_without_kv_and_with_n_merge_override():
+    cfg = inputs.tiny_config(n_tokens=48, d_model=64, n_heads=2, head_dim=8, n_query=4, keep=13,
+                             rank=20, dtype="f16", batch=2, seed=5, noise=0.3, rank_tol=0.0)
+    check_config(cfg, range(2), with_kv=False)
+    check_config(cfg, range(2), n_merge=3)
+
+
+# ------------------------------------------------------------------ medium, ragged against every tile
+@pytest.mark.parametrize("rank_cap", [0, 96])
+def test_medium_ragged(rank_cap):
+    cfg = inputs.tiny_config(n_tokens=200, d_model=264, n_heads=3, head_dim=24, n_query=37, keep=61,
+                             rank=40, dtype="f16", batch=5, seed=23, noise=0.01, tau=2.0,
+                             rank_tol=2e-3, dup_frac=0.05)
+    check_config(cfg, range(5), rank_cap=rank_cap)
+
+
+# ------------------------------------------------------------------ selection kernels alone
+def test_prune_exact_with_ties():
+    rng = np.random.default_rng(3)
+    N, B = 576, 4
+    p = tcb.Params(batch=B, n_tokens=N, d_model=64, n_heads=1, head_dim=8, n_query=1, keep=128)
+    M, P, nA, nB = tcb.tc_counts(p)
+    E = rng.integers(0, 40, size=(B, N)).astype(np.float32) / 8.0      # many exact ties
+    E[1] = 1.0                                                          # all equal
+    E[2, ::3] *= -1.0                                                   # negative scores
+    setA, setB = tcb.tc_prune(p, dev(E))
+    torch.cuda.synchronize()
+    for b in range(B):
+        a_o, b_o = orc.prune_split(E[b].astype(np.float64), P, nA)
+        assert host(setA)[b].tolist() == sorted(a_o.tolist())
+        assert host(setB)[b].tolist() == sorted(b_o.tolist())
+
+
+def test_merge_duplicate_rows_tie_to_lower_index():
+    # Set A holds two bit-identical rows; the Set-B twin of both must pick the lower index.
+    N, d = 32, 64
+    rng = np.random.default_rng(9)
+    O = rng.standard_normal((1, N, d)).astype(np.float16)
+    O[0, 20] = O[0, 5]
+    O[0, 11] = O[0, 5]
+    p = tcb.Params(batch=1, n_tokens=N, d_model=d, n_heads=1, head_dim=8, n_query=1, keep=6,
+                   n_merge=2)
+    M, P, nA, nB = tcb.tc_counts(p)            # P = 8, nA = 4, nB = 4
+    setA = np.array([[3, 5, 20, 30]], np.int32)
+    setB = np.array([[7, 11, 12, 25]], np.int32)
+    src, dst, kept = tcb.tc_merge(p, dev(O), dev(setA), dev(setB))
+    torch.cuda.synchronize()
+    src, dst, kept = host(src)[0], host(dst)[0], host(kept)[0]
+    assert 11 in src.tolist() and dst[src.tolist().index(11)] == 5
+    pu.check_merge(O[0].astype(np.float64), setA[0], setB[0], M, src, dst, kept, 6)
+
+
+# ------------------------------------------------------------------ the named workloads
+def test_cfg1_single_f32():
+    cfg = inputs.CONFIGS["cfg1_single_f32"]
+    check_config(cfg, [0])
+    check_config(cfg, [0], score_norm="sum1")
+
+
+@pytest.mark.parametrize("lam,norm", [(0.5, "none"), (0.5, "sum1"), (0.0, "none"), (1.0, "none")])
+def test_cfg2_llava7b(lam, norm):
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"]
+    check_config(cfg, [0, 7, 15], lam=lam, score_norm=norm)
+
+
+@pytest.mark.parametrize("norm", ["none", "sum1"])
+def test_cfg3_llava13b(norm):
+    cfg = inputs.CONFIGS["cfg3_llava13b_f16"]
+    check_config(cfg, [1, 14], score_norm=norm)
+
+
+def test_cfg2_full_solve_agrees():
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=2)
+    check_config(cfg, [0, 1], rank_cap=0)
+
+
+def test_rank_cap_too_small_is_reported():
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=1)
+    p = params_of(cfg, rank_cap=96)          # the numerical rank is 128
+    batch = inputs.make_batch(cfg, "OA")
+    sc = tcb.tc_score(p, dev(batch["O"]), dev(batch["A"]))
+    torch.cuda.synchronize()
+    assert host(sc["img_status"])[0] == 6
