@@ -238,7 +238,8 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const float* __restrict__
 // ==========================================================================================
 template <int R>
 __device__ inline int jacobi_pair(float* __restrict__ W, float* __restrict__ J, int n, int p,
-                                  int q, int lane, float tol, float floor2) {
+                                  int q, int lane, float tol, float floor2,
+                                  float count_floor2) {
   float wp[R], wq[R];
   float a = 0.f, bq = 0.f, g = 0.f;
   float* Wp = W + (size_t)p * n;
@@ -259,7 +260,7 @@ __device__ inline int jacobi_pair(float* __restrict__ W, float* __restrict__ J, 
     g += __shfl_xor_sync(0xffffffffu, g, o);
   }
   const float nn = sqrtf(a) * sqrtf(bq);
-  if (!(fabsf(g) > tol * nn) || !(nn > floor2)) return 0;
+  if (!(fabsf(g) > tol * nn) || !(fmaxf(a, bq) > floor2)) return 0;
   const float zeta = (bq - a) / (2.0f * g);
   const float t = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
   const float c = rsqrtf(fmaf(t, t, 1.0f));
@@ -283,7 +284,9 @@ __device__ inline int jacobi_pair(float* __restrict__ W, float* __restrict__ J, 
       Jq[r] = fmaf(s, jp, c * jq);
     }
   }
-  return 1;
+  // a rotation between two columns that both lie under the rank cut-off does not delay
+  // convergence: neither column enters Eq. 3-6
+  return fmaxf(a, bq) > count_floor2 ? 1 : 0;
 }
 
 template <int R>
@@ -291,7 +294,8 @@ __global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ H
                                                     float* __restrict__ Wg, float* __restrict__ ZTg,
                                                     float* __restrict__ theta, int n,
                                                     int max_sweeps, float tol, int use_smem,
-                                                    int32_t* __restrict__ status) {
+                                                    int32_t* __restrict__ status, float floor_rel,
+                                                    float count_rel) {
   extern __shared__ float sm[];
   __shared__ int s_rot;
   __shared__ float s_red[16];
@@ -317,9 +321,12 @@ __global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ H
   __syncthreads();
   md = s_red[0];
   for (int w = 1; w < 16; ++w) md = fmaxf(md, s_red[w]);
-  // column pairs whose norms are both at the rounding floor of the largest one are left alone
-  const float floor1 = 4e-7f * md;
+  // column pairs whose norms (eigenvalue estimates) are BOTH below the floor are left alone:
+  // they are rounding noise of the largest eigenvalue, or lie below the rank cut-off, and
+  // rotating them against each other only slows convergence
+  const float floor1 = floor_rel * md;
   const float floor2 = floor1 * floor1;
+  const float count_floor2 = (count_rel * md) * (count_rel * md);
 
   const int ne = (n + 1) & ~1;  // even number of players; index n (if any) is a bye
   const int m = ne - 1;
@@ -342,7 +349,7 @@ __global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ H
         }
         if (u >= n || v >= n) continue;
         const int p = min(u, v), q = max(u, v);
-        rot += jacobi_pair<R>(W, J, n, p, q, lane, tol, floor2);
+        rot += jacobi_pair<R>(W, J, n, p, q, lane, tol, floor2, count_floor2);
       }
       __syncthreads();
     }
@@ -376,7 +383,7 @@ __global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ H
   }
 }
 
-typedef void (*jacobi_fn)(const float*, float*, float*, float*, int, int, float, int, int32_t*);
+typedef void (*jacobi_fn)(const float*, float*, float*, float*, int, int, float, int, int32_t*, float, float);
 
 static jacobi_fn pick_jacobi(int n) {
   const int r = (n + 31) / 32;
@@ -398,15 +405,22 @@ static jacobi_fn pick_jacobi(int n) {
 constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared variables
 
 static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
-                          int max_sweeps, int32_t* status, cudaStream_t st) {
+                          int max_sweeps, float rank_tol, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_JACOBI, st);
   jacobi_fn fn = pick_jacobi(n);
   const size_t need = 2 * (size_t)n * n * sizeof(float);
   const int use_smem = need <= SMEM_LIMIT;
   const size_t smem = use_smem ? need : 0;
   if (use_smem) cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  const float tol = n <= 256 ? 1e-6f : 2e-6f;
-  { fn<<<batch, 512, smem, st>>>(H, W, ZT, theta, n, max_sweeps, tol, use_smem, status); note_launch(); }
+  // off-diagonal threshold a little above the rounding noise of a length-n float32 dot product
+  const float tol = fmaxf(1e-6f, 2.5f * sqrtf((float)n) * 1.1920929e-7f);
+  // Eigenvalue floors, relative to the largest diagonal entry.  Column pairs that are both
+  // under the float32 rounding level of that entry are never rotated; rotations between two
+  // columns that are both under the eigenvalue rank_tol cuts at are done but do not count
+  // towards "this sweep still rotated".
+  const float floor_rel = 1e-6f;
+  const float count_rel = fmaxf(floor_rel, rank_tol * rank_tol);
+  { fn<<<batch, 512, smem, st>>>(H, W, ZT, theta, n, max_sweeps, tol, use_smem, status, floor_rel, count_rel); note_launch(); }
 }
 
 static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
@@ -451,12 +465,20 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
   }
   const float smax = s_red[0];
   const float cut = rank_tol * smax;
+  // O has at most q = min(N, d) non-zero singular values: only the q largest eigenvalues of G
+  // can be one, whatever rounding left in the others.
   int cnt = 0;
   for (int p = tid; p < k; p += 256) {
-    const bool on = sig[p] > cut;
-    wgt[p] = on ? sig[p] : 0.f;
+    const float s = sig[p];
+    int pos = 0;
+    for (int o = 0; o < k; ++o) pos += (sig[o] > s) || (sig[o] == s && o < p);
+    const bool on = (s > cut) && (pos < q);
+    wgt[p] = on ? s : 0.f;
     cnt += on;
+    if (sigma_sorted && pos < q) sigma_sorted[(size_t)b * q + pos] = s;
   }
+  if (sigma_sorted)
+    for (int p = k + tid; p < q; p += 256) sigma_sorted[(size_t)b * q + p] = 0.f;
   s_cnt[tid] = cnt;
   __syncthreads();
   for (int s = 128; s > 0; s >>= 1) {
@@ -476,15 +498,6 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
       if (w != 0.f) acc = fmaf(fabsf(PTb[(size_t)p * N + x]), w, acc);
     }
     C[(size_t)b * N + x] = acc;
-  }
-  if (sigma_sorted) {
-    for (int p = tid; p < k; p += 256) {
-      const float s = sig[p];
-      int pos = 0;
-      for (int o = 0; o < k; ++o) pos += (sig[o] > s) || (sig[o] == s && o < p);
-      if (pos < q) sigma_sorted[(size_t)b * q + pos] = s;
-    }
-    for (int p = k + tid; p < q; p += 256) sigma_sorted[(size_t)b * q + p] = 0.f;
   }
 }
 
@@ -512,7 +525,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_
   const size_t sG = (size_t)N * N, sY = (size_t)N * k, sK = (size_t)k * k;
 
   if (D.full) {
-    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, img_status, st);
+    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, img_status, st);
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<B, 256, 2 * (size_t)N * sizeof(float), st>>>(theta, ZT, C_out, sigma_out, rank_out,
                                                              img_status, N, N, q, D.rank_tol, 1); note_launch(); }
@@ -553,7 +566,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_
   // 4. Rayleigh-Ritz:  H = Q1^T G Q1
   gemm<float, float, false, false>(G, Y2, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);   // T = G Q1
   gemm<float, float, true, false>(Y2, Y1, Hm, k, k, N, k, k, k, sY, sY, sK, B, st);   // H = Q1^T T
-  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, img_status, st);
+  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, img_status, st);
   // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]
   gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
   Scope scope_(KC_ICS, st);
