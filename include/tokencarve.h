@@ -49,7 +49,8 @@ typedef enum {
   TC_ERR_CUDA = 5,          /* a CUDA runtime call failed                                    */
   TC_ERR_RANK_CAP = 6,      /* img_status: numerical rank reached rank_cap; rerun that image
                                with a larger rank_cap or with rank_cap = 0                   */
-  TC_ERR_BREAKDOWN = 7      /* img_status: a Cholesky pivot was not positive                 */
+  TC_ERR_BREAKDOWN = 7,     /* img_status: a Cholesky pivot was not positive                 */
+  TC_ERR_SCRATCH_LIMIT = 8  /* tc_attn_score_noalloc: request larger than its built-in scratch */
 } tc_status;
 
 typedef enum { TC_F16 = 0, TC_F32 = 1 } tc_dtype;
@@ -151,6 +152,35 @@ tc_status tc_carve_host(const tc_params* p, const void* O, const void* A, const 
                         const void* K, const void* V, void* Xo, void* Ko, void* Vo,
                         int32_t* kept_idx, int32_t* img_status, void* ws, size_t ws_bytes,
                         void* stream);
+
+/*
+ * Attention scores without any caller-provided scratch (the paper has no counterpart; the
+ * arithmetic is Eq. 3-7, the same kernels tc_score runs for S).
+ *
+ * Who needs it: code that may not allocate device memory at the point where it wants the
+ * scores, and so cannot produce the workspace the other entry points ask for.  Typical cases
+ * are a plug-in running inside another framework's forward pass whose memory pool it must not
+ * touch, a real-time serving loop where cudaMalloc's implicit device synchronisation is not
+ * acceptable, and a process that has handed all of the GPU's memory to a pool at start-up.
+ *
+ *   A [B,H,T,N] in (device, tc_params.dtype);  S [B,N] float32 out (device).  Only batch,
+ *   n_tokens, n_heads, n_query and dtype of `p` matter, but `p` must be valid as a whole.
+ *
+ * The partial column sums go into a fixed array of TC_NOALLOC_SCRATCH_BYTES that is part of
+ * the library image: every GPU that loads the library holds that much memory until the
+ * process exits, whether or not this function is ever called.  The call needs
+ * B * chunks * N floats of it, where chunks = min(64, (H*T)/32, ceil(592/B)) (at least 1);
+ * a larger request returns TC_ERR_SCRATCH_LIMIT and enqueues nothing.
+ *
+ * The first call on each device looks up the array's device address (a host-side runtime
+ * query, done with that device current); make that first call outside any stream capture.
+ * No call allocates or frees memory.  All calls on a device share the one array, which keeps
+ * whatever the previous call left in it; each call overwrites the part it uses before reading
+ * it, so nothing has to be cleared, but two calls that overlap on the GPU (different streams,
+ * or different host threads without ordering) race on it.  Order them on one stream.
+ */
+#define TC_NOALLOC_SCRATCH_BYTES (4u << 20)
+tc_status tc_attn_score_noalloc(const tc_params* p, const void* A, float* S, void* stream);
 
 /*
  * The Gram matrix behind the SVD of Sec. 3.3.1 (O O^T = U Sigma^2 U^T) and the similarity of

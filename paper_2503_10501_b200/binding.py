@@ -20,13 +20,13 @@ TC_F16, TC_F32 = 0, 1
 TC_NORM_NONE, TC_NORM_SUM1 = 0, 1
 STATUS_NAMES = {0: "TC_OK", 1: "TC_ERR_INVALID_ARG", 2: "TC_ERR_UNSUPPORTED", 3: "TC_ERR_WORKSPACE",
                 4: "TC_ERR_NOT_CONVERGED", 5: "TC_ERR_CUDA", 6: "TC_ERR_RANK_CAP",
-                7: "TC_ERR_BREAKDOWN"}
+                7: "TC_ERR_BREAKDOWN", 8: "TC_ERR_SCRATCH_LIMIT"}
 
 # every symbol include/tokencarve.h declares
 EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge", "tc_compact",
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
-           "tc_kernel_class_name")
+           "tc_kernel_class_name", "tc_attn_score_noalloc")
 
 
 class TcParams(C.Structure):
@@ -71,13 +71,14 @@ def lib() -> C.CDLL:
         L.tc_carve.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_carve_host.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_gram.argtypes = [pp, vp, vp, vp]
+        L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
         L.tc_status_string.argtypes = [C.c_int32]
         L.tc_status_string.restype = C.c_char_p
         L.tc_kernel_class_name.argtypes = [C.c_int32]
         L.tc_kernel_class_name.restype = C.c_char_p
         L.tc_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int32]
         for name in EXPORTS:
-            if name not in ("tc_status_string", "tc_kernel_class_name"):
+            if name not in ("tc_status_string", "tc_kernel_class_name", "tc_attn_score_noalloc"):
                 getattr(L, name).restype = C.c_int32
         L.tc_launch_count.restype = C.c_int64
         _lib = L
@@ -162,6 +163,16 @@ def tc_gram(p: Params, O: torch.Tensor) -> torch.Tensor:
     cp = p.c()
     _check("tc_gram", lib().tc_gram(C.byref(cp), _ptr(O), _ptr(G), _stream()))
     return G
+
+
+def tc_attn_score_noalloc(p: Params, A: torch.Tensor, S: torch.Tensor) -> torch.Tensor:
+    """Eq. 3-7 into the caller's S [B, N] float32 tensor, using the library's built-in scratch
+    array instead of a workspace: this call creates no tensor and allocates nothing."""
+    assert S.dtype == torch.float32 and tuple(S.shape) == (p.batch, p.n_tokens)
+    cp = p.c()
+    _check("tc_attn_score_noalloc",
+           lib().tc_attn_score_noalloc(C.byref(cp), _ptr(A), _ptr(S), _stream()))
+    return S
 
 
 def tc_score(p: Params, O, A, ws=None) -> Dict[str, torch.Tensor]:

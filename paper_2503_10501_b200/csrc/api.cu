@@ -395,6 +395,7 @@ const char* tc_status_string(int32_t status) {
     case TC_ERR_CUDA: return "CUDA runtime error";
     case TC_ERR_RANK_CAP: return "numerical rank reached rank_cap";
     case TC_ERR_BREAKDOWN: return "Cholesky breakdown";
+    case TC_ERR_SCRATCH_LIMIT: return "request exceeds the built-in scratch of tc_attn_score_noalloc";
     default: return "unknown status";
   }
 }
