@@ -50,6 +50,7 @@ Scope::~Scope() {
 }
 
 tc_status launch_gram_simt(const Dims& D, const void* O, float* G, cudaStream_t st);
+tc_status launch_gram_tc(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 void fill_i32(int32_t* p, int n, int v, cudaStream_t st);
 
 tc_status make_dims(const tc_params* p, Dims* out) {
@@ -144,7 +145,9 @@ Plan make_plan(const Dims& D) {
   return P;
 }
 
-tc_status launch_gram(const Dims& D, const void* O, float* G, cudaStream_t st) {
+// float16 inputs go to the tensor cores; float32 inputs keep full precision on the plain ALUs
+tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st) {
+  if (D.f16) return launch_gram_tc(D, O, G, status, st);
   return launch_gram_simt(D, O, G, st);
 }
 
@@ -178,7 +181,7 @@ static void enqueue_score(const Ctx& c, const void* O, const void* A, float* E, 
   const Dims& D = c.D;
   fill_i32(img_status, D.B, 0, c.st);
   launch_attn_colsum(D, A, (float*)(c.ws + c.P.s_part), c.st);
-  launch_gram(D, O, (float*)(c.ws + c.P.G), c.st);
+  launch_gram(D, O, (float*)(c.ws + c.P.G), img_status, c.st);
   launch_ics(D, c.P, c.ws, O, C, sigma, rank, img_status, c.st);
   launch_combine(D, (const float*)(c.ws + c.P.s_part), C, S, E, c.st);
 }
@@ -380,7 +383,7 @@ tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream) {
   tc_status s = make_dims(p, &D);
   if (s != TC_OK) return s;
   if (!O || !G || misaligned(O) || misaligned(G)) return TC_ERR_INVALID_ARG;
-  s = launch_gram(D, O, G, (cudaStream_t)stream);
+  s = launch_gram(D, O, G, nullptr, (cudaStream_t)stream);
   if (s != TC_OK) return s;
   return check_launch();
 }

@@ -1,0 +1,335 @@
+// G = O O^T for float16 O on the 5th-generation tensor cores (tcgen05), float32 accumulate.
+//
+// The SVD of Sec. 3.3.1 is taken through the Gram matrix (O O^T = U Sigma^2 U^T) and the cosine
+// similarities of Eq. 3-10 are its normalised entries, so this is the one dense contraction of
+// the path.  One CTA produces one 128 x 128 tile of G for one image:
+//   - warp 4 (one lane) streams 128 x 64 slices of the two row blocks of O into a ring of
+//     shared-memory stages with TMA (128-byte swizzle, out-of-range rows/columns read as zero);
+//   - warp 5 (one lane) issues tcgen05.mma (M = N = 128, K = 16, both operands K-major) into one
+//     of two 128-column TMEM accumulators and frees each stage with tcgen05.commit;
+//   - warps 0-3 read a finished accumulator back with tcgen05.ld, add it to a float32 register
+//     tile, and at the end store the tile and, for a tile below the diagonal, its mirror image,
+//     so G is symmetric bit for bit.
+// The tensor core adds into its accumulator with truncation, and over the 256 MMA steps of
+// d = 4096 that bias reaches 2e-5 relative: enough to move the small singular values the rank
+// cut-off sits next to by several 1e-3.  So the K loop is cut into chunks of DRAIN_KB * 64
+// elements; each chunk starts a fresh accumulator and the chunk sums are added in registers with
+// round-to-nearest, while the tensor core already works on the other accumulator.
+// Only tiles on or below the diagonal are computed.  Every mbarrier wait is bounded: a wait
+// that runs out records an error for the image and the CTA winds down (TMEM is still freed).
+#include <cuda.h>
+
+#include "tc_internal.cuh"
+
+namespace tc {
+
+namespace {
+
+constexpr int TILE = 128;         // rows of O per operand tile = tile edge of G
+constexpr int BK = 64;            // K elements per stage: 64 halves = one 128-byte swizzle row
+constexpr int STAGES = 3;
+constexpr int UMMA_K = 16;
+constexpr uint32_t TILE_BYTES = TILE * BK * 2;  // 16 KB
+constexpr uint32_t SMEM_BYTES = STAGES * 2 * TILE_BYTES + 1024;  // + alignment slack
+constexpr uint32_t TMEM_COLS = 256;  // two 128-column accumulators
+constexpr int DRAIN_KB = 2;          // stages per accumulation chunk (128 elements of K)
+constexpr uint32_t WAIT_LIMIT = 1u << 20;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+
+// Bounded wait: false when the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                            int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile, rows of 128 bytes, 128-byte swizzle; groups of
+// eight rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address
+  d |= (uint64_t)(1024u >> 4) << 32;             // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: D float32, A and B float16, both K-major, M = 128, N = 128.
+constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accum)
+      : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CUtensorMap map,
+                                                     float* __restrict__ G, int N, int d,
+                                                     int tiles_per_image,
+                                                     int32_t* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[STAGES];
+  __shared__ __align__(8) uint64_t bar_empty[STAGES];
+  __shared__ __align__(8) uint64_t bar_acc_full[2];
+  __shared__ __align__(8) uint64_t bar_acc_empty[2];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x / tiles_per_image;
+  int t = blockIdx.x % tiles_per_image;
+  // t -> (ti, tj) with ti >= tj: t = ti (ti + 1) / 2 + tj
+  int ti = 0;
+  while ((ti + 1) * (ti + 2) / 2 <= t) ++ti;
+  const int tj = t - ti * (ti + 1) / 2;
+  const bool diag = (ti == tj);
+  const int kblocks = (d + BK - 1) / BK;
+  const int nchunks = (kblocks + DRAIN_KB - 1) / DRAIN_KB;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  auto stage_a = [&](int s) { return smem_base + (uint32_t)s * 2u * TILE_BYTES; };
+  auto stage_b = [&](int s) { return smem_base + (uint32_t)s * 2u * TILE_BYTES + TILE_BYTES; };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bar_acc_full[i]), 1);
+      mbar_init(smem_u32(&bar_acc_empty[i]), 4);  // one arrival per epilogue warp
+    }
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&s_tmem)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = s_tmem;
+
+  if (warp == 4) {
+    // ---- TMA producer ----
+    if (lane == 0) {
+      for (int kb = 0; kb < kblocks; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t round = (uint32_t)(kb / STAGES);
+        if (!mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u)) {
+          s_fail = 1;
+          break;
+        }
+        const uint32_t full = smem_u32(&bar_full[s]);
+        mbar_expect_tx(full, diag ? TILE_BYTES : 2u * TILE_BYTES);
+        tma_load_3d(stage_a(s), &map, kb * BK, ti * TILE, b, full);
+        if (!diag) tma_load_3d(stage_b(s), &map, kb * BK, tj * TILE, b, full);
+      }
+    }
+  } else if (warp == 5) {
+    // ---- MMA issuer ----
+    if (lane == 0) {
+      bool ok = true;
+      for (int c = 0; c < nchunks && ok; ++c) {
+        const int buf = c & 1;
+        if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), (((uint32_t)c >> 1) & 1u) ^ 1u)) {
+          s_fail = 1;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t tmem_d = tmem_base + (uint32_t)buf * 128u;
+        const int kb_end = min(kblocks, (c + 1) * DRAIN_KB);
+        for (int kb = c * DRAIN_KB; kb < kb_end; ++kb) {
+          const int s = kb % STAGES;
+          const uint32_t round = (uint32_t)(kb / STAGES);
+          if (!mbar_wait(smem_u32(&bar_full[s]), round & 1u)) {
+            s_fail = 1;
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint64_t da = umma_desc(stage_a(s));
+          const uint64_t db = diag ? da : umma_desc(stage_b(s));
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // 16 halves = 32 bytes further along K inside the swizzled row: +2 in 16-byte units
+            umma_f16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
+                     (kb > c * DRAIN_KB || k > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&bar_empty[s]));
+        }
+        umma_commit(smem_u32(&bar_acc_full[buf]));
+      }
+    }
+  } else {
+    // ---- epilogue: warps 0..3 own TMEM lanes 32 w .. 32 w + 31 (= rows of the tile) ----
+    float acc[TILE];
+#pragma unroll
+    for (int j = 0; j < TILE; ++j) acc[j] = 0.f;
+    bool ok = true;
+    for (int c = 0; c < nchunks; ++c) {
+      const int buf = c & 1;
+      if (!mbar_wait(smem_u32(&bar_acc_full[buf]), ((uint32_t)c >> 1) & 1u)) {
+        ok = false;
+        break;
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * 128u;
+#pragma unroll
+      for (int q = 0; q < TILE / 32; ++q) {
+        float v[32];
+        tmem_ld32(taddr + (uint32_t)(q * 32), v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[q * 32 + j] += v[j];
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_acc_empty[buf]))
+                     : "memory");
+    }
+    if (ok && s_fail == 0) {
+      float* Gb = G + (size_t)b * N * N;
+      const int row = ti * TILE + warp * 32 + lane;
+      if (row < N) {
+#pragma unroll
+        for (int q = 0; q < TILE / 32; ++q) {
+          const int col0 = tj * TILE + q * 32;
+          if (col0 + 32 <= N && (N & 3) == 0) {
+            float4* dst = reinterpret_cast<float4*>(Gb + (size_t)row * N + col0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              dst[j] = make_float4(acc[q * 32 + 4 * j], acc[q * 32 + 4 * j + 1],
+                                   acc[q * 32 + 4 * j + 2], acc[q * 32 + 4 * j + 3]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < N) Gb[(size_t)row * N + col0 + j] = acc[q * 32 + j];
+          }
+          if (!diag) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < N) Gb[(size_t)(col0 + j) * N + row] = acc[q * 32 + j];
+          }
+        }
+      }
+    } else if (status != nullptr && threadIdx.x == 0) {
+      atomicMax(&status[b], (int)TC_ERR_CUDA);
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 5) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(TMEM_COLS)
+                 : "memory");
+  }
+}
+
+typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                              CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                              CUtensorMapFloatOOBfill);
+
+encode_fn get_encode() {
+  static encode_fn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (encode_fn)p;
+  }
+  return fn;
+}
+
+}  // namespace
+
+// Returns TC_ERR_UNSUPPORTED when the tensor map cannot be built (caller may not fall back
+// silently: it reports the error).
+tc_status launch_gram_tc(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st) {
+  encode_fn enc = get_encode();
+  if (enc == nullptr) return TC_ERR_CUDA;
+  CUtensorMap map;
+  const cuuint64_t dims[3] = {(cuuint64_t)D.d, (cuuint64_t)D.N, (cuuint64_t)D.B};
+  const cuuint64_t strides[2] = {(cuuint64_t)D.d * 2, (cuuint64_t)D.N * D.d * 2};
+  const cuuint32_t box[3] = {BK, TILE, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(O), dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return TC_ERR_CUDA;
+  if (cudaFuncSetAttribute((const void*)gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)SMEM_BYTES) != cudaSuccess)
+    return TC_ERR_CUDA;
+  const int nt = (D.N + TILE - 1) / TILE;
+  const int tiles = nt * (nt + 1) / 2;
+  Scope scope_(KC_GRAM, st);
+  gram_tc_kernel<<<D.B * tiles, 192, SMEM_BYTES, st>>>(map, G, D.N, D.d, tiles, status);
+  note_launch();
+  return TC_OK;
+}
+
+}  // namespace tc

@@ -84,7 +84,7 @@ void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
                     void* Ko, void* Vo, cudaStream_t st);
 
 // G = O O^T (float32 out).
-tc_status launch_gram(const Dims& D, const void* O, float* G, cudaStream_t st);
+tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 
 // Eigen-decomposition of G and Eq. 3-6:  C, theta (unsorted), then sorted sigma / rank.
 void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_out,

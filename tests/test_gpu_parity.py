@@ -183,3 +183,24 @@ def test_rank_cap_too_small_is_reported():
     sc = tcb.tc_score(p, dev(batch["O"]), dev(batch["A"]))
     torch.cuda.synchronize()
     assert host(sc["img_status"])[0] == 6
+
+
+# ------------------------------------------------------------------ the Gram matrix alone
+@pytest.mark.parametrize("B,N,d", [(2, 576, 4096), (3, 200, 264), (2, 64, 128), (1, 130, 72)])
+def test_gram_f16_against_float64(B, N, d):
+    rng = np.random.default_rng(N + d)
+    O = (rng.standard_normal((B, N, 24)) @ rng.standard_normal((24, d)) * 3.0
+         + 0.01 * rng.standard_normal((B, N, d))).astype(np.float16)
+    O[:, 7] = O[:, 3]                       # identical rows must give identical entries
+    p = tcb.Params(batch=B, n_tokens=N, d_model=d, n_heads=1, head_dim=8, n_query=1, keep=1,
+                   dtype="f16")
+    G = host(tcb.tc_gram(p, dev(O)))
+    torch.cuda.synchronize()
+    O64 = O.astype(np.float64)
+    G64 = O64 @ O64.transpose(0, 2, 1)
+    scale = np.sqrt(np.einsum("bii->bi", G64))
+    err = np.abs(G - G64) / (scale[:, :, None] * scale[:, None, :])
+    # float32 accumulation of d products of float16 values: a few 1e-7 relative to |O_i||O_j|
+    assert err.max() <= 2e-6, err.max()
+    assert np.array_equal(G, G.transpose(0, 2, 1)), "G must be symmetric bit for bit"
+    assert np.array_equal(G[:, 7], G[:, 3]) and np.array_equal(G[:, :, 7], G[:, :, 3])
