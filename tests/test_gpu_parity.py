@@ -204,3 +204,22 @@ def test_gram_f16_against_float64(B, N, d):
     assert err.max() <= 2e-6, err.max()
     assert np.array_equal(G, G.transpose(0, 2, 1)), "G must be symmetric bit for bit"
     assert np.array_equal(G[:, 7], G[:, 3]) and np.array_equal(G[:, :, 7], G[:, :, 3])
+
+
+# ------------------------------------------------------------------ large shapes
+def test_cfg5_bench_point_sampled_images():
+    # the launch configuration bench.py times: 64 images, T = 128, keep = 128
+    cfg = inputs.CONFIGS["cfg5_sweep_f16"]
+    flips = check_config(cfg, [0, 31, 63])
+    assert flips["flips_sets"] <= 2 and flips["flips_merge"] <= 2, flips
+
+
+@pytest.mark.parametrize("T,keep", [(32, 64), (512, 288)])
+def test_cfg5_sweep_corners(T, keep):
+    cfg = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=8, n_query=T, keep=keep)
+    check_config(cfg, [0, 7])
+
+
+def test_cfg4_anyres():
+    cfg = inputs.CONFIGS["cfg4_anyres_f16"]
+    check_config(cfg, [2])
