@@ -229,6 +229,220 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const float* __restrict__
 }
 
 // ==========================================================================================
+// The same factorisation and inverse for k small enough that one k x k float32 array fits in
+// shared memory: blocked (16 columns at a time) so that the block-wide barriers number a few
+// dozen instead of three per column, and the inverse is formed in place of the factor.
+//   phase 1  R^T R = S + shift I   (right-looking: diagonal block in one warp's registers,
+//            block row by forward substitution, trailing update in 4 x 4 register tiles)
+//   phase 2  R <- R^{-1}           (left to right over block columns; a finished leading
+//            block of the inverse multiplies the next block column)
+// ==========================================================================================
+constexpr int CNB = 16;
+
+__global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __restrict__ S,
+                                                              float* __restrict__ RinvT, int k,
+                                                              float shift_rel,
+                                                              int32_t* __restrict__ status) {
+  extern __shared__ float A[];  // [k][ld], ld odd: rows and columns both walk all banks
+  __shared__ float s_red[16];
+  __shared__ int s_bad;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ld = k | 1;
+  const size_t kk = (size_t)k * k;
+  const float* Sb = S + b * kk;
+
+  float md = 0.f;
+  for (int i = tid; i < k; i += 512) md = fmaxf(md, Sb[(size_t)i * k + i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, o));
+  if (lane == 0) s_red[warp] = md;
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  md = s_red[0];
+  for (int w = 1; w < 16; ++w) md = fmaxf(md, s_red[w]);
+  const float shift = shift_rel * md;
+  const float tiny = fmaxf(md, 1e-30f) * 1e-12f;
+  for (int e = tid; e < (int)kk; e += 512) {
+    const int r = e / k, c = e - r * k;
+    A[r * ld + c] = Sb[e] + (r == c ? shift : 0.f);
+  }
+  __syncthreads();
+
+  const int nblk = (k + CNB - 1) / CNB;
+  // ---------------- phase 1: Cholesky ----------------
+  for (int jb = 0; jb < nblk; ++jb) {
+    const int j0 = jb * CNB, j1 = min(k, j0 + CNB);
+    if (warp == 0) {
+      // lane c (< 16) keeps column c of the diagonal block; rows/columns past k act as identity
+      float col[CNB];
+      const int gc = j0 + lane;
+#pragma unroll
+      for (int r = 0; r < CNB; ++r) {
+        const int gr = j0 + r;
+        float v = (r == lane) ? 1.f : 0.f;
+        if (lane < CNB && gc < k && gr < k && r <= lane) v = A[gr * ld + gc];
+        col[r] = v;
+      }
+#pragma unroll
+      for (int i = 0; i < CNB; ++i) {
+        float piv = __shfl_sync(0xffffffffu, col[i], i);
+        if (!(piv > 0.f)) {
+          piv = tiny;
+          if (lane == 0) s_bad = 1;
+        }
+        const float dd = sqrtf(piv);
+        if (lane == i) col[i] = dd;
+        else if (lane > i) col[i] = col[i] / dd;
+#pragma unroll
+        for (int r = i + 1; r < CNB; ++r) {
+          const float v = __shfl_sync(0xffffffffu, col[i], r);
+          if (lane >= r) col[r] = fmaf(-v, col[i], col[r]);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < CNB; ++r) {
+        const int gr = j0 + r;
+        if (lane < CNB && gc < k && gr < k && r <= lane) A[gr * ld + gc] = col[r];
+      }
+    }
+    __syncthreads();
+    // block row: R[j0.., c] for c >= j1, one thread per column
+    for (int c = j1 + tid; c < k; c += 512) {
+      float x[CNB];
+#pragma unroll
+      for (int i = 0; i < CNB; ++i) {
+        if (j0 + i < k) {
+          float sacc = A[(j0 + i) * ld + c];
+#pragma unroll
+          for (int m = 0; m < i; ++m) sacc = fmaf(-A[(j0 + m) * ld + j0 + i], x[m], sacc);
+          x[i] = sacc / A[(j0 + i) * ld + j0 + i];
+        } else {
+          x[i] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < CNB; ++i)
+        if (j0 + i < k) A[(j0 + i) * ld + c] = x[i];
+    }
+    __syncthreads();
+    // trailing update of the upper triangle in 4 x 4 tiles
+    const int m = k - j1;
+    if (m > 0) {
+      const int mt = (m + 3) >> 2;
+      for (int t = tid; t < mt * mt; t += 512) {
+        const int tr = t / mt, tc = t - tr * mt;
+        if (tc < tr) continue;
+        const int r0 = j1 + 4 * tr, c0 = j1 + 4 * tc;
+        float acc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+        for (int i = j0; i < j1; ++i) {
+          float a[4], bb[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            a[u] = (r0 + u < k) ? A[i * ld + r0 + u] : 0.f;
+            bb[u] = (c0 + u < k) ? A[i * ld + c0 + u] : 0.f;
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(a[u], bb[v], acc[u][v]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            if (r0 + u < k && c0 + v < k && c0 + v >= r0 + u) A[(r0 + u) * ld + c0 + v] -= acc[u][v];
+      }
+    }
+    __syncthreads();
+  }
+  if (tid == 0 && s_bad) atomicMax(&status[b], (int)TC_ERR_BREAKDOWN);
+
+  // ---------------- phase 2: in-place inverse of the upper-triangular factor ----------------
+  for (int jb = 0; jb < nblk; ++jb) {
+    const int j0 = jb * CNB, j1 = min(k, j0 + CNB), w = j1 - j0;
+    if (warp == 0) {
+      // lane c solves R_JJ x = e_c by back substitution (x has entries 0..c)
+      float x[CNB];
+#pragma unroll
+      for (int i = 0; i < CNB; ++i) x[i] = 0.f;
+      if (lane < w) {
+#pragma unroll
+        for (int i = CNB - 1; i >= 0; --i) {
+          if (i <= lane) {
+            float sacc = (i == lane) ? 1.f : 0.f;
+#pragma unroll
+            for (int mm = i + 1; mm < CNB; ++mm)
+              if (mm <= lane) sacc = fmaf(-A[(j0 + i) * ld + j0 + mm], x[mm], sacc);
+            x[i] = sacc / A[(j0 + i) * ld + j0 + i];
+          }
+        }
+      }
+      __syncwarp();
+      if (lane < w) {
+#pragma unroll
+        for (int i = 0; i < CNB; ++i)
+          if (i <= lane) A[(j0 + i) * ld + j0 + lane] = x[i];
+      }
+    }
+    __syncthreads();
+    if (j0 > 0) {
+      // T = R[0:j0, J] * X_JJ, one thread per row, written back over R[0:j0, J]
+      for (int r = tid; r < j0; r += 512) {
+        float rr[CNB], tt[CNB];
+#pragma unroll
+        for (int mm = 0; mm < CNB; ++mm) rr[mm] = (mm < w) ? A[r * ld + j0 + mm] : 0.f;
+#pragma unroll
+        for (int c = 0; c < CNB; ++c) {
+          float sacc = 0.f;
+#pragma unroll
+          for (int mm = 0; mm <= c; ++mm)
+            if (c < w) sacc = fmaf(rr[mm], A[(j0 + mm) * ld + j0 + c], sacc);
+          tt[c] = sacc;
+        }
+#pragma unroll
+        for (int c = 0; c < CNB; ++c)
+          if (c < w) A[r * ld + j0 + c] = tt[c];
+      }
+      __syncthreads();
+      // X[0:j0, J] = - X[0:j0, 0:j0] * T : all outputs into registers first, then written
+      float outv[8];
+      const int total = j0 * w;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int e = tid + q * 512;
+        float sacc = 0.f;
+        if (e < total) {
+          const int r = e / w, c = e - r * w;
+          for (int mm = r; mm < j0; ++mm) sacc = fmaf(A[r * ld + mm], A[mm * ld + j0 + c], sacc);
+        }
+        outv[q] = -sacc;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int e = tid + q * 512;
+        if (e < total) {
+          const int r = e / w, c = e - r * w;
+          A[r * ld + j0 + c] = outv[q];
+        }
+      }
+      __syncthreads();
+    }
+  }
+  // RinvT[c][m] = X[m][c] for m <= c, zero otherwise
+  float* out = RinvT + b * kk;
+  for (int e = tid; e < (int)kk; e += 512) {
+    const int c = e / k, mrow = e - c * k;
+    out[e] = (mrow <= c) ? A[mrow * ld + c] : 0.f;
+  }
+}
+
+// ==========================================================================================
 // One-sided Jacobi eigen-solver for a symmetric positive semi-definite n x n matrix.
 // One block (16 warps) per image.  W (column-major) starts as the matrix, J as the identity;
 // each pair step rotates columns p, q of both so that the W columns become orthogonal.  At
@@ -383,6 +597,351 @@ __global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ H
   }
 }
 
+// ==========================================================================================
+// Symmetric eigen-solver for matrices that fit in shared memory (n <= ~230):
+//   1. Householder reduction to a tridiagonal matrix T, the orthogonal factor Q formed in place;
+//   2. every eigenvalue of T by bisection on the Sturm count, one thread per eigenvalue;
+//   3. the eigenvector of T for every eigenvalue that can pass the rank cut-off, by inverse
+//      iteration (tridiagonal elimination with partial pivoting), one thread per eigenvalue,
+//      its four work vectors in global scratch laid out thread-fastest;
+//   4. eigenvalues refined as Rayleigh quotients on T, eigenvectors of H as Z = Q Y.
+// Nothing here is a serial recurrence over the whole matrix, which is what makes it several
+// times faster than sweeping Jacobi rotations or chasing QL bulges from one thread.
+// Eigenvectors of eigenvalues closer together than the rounding level of T are not
+// re-orthogonalised against each other (Eq. 3-6 is not unique there in the first place).
+//   in   H [n][n] symmetric (only its symmetric part is used)
+//   out  theta [n] eigenvalues (ascending), ZT [n][n] with ZT[p][i] = component i of
+//        eigenvector p (all zero for eigenvalues under a quarter of the rank cut-off)
+//   scratch u0, u1, u2, yv: [n][n] float each, per image
+// One block (16 warps) per image.
+// ==========================================================================================
+__global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
+                                                         float* __restrict__ ZTg,
+                                                         float* __restrict__ theta, int n, float rank_tol,
+                                                         float* __restrict__ u0g, float* __restrict__ u1g,
+                                                         float* __restrict__ u2g, float* yg,
+                                                         int32_t* __restrict__ status) {
+  extern __shared__ float sm[];
+  const int ld = n | 1;
+  float* A = sm;                       // [n][ld]
+  float* dv = A + (size_t)n * ld;      // [n] diagonal
+  float* ev = dv + n;                  // [n] sub-diagonal (ev[i] couples i and i+1)
+  float* vv = ev + n;                  // [n] Householder vector of the current step
+  float* pv = vv + n;                  // [n] work vector
+  float* beta = pv + n;                // [n] reflector scales
+  float2* cs = reinterpret_cast<float2*>(beta + n);  // [2][n] rotation batches
+  __shared__ float s_red[16];
+  __shared__ int s_fail;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* Hb = Hin + (size_t)b * n * n;
+
+  for (int e = tid; e < n * n; e += 512) {
+    const int r = e / n, c = e - r * n;
+    A[r * ld + c] = 0.5f * (Hb[e] + Hb[(size_t)c * n + r]);
+  }
+  if (tid == 0) s_fail = 0;
+  __syncthreads();
+
+  // ---------------- Householder tridiagonalisation ----------------
+  for (int j = 0; j + 2 < n; ++j) {
+    const int m = n - j - 1;  // length of the column below the diagonal
+    // sigma = |x|^2, x = A[j+1.., j]
+    float part = 0.f;
+    for (int r = tid; r < m; r += 512) {
+      const float x = A[(j + 1 + r) * ld + j];
+      part = fmaf(x, x, part);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if (lane == 0) s_red[warp] = part;
+    __syncthreads();
+    float sigma = 0.f;
+#pragma unroll
+    for (int w = 0; w < 16; ++w) sigma += s_red[w];
+    const float x0 = A[(j + 1) * ld + j];
+    const float tail = sigma - x0 * x0;  // |x|^2 without its first entry
+    if (tid == 0) dv[j] = A[j * ld + j];
+    if (!(tail > 1e-30f * sigma) || !(sigma > 0.f)) {
+      // column already in tridiagonal form
+      if (tid == 0) {
+        ev[j] = x0;
+        beta[j] = 0.f;
+      }
+      __syncthreads();
+      continue;
+    }
+    const float alpha = -copysignf(sqrtf(sigma), x0);
+    const float v0 = x0 - alpha;
+    const float bj = 2.0f / (tail + v0 * v0);
+    for (int r = tid; r < m; r += 512) {
+      const float x = (r == 0) ? v0 : A[(j + 1 + r) * ld + j];
+      vv[r] = x;
+      A[(j + 1 + r) * ld + j] = x;  // kept for the accumulation of Q
+    }
+    if (tid == 0) {
+      ev[j] = alpha;
+      beta[j] = bj;
+    }
+    __syncthreads();
+    // p = beta * B v, one warp per row of the trailing block B = A[j+1.., j+1..]
+    for (int r = warp; r < m; r += 16) {
+      const float* row = A + (j + 1 + r) * ld + j + 1;
+      float acc = 0.f;
+      for (int c = lane; c < m; c += 32) acc = fmaf(row[c], vv[c], acc);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == 0) pv[r] = bj * acc;
+    }
+    __syncthreads();
+    // K = beta/2 * v.p ;  w = p - K v  (every thread forms K itself from the same partial sums)
+    part = 0.f;
+    for (int r = tid; r < m; r += 512) part = fmaf(vv[r], pv[r], part);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if (lane == 0) s_red[warp] = part;
+    __syncthreads();
+    float vp = 0.f;
+#pragma unroll
+    for (int w = 0; w < 16; ++w) vp += s_red[w];
+    const float K = 0.5f * bj * vp;
+    __syncthreads();  // s_red is reused next step; pv is rewritten below
+    for (int r = tid; r < m; r += 512) pv[r] = fmaf(-K, vv[r], pv[r]);
+    __syncthreads();
+    // B -= v w^T + w v^T
+    for (int r = warp; r < m; r += 16) {
+      float* row = A + (j + 1 + r) * ld + j + 1;
+      const float vr = vv[r], wr = pv[r];
+      for (int c = lane; c < m; c += 32) row[c] -= fmaf(vr, pv[c], wr * vv[c]);
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    if (n >= 2) {
+      dv[n - 2] = A[(n - 2) * ld + n - 2];
+      ev[n - 2] = A[(n - 1) * ld + n - 2];
+      beta[n - 2] = 0.f;
+    }
+    dv[n - 1] = A[(n - 1) * ld + n - 1];
+    ev[n - 1] = 0.f;
+    A[(n - 1) * ld + n - 1] = 1.f;  // the accumulation of Q starts from the identity
+  }
+  __syncthreads();
+
+  // ---------------- Q = H_0 H_1 ... H_{n-3}, accumulated backwards, in place ----------------
+  // Reflector j sits in A[j+1.., j]; column c >= j+2 of A, rows >= j+2, already holds the
+  // product of the later reflectors; row j+1 of those columns counts as zero.
+  {
+    const int cw = (n + 31) / 32;            // warps needed to cover the columns
+    const int groups = max(1, 16 / cw);      // row ranges worked on side by side
+    const int g = warp / cw;                 // this thread's row range
+    const int cl = (warp % cw) * 32 + lane;  // this thread's column, relative to j+2
+    float* tbuf = reinterpret_cast<float*>(cs);  // [<=4][n] partial dots (cs is free here)
+    const int gmax = min(groups, 4);
+    for (int j = n - 3; j >= 0; --j) {
+      const float bj = beta[j];
+      const int m = n - j - 1;       // rows j+1 .. n-1
+      const int ncol = m - 1;        // columns j+2 .. n-1
+      const int rows = m - 1;        // rows j+2 .. n-1 take part in the dots
+      const int per = (rows + gmax - 1) / gmax;
+      const int r_lo = j + 2 + g * per, r_hi = min(n, r_lo + per);
+      const bool active = (g < gmax) && (cl < ncol);
+      const int c = j + 2 + cl;
+      float tsum = 0.f;
+      if (active && bj != 0.f)
+        for (int r = r_lo; r < r_hi; ++r) tsum = fmaf(A[r * ld + j], A[r * ld + c], tsum);
+      if (g < gmax && cl < n) tbuf[g * n + cl] = tsum;
+      __syncthreads();
+      if (active) {
+        float t = 0.f;
+        for (int q = 0; q < gmax; ++q) t += tbuf[q * n + cl];
+        const float bt = bj * t;
+        for (int r = r_lo; r < r_hi; ++r) A[r * ld + c] = fmaf(-bt, A[r * ld + j], A[r * ld + c]);
+        if (g == 0) A[(j + 1) * ld + c] = -bt * A[(j + 1) * ld + j];
+      }
+      __syncthreads();
+      // column j+1: H_j e_{j+1}
+      const float vj1 = A[(j + 1) * ld + j];
+      for (int r = j + 2 + tid; r < n; r += 512) A[r * ld + j + 1] = -bj * A[r * ld + j] * vj1;
+      if (tid == 0) A[(j + 1) * ld + j + 1] = 1.0f - bj * vj1 * vj1;
+      __syncthreads();
+    }
+    // first row and column of Q are e_0
+    for (int i = tid; i < n; i += 512) {
+      A[i * ld] = (i == 0) ? 1.f : 0.f;
+      A[i] = (i == 0) ? 1.f : 0.f;
+    }
+    if (n == 2 && tid == 0) {  // no reflector at all: Q = I
+      A[ld + 1] = 1.f;
+    }
+    __syncthreads();
+  }
+
+  // ---------------- eigenvalues of T by bisection ----------------
+  // dv = diagonal, ev[i] couples i and i+1.  vv <- ev^2, pv <- eigenvalues (ascending).
+  float* e2 = vv;
+  float* lam = pv;
+  float tnorm = 0.f;
+  {
+    float lo = 3.0e38f, hi = -3.0e38f;
+    for (int i = tid; i < n; i += 512) {
+      const float el = (i > 0) ? fabsf(ev[i - 1]) : 0.f, er = (i + 1 < n) ? fabsf(ev[i]) : 0.f;
+      lo = fminf(lo, dv[i] - el - er);
+      hi = fmaxf(hi, dv[i] + el + er);
+      e2[i] = ev[i] * ev[i];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (lane == 0) {
+      s_red[warp] = lo;
+      reinterpret_cast<float*>(cs)[warp] = hi;
+    }
+    __syncthreads();
+    lo = s_red[0];
+    hi = reinterpret_cast<float*>(cs)[0];
+    for (int w = 1; w < 16; ++w) {
+      lo = fminf(lo, s_red[w]);
+      hi = fmaxf(hi, reinterpret_cast<float*>(cs)[w]);
+    }
+    const float tn = fmaxf(fabsf(lo), fabsf(hi));
+    const float pivmin = fmaxf(tn, 1e-30f) * 1e-12f;
+    lo -= 2.4e-7f * tn + pivmin;
+    hi += 2.4e-7f * tn + pivmin;
+    if (tid < n) {
+      // eigenvalue number tid (0 = smallest): count(x) = number of eigenvalues below x
+      float a = lo, bhi = hi;
+      for (int it = 0; it < 48; ++it) {
+        const float x = 0.5f * (a + bhi);
+        if (!(x > a) || !(x < bhi)) break;
+        float q = dv[0] - x;
+        int cnt = q < 0.f;
+        for (int i = 1; i < n; ++i) {
+          if (fabsf(q) < pivmin) q = -pivmin;
+          q = dv[i] - x - __fdividef(e2[i - 1], q);
+          cnt += q < 0.f;
+        }
+        if (cnt > tid) bhi = x; else a = x;
+      }
+      lam[tid] = 0.5f * (a + bhi);
+    }
+    tnorm = tn;
+  }
+  __syncthreads();
+
+  // ---------------- eigenvectors of T by inverse iteration ----------------
+  const float keep_floor = 0.25f * rank_tol * rank_tol * tnorm;
+  {
+    const size_t img = (size_t)b * n * n;
+    float* u0 = u0g + img;
+    float* u1 = u1g + img;
+    float* u2 = u2g + img;
+    float* y = yg + img;
+    if (tid < n) {
+      const int t = tid;
+      float x = lam[t];
+      const bool wanted = x >= keep_floor;
+      // an eigenvalue bisection could not tell from its lower neighbour is nudged up so the two
+      // solves do not return the same vector
+      const float sep = 1.2e-6f * fmaxf(fabsf(x), 1e-3f * tnorm);
+      if (t > 0 && x - lam[t - 1] < sep) x = lam[t - 1] + sep * (float)(1 + (t & 3));
+      const float tiny = fmaxf(tnorm, 1e-30f) * 1.1920929e-7f;
+      if (wanted) {
+        for (int it = 0; it < 3; ++it) {
+          // forward: eliminate the sub-diagonal with row interchanges, the right-hand side with it
+          float a = dv[0] - x, bb = (n > 1) ? ev[0] : 0.f, c = 0.f;
+          float r = (it == 0) ? 1.f : y[t];
+          for (int i = 0; i + 1 < n; ++i) {
+            const float sub = ev[i], dn = dv[i + 1] - x, en = (i + 2 < n) ? ev[i + 1] : 0.f;
+            float rn = (it == 0) ? 1.f : y[(size_t)(i + 1) * n + t];
+            if (fabsf(a) >= fabsf(sub)) {
+              if (fabsf(a) < tiny) a = copysignf(tiny, a);
+              const float mlt = sub / a;
+              u0[(size_t)i * n + t] = a;
+              u1[(size_t)i * n + t] = bb;
+              u2[(size_t)i * n + t] = c;
+              y[(size_t)i * n + t] = r;
+              a = fmaf(-mlt, bb, dn);
+              bb = fmaf(-mlt, c, en);
+              c = 0.f;
+              r = (it == 0) ? 1.f : fmaf(-mlt, r, rn);
+            } else {
+              const float mlt = a / sub;
+              u0[(size_t)i * n + t] = sub;
+              u1[(size_t)i * n + t] = dn;
+              u2[(size_t)i * n + t] = en;
+              y[(size_t)i * n + t] = (it == 0) ? 1.f : rn;
+              a = fmaf(-mlt, dn, bb);
+              bb = fmaf(-mlt, en, c);
+              c = 0.f;
+              r = (it == 0) ? 1.f : fmaf(-mlt, rn, r);
+            }
+          }
+          if (fabsf(a) < tiny) a = copysignf(tiny, a);
+          // backward substitution, keeping the largest entry for the scaling
+          float y1 = r / a, y2 = 0.f, big = fabsf(y1);
+          y[(size_t)(n - 1) * n + t] = y1;
+          for (int i = n - 2; i >= 0; --i) {
+            const float rhs = y[(size_t)i * n + t];
+            const float yi = (rhs - u1[(size_t)i * n + t] * y1 - u2[(size_t)i * n + t] * y2) / u0[(size_t)i * n + t];
+            y[(size_t)i * n + t] = yi;
+            big = fmaxf(big, fabsf(yi));
+            y2 = y1;
+            y1 = yi;
+          }
+          // scale to unit maximum (keeps the next solve in range); the last pass normalises
+          const float sc = 1.0f / fmaxf(big, 1e-30f);
+          float nrm = 0.f;
+          for (int i = 0; i < n; ++i) {
+            const float v = y[(size_t)i * n + t] * sc;
+            y[(size_t)i * n + t] = v;
+            nrm = fmaf(v, v, nrm);
+          }
+          if (it == 2) {
+            const float inv = rsqrtf(fmaxf(nrm, 1e-30f));
+            float rq = 0.f, prev = 0.f;
+            for (int i = 0; i < n; ++i) {
+              const float v = y[(size_t)i * n + t] * inv;
+              y[(size_t)i * n + t] = v;
+              rq = fmaf(dv[i] * v, v, rq);
+              if (i > 0) rq = fmaf(2.0f * ev[i - 1] * prev, v, rq);
+              prev = v;
+            }
+            e2[t] = rq;  // Rayleigh quotient on T (e2 is free after the bisection)
+          }
+        }
+      } else {
+        for (int i = 0; i < n; ++i) y[(size_t)i * n + t] = 0.f;
+        e2[t] = lam[t];
+      }
+    }
+    __syncthreads();
+    for (int p = tid; p < n; p += 512) theta[(size_t)b * n + p] = fmaxf(e2[p], 0.f);
+    // ---------------- Z = Q Y:  ZT[p][i] = sum_j Q[i][j] Y[j][p] ----------------
+    // thread = (eigenvector p, group of 8 rows i); Q rows are broadcast reads from shared memory
+    float* out = ZTg + img;
+    const int ngrp = (n + 7) / 8;
+    for (int w = tid; w < n * ngrp; w += 512) {
+      const int grp = w / n, p = w - grp * n;
+      const int i0 = grp * 8;
+      float acc[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc[u] = 0.f;
+      for (int j = 0; j < n; ++j) {
+        const float yv = __ldcg(y + (size_t)j * n + p);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (i0 + u < n) acc[u] = fmaf(A[(i0 + u) * ld + j], yv, acc[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (i0 + u < n) out[(size_t)p * n + i0 + u] = acc[u];
+    }
+  }
+  if (tid == 0 && s_fail) atomicMax(&status[b], (int)TC_ERR_NOT_CONVERGED);
+}
+
 typedef void (*jacobi_fn)(const float*, float*, float*, float*, int, int, float, int, int32_t*, float, float);
 
 static jacobi_fn pick_jacobi(int n) {
@@ -405,8 +964,17 @@ static jacobi_fn pick_jacobi(int n) {
 constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared variables
 
 static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
-                          int max_sweeps, float rank_tol, int32_t* status, cudaStream_t st) {
+                          int max_sweeps, float rank_tol, float* scr1, float* scr2, float* scr3,
+                          int32_t* status, cudaStream_t st) {
   Scope scope_(KC_JACOBI, st);
+  {
+    const size_t tri = ((size_t)n * (n | 1) + 9 * (size_t)n) * sizeof(float);
+    if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
+      cudaFuncSetAttribute((const void*)tridiag_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
+      { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, status); note_launch(); }
+      return;
+    }
+  }
   jacobi_fn fn = pick_jacobi(n);
   const size_t need = 2 * (size_t)n * n * sizeof(float);
   const int use_smem = need <= SMEM_LIMIT;
@@ -426,6 +994,14 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
 static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
                             float shift_rel, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_CHOL, st);
+  const size_t blocked = (size_t)k * (k | 1) * sizeof(float);
+  // (the blocked kernel keeps up to 8 outputs per thread in registers in its last step)
+  if (blocked <= SMEM_LIMIT && (size_t)k * CNB <= 8 * 512) {
+    cudaFuncSetAttribute((const void*)chol_inv_blocked_kernel,
+                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)blocked);
+    { chol_inv_blocked_kernel<<<batch, 512, blocked, st>>>(S, RinvT, k, shift_rel, status); note_launch(); }
+    return;
+  }
   const size_t need = 2 * (size_t)k * k * sizeof(float);
   const int use_smem = need <= SMEM_LIMIT;
   const size_t smem = use_smem ? need : 0;
@@ -525,7 +1101,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_
   const size_t sG = (size_t)N * N, sY = (size_t)N * k, sK = (size_t)k * k;
 
   if (D.full) {
-    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, img_status, st);
+    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, nullptr, nullptr, nullptr, img_status, st);
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<B, 256, 2 * (size_t)N * sizeof(float), st>>>(theta, ZT, C_out, sigma_out, rank_out,
                                                              img_status, N, N, q, D.rank_tol, 1); note_launch(); }
@@ -555,9 +1131,10 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_
     gemm<float, float, false, true>(src, Rinv, dst, N, k, k, k, k, k, sY, sK, sY, B, st);
   };
   const float kShift = 1e-6f;
-  // 2. orthonormal basis Q0 of the sketch
+  // 2. a well-conditioned (not orthonormal) basis Q0 of the sketch: one shifted pass takes the
+  //    condition number from ~1e3 to a few units, which is all the next product needs
   cholqr_pass(Y0, Y1, kShift);
-  cholqr_pass(Y1, Y0, 0.f);  // Q0 in Y0
+  { float* t = Y0; Y0 = Y1; Y1 = t; }  // Q0 in Y0
   // 3. one multiplication by G sharpens the subspace:  Y1 = G Q0, then orthonormalise
   gemm<float, float, false, false>(G, Y0, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);
   cholqr_pass(Y1, Y2, kShift);
@@ -566,7 +1143,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_
   // 4. Rayleigh-Ritz:  H = Q1^T G Q1
   gemm<float, float, false, false>(G, Y2, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);   // T = G Q1
   gemm<float, float, true, false>(Y2, Y1, Hm, k, k, N, k, k, k, sY, sY, sK, B, st);   // H = Q1^T T
-  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, img_status, st);
+  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, Sm, Rinv, Hm, img_status, st);
   // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]
   gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
   Scope scope_(KC_ICS, st);
