@@ -290,9 +290,9 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
           piv = tiny;
           if (lane == 0) s_bad = 1;
         }
-        const float dd = sqrtf(piv);
-        if (lane == i) col[i] = dd;
-        else if (lane > i) col[i] = col[i] / dd;
+        const float rinv = rsqrtf(piv);
+        if (lane == i) col[i] = piv * rinv;
+        else if (lane > i) col[i] = col[i] * rinv;
 #pragma unroll
         for (int r = i + 1; r < CNB; ++r) {
           const float v = __shfl_sync(0xffffffffu, col[i], r);
@@ -852,61 +852,104 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
           // forward: eliminate the sub-diagonal with row interchanges, the right-hand side with it
           float a = dv[0] - x, bb = (n > 1) ? ev[0] : 0.f, c = 0.f;
           float r = (it == 0) ? 1.f : y[t];
-          for (int i = 0; i + 1 < n; ++i) {
-            const float sub = ev[i], dn = dv[i + 1] - x, en = (i + 2 < n) ? ev[i + 1] : 0.f;
-            float rn = (it == 0) ? 1.f : y[(size_t)(i + 1) * n + t];
-            if (fabsf(a) >= fabsf(sub)) {
-              if (fabsf(a) < tiny) a = copysignf(tiny, a);
-              const float mlt = sub / a;
-              u0[(size_t)i * n + t] = a;
-              u1[(size_t)i * n + t] = bb;
-              u2[(size_t)i * n + t] = c;
-              y[(size_t)i * n + t] = r;
-              a = fmaf(-mlt, bb, dn);
-              bb = fmaf(-mlt, c, en);
-              c = 0.f;
-              r = (it == 0) ? 1.f : fmaf(-mlt, r, rn);
-            } else {
-              const float mlt = a / sub;
-              u0[(size_t)i * n + t] = sub;
-              u1[(size_t)i * n + t] = dn;
-              u2[(size_t)i * n + t] = en;
-              y[(size_t)i * n + t] = (it == 0) ? 1.f : rn;
-              a = fmaf(-mlt, dn, bb);
-              bb = fmaf(-mlt, en, c);
-              c = 0.f;
-              r = (it == 0) ? 1.f : fmaf(-mlt, rn, r);
+          for (int i0 = 0; i0 + 1 < n; i0 += 8) {
+            float rnx[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              rnx[u] = (it != 0 && i0 + u + 1 < n) ? y[(size_t)(i0 + u + 1) * n + t] : 1.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int i = i0 + u;
+              if (i + 1 < n) {
+                const float sub = ev[i], dn = dv[i + 1] - x, en = (i + 2 < n) ? ev[i + 1] : 0.f;
+                const float rn = rnx[u];
+                if (fabsf(a) >= fabsf(sub)) {
+                  if (fabsf(a) < tiny) a = copysignf(tiny, a);
+                  const float mlt = sub / a;
+                  u0[(size_t)i * n + t] = a;
+                  u1[(size_t)i * n + t] = bb;
+                  u2[(size_t)i * n + t] = c;
+                  y[(size_t)i * n + t] = r;
+                  a = fmaf(-mlt, bb, dn);
+                  bb = fmaf(-mlt, c, en);
+                  c = 0.f;
+                  r = (it == 0) ? 1.f : fmaf(-mlt, r, rn);
+                } else {
+                  const float mlt = a / sub;
+                  u0[(size_t)i * n + t] = sub;
+                  u1[(size_t)i * n + t] = dn;
+                  u2[(size_t)i * n + t] = en;
+                  y[(size_t)i * n + t] = (it == 0) ? 1.f : rn;
+                  a = fmaf(-mlt, dn, bb);
+                  bb = fmaf(-mlt, en, c);
+                  c = 0.f;
+                  r = (it == 0) ? 1.f : fmaf(-mlt, rn, r);
+                }
+              }
             }
           }
           if (fabsf(a) < tiny) a = copysignf(tiny, a);
-          // backward substitution, keeping the largest entry for the scaling
+          // backward substitution, keeping the largest entry for the scaling.  The four global
+          // vectors are read eight rows at a time so their latency is paid once per group.
           float y1 = r / a, y2 = 0.f, big = fabsf(y1);
           y[(size_t)(n - 1) * n + t] = y1;
-          for (int i = n - 2; i >= 0; --i) {
-            const float rhs = y[(size_t)i * n + t];
-            const float yi = (rhs - u1[(size_t)i * n + t] * y1 - u2[(size_t)i * n + t] * y2) / u0[(size_t)i * n + t];
-            y[(size_t)i * n + t] = yi;
-            big = fmaxf(big, fabsf(yi));
-            y2 = y1;
-            y1 = yi;
+          for (int i1 = n - 2; i1 >= 0; i1 -= 8) {
+            float rh[8], p0[8], p1[8], p2[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int i = i1 - u;
+              if (i >= 0) {
+                rh[u] = y[(size_t)i * n + t];
+                p0[u] = u0[(size_t)i * n + t];
+                p1[u] = u1[(size_t)i * n + t];
+                p2[u] = u2[(size_t)i * n + t];
+              }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int i = i1 - u;
+              if (i >= 0) {
+                const float yi = (rh[u] - p1[u] * y1 - p2[u] * y2) / p0[u];
+                y[(size_t)i * n + t] = yi;
+                big = fmaxf(big, fabsf(yi));
+                y2 = y1;
+                y1 = yi;
+              }
+            }
           }
           // scale to unit maximum (keeps the next solve in range); the last pass normalises
           const float sc = 1.0f / fmaxf(big, 1e-30f);
           float nrm = 0.f;
-          for (int i = 0; i < n; ++i) {
-            const float v = y[(size_t)i * n + t] * sc;
-            y[(size_t)i * n + t] = v;
-            nrm = fmaf(v, v, nrm);
+          for (int i0 = 0; i0 < n; i0 += 8) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              if (i0 + u < n) v[u] = y[(size_t)(i0 + u) * n + t] * sc;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              if (i0 + u < n) {
+                y[(size_t)(i0 + u) * n + t] = v[u];
+                nrm = fmaf(v[u], v[u], nrm);
+              }
           }
           if (it == 2) {
             const float inv = rsqrtf(fmaxf(nrm, 1e-30f));
             float rq = 0.f, prev = 0.f;
-            for (int i = 0; i < n; ++i) {
-              const float v = y[(size_t)i * n + t] * inv;
-              y[(size_t)i * n + t] = v;
-              rq = fmaf(dv[i] * v, v, rq);
-              if (i > 0) rq = fmaf(2.0f * ev[i - 1] * prev, v, rq);
-              prev = v;
+            for (int i0 = 0; i0 < n; i0 += 8) {
+              float v[8];
+#pragma unroll
+              for (int u = 0; u < 8; ++u)
+                if (i0 + u < n) v[u] = y[(size_t)(i0 + u) * n + t] * inv;
+#pragma unroll
+              for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u;
+                if (i < n) {
+                  y[(size_t)i * n + t] = v[u];
+                  rq = fmaf(dv[i] * v[u], v[u], rq);
+                  if (i > 0) rq = fmaf(2.0f * ev[i - 1] * prev, v[u], rq);
+                  prev = v[u];
+                }
+              }
             }
             e2[t] = rq;  // Rayleigh quotient on T (e2 is free after the bisection)
           }
