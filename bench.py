@@ -159,6 +159,8 @@ def run_ours(args):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     tcb.lib()
+    if args.groups:
+        tcb.tc_set_groups(args.groups)
 
     cfg, name = workload(args)
     M, P, nA, nB = 0, 0, 0, 0
@@ -308,6 +310,7 @@ def main():
     ap.add_argument("--batch", type=int, default=64, help="images per GPU per step")
     ap.add_argument("--n-query", type=int, default=128)
     ap.add_argument("--keep", type=int, default=128)
+    ap.add_argument("--groups", type=int, default=0, help="concurrent image groups (0 = library default)")
     ap.add_argument("--cpu-images", type=int, default=12,
                     help="images the CPU oracle is timed on (0 = skip)")
     args = ap.parse_args()

@@ -189,6 +189,15 @@ tc_status tc_attn_score_noalloc(const tc_params* p, const void* A, float* S, voi
 tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream);
 
 /*
+ * Number of image groups tc_score / tc_carve run side by side (1..8, default 4; the paper has no
+ * counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
+ * chains are enqueued on internal streams forked from `stream` and joined back into it before
+ * the call's remaining kernels, so that the one-block-per-image solver kernels of one group
+ * overlap the GEMMs of another.  Results do not depend on the setting.  Process-wide.
+ */
+tc_status tc_set_groups(int32_t groups);
+
+/*
  * Optional event profile (diagnostics; the paper has no counterpart).  Between
  * tc_profile_begin() and tc_profile_end() every kernel launch of the library is bracketed by
  * CUDA events on its stream.  tc_profile_end() waits for those events and returns, per kernel

@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TC_OK", 1: "TC_ERR_INVALID_ARG", 2: "TC_ERR_UNSUPPORTED", 3:
 EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge", "tc_compact",
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
-           "tc_kernel_class_name", "tc_attn_score_noalloc")
+           "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups")
 
 
 class TcParams(C.Structure):
@@ -71,6 +71,7 @@ def lib() -> C.CDLL:
         L.tc_carve.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_carve_host.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_gram.argtypes = [pp, vp, vp, vp]
+        L.tc_set_groups.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
         L.tc_status_string.argtypes = [C.c_int32]
         L.tc_status_string.restype = C.c_char_p
@@ -78,7 +79,7 @@ def lib() -> C.CDLL:
         L.tc_kernel_class_name.restype = C.c_char_p
         L.tc_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int32]
         for name in EXPORTS:
-            if name not in ("tc_status_string", "tc_kernel_class_name", "tc_attn_score_noalloc"):
+            if name not in ("tc_status_string", "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups"):
                 getattr(L, name).restype = C.c_int32
         L.tc_launch_count.restype = C.c_int64
         _lib = L
@@ -275,6 +276,10 @@ def tc_carve_host(p: Params, O, A, X, K, V, out, ws):
 
 def tc_status_string(status: int) -> str:
     return lib().tc_status_string(status).decode()
+
+
+def tc_set_groups(groups: int) -> None:
+    _check("tc_set_groups", lib().tc_set_groups(C.c_int32(groups)))
 
 
 def tc_version() -> int:

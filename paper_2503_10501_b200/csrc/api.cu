@@ -175,14 +175,68 @@ static tc_status open_ctx(const tc_params* p, void* ws, size_t ws_bytes, void* s
   return TC_OK;
 }
 
-// score: S partial sums || Gram -> eigen-solve -> C -> E
+// ---- concurrent image groups ----------------------------------------------------------------
+// The Cholesky and eigen-solver kernels run one block per image and so leave most of the GPU
+// idle at batch sizes below the SM count.  The batch is therefore cut into a few groups whose
+// Gram -> eigen-solve chains run on separate internal streams, forked from and joined back into
+// the caller's stream with events: one group's single-block kernels overlap another group's
+// GEMMs.  Per-image results do not depend on the grouping.
+constexpr int kMaxGroups = 8;
+struct GroupStreams {
+  bool ready = false;
+  cudaStream_t s[kMaxGroups];
+  cudaEvent_t fork, join[kMaxGroups];
+};
+static std::mutex g_groups_mu;
+static GroupStreams g_groups[64];
+static std::atomic<int> g_n_groups{4};
+
+static GroupStreams* group_streams() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  GroupStreams& g = g_groups[dev];
+  if (!g.ready) {
+    for (int i = 0; i < kMaxGroups; ++i) {
+      if (cudaStreamCreateWithFlags(&g.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&g.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    if (cudaEventCreateWithFlags(&g.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    g.ready = true;
+  }
+  return &g;
+}
+
+// score: S partial sums || (Gram -> eigen-solve -> C per image group) -> E
 static void enqueue_score(const Ctx& c, const void* O, const void* A, float* E, float* C, float* S,
                           float* sigma, int32_t* rank, int32_t* img_status) {
   const Dims& D = c.D;
+  const int q = D.N < D.d ? D.N : D.d;
   fill_i32(img_status, D.B, 0, c.st);
+  int ng = g_n_groups.load();
+  if (ng > D.B) ng = D.B;
+  std::lock_guard<std::mutex> lk(g_groups_mu);
+  GroupStreams* gs = ng > 1 ? group_streams() : nullptr;
+  if (gs == nullptr) ng = 1;
+  if (ng > 1) cudaEventRecord(gs->fork, c.st);
   launch_attn_colsum(D, A, (float*)(c.ws + c.P.s_part), c.st);
-  launch_gram(D, O, (float*)(c.ws + c.P.G), img_status, c.st);
-  launch_ics(D, c.P, c.ws, O, C, sigma, rank, img_status, c.st);
+  const int base = D.B / ng, extra = D.B % ng;
+  int b0 = 0;
+  for (int g = 0; g < ng; ++g) {
+    const int nb = base + (g < extra ? 1 : 0);
+    cudaStream_t st = ng > 1 ? gs->s[g] : c.st;
+    if (ng > 1) cudaStreamWaitEvent(st, gs->fork, 0);
+    Dims Dg = D;
+    Dg.B = nb;
+    const char* Og = (const char*)O + (size_t)b0 * D.N * D.d * D.esz;
+    launch_gram(Dg, Og, (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N, img_status + b0, st);
+    launch_ics(Dg, c.P, c.ws, b0, Og, C + (size_t)b0 * D.N, sigma ? sigma + (size_t)b0 * q : nullptr,
+               rank ? rank + b0 : nullptr, img_status + b0, st);
+    if (ng > 1) {
+      cudaEventRecord(gs->join[g], st);
+      cudaStreamWaitEvent(c.st, gs->join[g], 0);
+    }
+    b0 += nb;
+  }
   launch_combine(D, (const float*)(c.ws + c.P.s_part), C, S, E, c.st);
 }
 
@@ -404,6 +458,12 @@ const char* tc_status_string(int32_t status) {
 }
 
 int32_t tc_version(void) { return 100; }
+
+tc_status tc_set_groups(int32_t groups) {
+  if (groups < 1 || groups > tc::kMaxGroups) return TC_ERR_INVALID_ARG;
+  tc::g_n_groups.store(groups);
+  return TC_OK;
+}
 
 int32_t tc_profile_begin(void) {
   std::lock_guard<std::mutex> lk(tc::g_prof.mu);

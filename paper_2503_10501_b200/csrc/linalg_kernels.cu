@@ -23,44 +23,55 @@ namespace tc {
 __device__ inline float ld_f32(const float* p) { return __ldg(p); }
 __device__ inline float ld_f32(const __half* p) { return __half2float(__ldg(p)); }
 
-template <typename TA, typename TB, bool TRA, bool TRB>
+// flags for structured products
+constexpr int GEMM_SYM = 1;       // C is symmetric (A^T A): tiles below the diagonal are mirrored
+constexpr int GEMM_B_UPPER = 2;   // opB[k][n] = 0 for k > n: the K loop stops at the tile's edge
+
+template <typename TA, typename TB, bool TRA, bool TRB, int RM>
 __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
                                                   const TB* __restrict__ B, float* __restrict__ C,
                                                   int M, int N, int K, int lda, int ldb, int ldc,
-                                                  size_t sA, size_t sB, size_t sC) {
-  constexpr int BM = 64, BN = 64, BK = 16;
-  __shared__ float As[BK][BM + 4];
-  __shared__ float Bs[BK][BN + 4];
+                                                  size_t sA, size_t sB, size_t sC, int flags) {
+  // (64 RM) x 64 tile per block, 16-deep slices, (4 RM) x 4 outputs per thread.  The next slice
+  // is fetched into registers while the current one is multiplied out of shared memory, whose
+  // rows are read four floats at a time.
+  constexpr int BM = 64 * RM, BN = 64, BK = 16;
+  constexpr int LA = BM * BK / 256, LB = BN * BK / 256;
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  if ((flags & GEMM_SYM) && n0 + BN <= m0) return;  // strictly below the diagonal
   A += (size_t)blockIdx.z * sA;
   B += (size_t)blockIdx.z * sB;
   C += (size_t)blockIdx.z * sC;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  float acc[4][4];
+  const int Kend = (flags & GEMM_B_UPPER) ? min(K, n0 + BN) : K;
+  float acc[4 * RM][4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 4 * RM; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  float ra[LA], rb[LB];
 
-  for (int k0 = 0; k0 < K; k0 += BK) {
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < LA; ++i) {
       const int e = tid + i * 256;
       int m, k;
       if (TRA) {
-        m = e & 63;
-        k = e >> 6;
+        m = e % BM;
+        k = e / BM;
       } else {
         k = e & 15;
         m = e >> 4;
       }
       const int gm = m0 + m, gk = k0 + k;
       float v = 0.f;
-      if (gm < M && gk < K) v = TRA ? ld_f32(A + (size_t)gk * lda + gm) : ld_f32(A + (size_t)gm * lda + gk);
-      As[k][m] = v;
+      if (gm < M && gk < Kend) v = TRA ? ld_f32(A + (size_t)gk * lda + gm) : ld_f32(A + (size_t)gm * lda + gk);
+      ra[i] = v;
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < LB; ++i) {
       const int e = tid + i * 256;
       int n, k;
       if (TRB) {
@@ -72,43 +83,79 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
       }
       const int gn = n0 + n, gk = k0 + k;
       float v = 0.f;
-      if (gn < N && gk < K) v = TRB ? ld_f32(B + (size_t)gn * ldb + gk) : ld_f32(B + (size_t)gk * ldb + gn);
-      Bs[k][n] = v;
+      if (gn < N && gk < Kend) v = TRB ? ld_f32(B + (size_t)gn * ldb + gk) : ld_f32(B + (size_t)gk * ldb + gn);
+      rb[i] = v;
     }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int i = 0; i < LA; ++i) {
+      const int e = tid + i * 256;
+      if (TRA) As[e / BM][e % BM] = ra[i];
+      else As[e & 15][e >> 4] = ra[i];
+    }
+#pragma unroll
+    for (int i = 0; i < LB; ++i) {
+      const int e = tid + i * 256;
+      if (TRB) Bs[e & 15][e >> 4] = rb[i];
+      else Bs[e >> 6][e & 63] = rb[i];
+    }
+  };
+
+  fetch(0);
+  for (int k0 = 0; k0 < Kend; k0 += BK) {
+    stash();
     __syncthreads();
+    if (k0 + BK < Kend) fetch(k0 + BK);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
-      float a[4], bb[4];
+      float4 av[RM];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+      for (int g = 0; g < RM; ++g) av[g] = *reinterpret_cast<const float4*>(&As[kk][g * 64 + ty * 4]);
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float bb[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
-      for (int j = 0; j < 4; ++j) bb[j] = Bs[kk][tx * 4 + j];
+      for (int g = 0; g < RM; ++g) {
+        const float a[4] = {av[g].x, av[g].y, av[g].z, av[g].w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+          for (int j = 0; j < 4; ++j) acc[g * 4 + i][j] = fmaf(a[i], bb[j], acc[g * 4 + i][j]);
+      }
     }
     __syncthreads();
   }
+  const bool mirror = (flags & GEMM_SYM) && (n0 >= m0 + BM);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int gm = m0 + ty * 4 + i;
-    if (gm >= M) continue;
+  for (int g = 0; g < RM; ++g)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int gn = n0 + tx * 4 + j;
-      if (gn < N) C[(size_t)gm * ldc + gn] = acc[i][j];
+    for (int i = 0; i < 4; ++i) {
+      const int gm = m0 + g * 64 + ty * 4 + i;
+      if (gm >= M) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gn = n0 + tx * 4 + j;
+        if (gn < N) {
+          C[(size_t)gm * ldc + gn] = acc[g * 4 + i][j];
+          if (mirror) C[(size_t)gn * ldc + gm] = acc[g * 4 + i][j];
+        }
+      }
     }
-  }
 }
 
 template <typename TA, typename TB, bool TRA, bool TRB>
 static void gemm(const TA* A, const TB* B, float* C, int M, int N, int K, int lda, int ldb,
                  int ldc, size_t sA, size_t sB, size_t sC, int batch, cudaStream_t st,
-                 int cls = KC_GEMM) {
+                 int cls = KC_GEMM, int flags = 0) {
   Scope scope_(cls, st);
-  dim3 grid((N + 63) / 64, (M + 63) / 64, batch);
-  { gemm_kernel<TA, TB, TRA, TRB><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC); note_launch(); }
+  // tall outputs take 128-row tiles; small square ones (k x k) keep 64 x 64 tiles
+  if (M >= 256 && !(flags & GEMM_SYM)) {
+    dim3 grid((N + 63) / 64, (M + 127) / 128, batch);
+    { gemm_kernel<TA, TB, TRA, TRB, 2><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
+  } else {
+    dim3 grid((N + 63) / 64, (M + 63) / 64, batch);
+    { gemm_kernel<TA, TB, TRA, TRB, 1><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
+  }
 }
 
 // G = O O^T for float32 inputs (and, until the tensor-core kernel takes over, float16 ones).
@@ -1133,15 +1180,17 @@ void fill_i32(int32_t* p, int n, int v, cudaStream_t st) {
 // ==========================================================================================
 // The whole of Eq. 3-5 / 3-6 for a batch, given G in the workspace.
 // ==========================================================================================
-void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_out,
+void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
                 float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st) {
+  // D.B images starting at image b0 of the workspace arrays; O and the outputs already point at
+  // image b0.
   const int B = D.B, N = D.N, k = D.k;
-  float* G = (float*)(ws + P.G);
-  float* W = (float*)(ws + P.W);
-  float* ZT = (float*)(ws + P.ZT);
-  float* theta = (float*)(ws + P.sigma);
   const int q = min(D.N, D.d);
   const size_t sG = (size_t)N * N, sY = (size_t)N * k, sK = (size_t)k * k;
+  float* G = (float*)(ws + P.G) + b0 * sG;
+  float* W = (float*)(ws + P.W) + b0 * sK;
+  float* ZT = (float*)(ws + P.ZT) + b0 * sK;
+  float* theta = (float*)(ws + P.sigma) + (size_t)b0 * k;
 
   if (D.full) {
     launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, nullptr, nullptr, nullptr, img_status, st);
@@ -1150,12 +1199,12 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_
                                                              img_status, N, N, q, D.rank_tol, 1); note_launch(); }
     return;
   }
-  float* Y0 = (float*)(ws + P.Y0);
-  float* Y1 = (float*)(ws + P.Y1);
-  float* Y2 = (float*)(ws + P.Y2);
-  float* Sm = (float*)(ws + P.Sm);
-  float* Rinv = (float*)(ws + P.Rinv);
-  float* Hm = (float*)(ws + P.Hm);
+  float* Y0 = (float*)(ws + P.Y0) + b0 * sY;
+  float* Y1 = (float*)(ws + P.Y1) + b0 * sY;
+  float* Y2 = (float*)(ws + P.Y2) + b0 * sY;
+  float* Sm = (float*)(ws + P.Sm) + b0 * sK;
+  float* Rinv = (float*)(ws + P.Rinv) + b0 * sK;
+  float* Hm = (float*)(ws + P.Hm) + b0 * sK;
 
   // 1. sketch of the column space of O
   {
@@ -1169,9 +1218,9 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_
   }
   // one Cholesky-QR pass: dst = src R^{-1},  R^T R = src^T src (+ shift)
   auto cholqr_pass = [&](const float* src, float* dst, float shift_rel) {
-    gemm<float, float, true, false>(src, src, Sm, k, k, N, k, k, k, sY, sY, sK, B, st);
+    gemm<float, float, true, false>(src, src, Sm, k, k, N, k, k, k, sY, sY, sK, B, st, KC_GEMM, GEMM_SYM);
     launch_chol_inv(Sm, Rinv, W, k, B, shift_rel, img_status, st);
-    gemm<float, float, false, true>(src, Rinv, dst, N, k, k, k, k, k, sY, sK, sY, B, st);
+    gemm<float, float, false, true>(src, Rinv, dst, N, k, k, k, k, k, sY, sK, sY, B, st, KC_GEMM, GEMM_B_UPPER);
   };
   const float kShift = 1e-6f;
   // 2. a well-conditioned (not orthonormal) basis Q0 of the sketch: one shifted pass takes the

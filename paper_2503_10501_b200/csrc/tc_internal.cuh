@@ -87,7 +87,7 @@ void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
 tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 
 // Eigen-decomposition of G and Eq. 3-6:  C, theta (unsorted), then sorted sigma / rank.
-void launch_ics(const Dims& D, const Plan& P, char* ws, const void* O, float* C_out,
+void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
                 float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st);
 
 }  // namespace tc
