@@ -80,7 +80,7 @@ CONFIGS: Dict[str, CarveConfig] = {
                                    rank=384, noise=0.01, tau=2.0, keep=640,
                                    rank_cap=736, near_frac=0.10, seed=4),
     "cfg5_sweep_f16": CarveConfig("cfg5_sweep_f16", 64, 576, 4096, 32, 128, 128, "f16",
-                                  rank=128, noise=0.01, tau=2.0, keep=128, rank_cap=160,
+                                  rank=128, noise=0.01, tau=2.0, keep=128, rank_cap=144,
                                   seed=5),
 }
 
