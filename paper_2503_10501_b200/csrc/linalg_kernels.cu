@@ -292,6 +292,7 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
                                                               int32_t* __restrict__ status) {
   extern __shared__ float A[];  // [k][ld], ld odd: rows and columns both walk all banks
   __shared__ float s_red[16];
+  __shared__ float s_row[2][CNB];
   __shared__ int s_bad;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ld = k | 1;
@@ -340,9 +341,13 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
         const float rinv = rsqrtf(piv);
         if (lane == i) col[i] = piv * rinv;
         else if (lane > i) col[i] = col[i] * rinv;
+        // row i of the factor goes through shared memory: broadcast reads pipeline, a chain
+        // of fifteen shuffles does not
+        if (lane < CNB) s_row[i & 1][lane] = col[i];
+        __syncwarp();
 #pragma unroll
         for (int r = i + 1; r < CNB; ++r) {
-          const float v = __shfl_sync(0xffffffffu, col[i], r);
+          const float v = s_row[i & 1][r];
           if (lane >= r) col[r] = fmaf(-v, col[i], col[r]);
         }
       }
@@ -456,26 +461,35 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
           if (c < w) A[r * ld + j0 + c] = tt[c];
       }
       __syncthreads();
-      // X[0:j0, J] = - X[0:j0, 0:j0] * T : all outputs into registers first, then written
-      float outv[8];
-      const int total = j0 * w;
+      // X[0:j0, J] = - X[0:j0, 0:j0] * T.  A thread owns one row r and four columns: four
+      // independent sums share each X[r][m].  All outputs stay in registers until every
+      // thread has finished reading T, then they overwrite it.
+      float o4[2][4];
+      const int items = j0 * (CNB / 4);
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
+      for (int q = 0; q < 2; ++q) {
         const int e = tid + q * 512;
-        float sacc = 0.f;
-        if (e < total) {
-          const int r = e / w, c = e - r * w;
-          for (int mm = r; mm < j0; ++mm) sacc = fmaf(A[r * ld + mm], A[mm * ld + j0 + c], sacc);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) o4[q][u] = 0.f;
+        if (e < items) {
+          const int r = e >> 2, c0 = j0 + ((e & 3) << 2);
+          for (int mm = r; mm < j0; ++mm) {
+            const float xv = A[r * ld + mm];
+            const float* trow = A + mm * ld + c0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) o4[q][u] = fmaf(xv, trow[u], o4[q][u]);
+          }
         }
-        outv[q] = -sacc;
       }
       __syncthreads();
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
+      for (int q = 0; q < 2; ++q) {
         const int e = tid + q * 512;
-        if (e < total) {
-          const int r = e / w, c = e - r * w;
-          A[r * ld + j0 + c] = outv[q];
+        if (e < items) {
+          const int r = e >> 2, c0 = j0 + ((e & 3) << 2);
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (c0 + u < j1) A[r * ld + c0 + u] = -o4[q][u];
         }
       }
       __syncthreads();
@@ -690,76 +704,89 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   __syncthreads();
 
   // ---------------- Householder tridiagonalisation ----------------
-  for (int j = 0; j + 2 < n; ++j) {
-    const int m = n - j - 1;  // length of the column below the diagonal
-    // sigma = |x|^2, x = A[j+1.., j]
+  // Three block barriers per column.  |x|^2 of the next column is gathered while the trailing
+  // block is updated; v and w live in registers (lane l keeps entries l, l + 32, ...).
+  constexpr int VR = 8;  // n <= 256
+  __shared__ float s_sig[16];
+  {
     float part = 0.f;
-    for (int r = tid; r < m; r += 512) {
-      const float x = A[(j + 1 + r) * ld + j];
+    for (int r = tid; r + 1 < n; r += 512) {
+      const float x = A[(1 + r) * ld];
       part = fmaf(x, x, part);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    if (lane == 0) s_red[warp] = part;
+    if (lane == 0) s_sig[warp] = part;
     __syncthreads();
+  }
+  for (int j = 0; j + 2 < n; ++j) {
+    const int m = n - j - 1;  // length of the column below the diagonal
     float sigma = 0.f;
 #pragma unroll
-    for (int w = 0; w < 16; ++w) sigma += s_red[w];
+    for (int w = 0; w < 16; ++w) sigma += s_sig[w];
     const float x0 = A[(j + 1) * ld + j];
     const float tail = sigma - x0 * x0;  // |x|^2 without its first entry
-    if (tid == 0) dv[j] = A[j * ld + j];
-    if (!(tail > 1e-30f * sigma) || !(sigma > 0.f)) {
-      // column already in tridiagonal form
-      if (tid == 0) {
-        ev[j] = x0;
-        beta[j] = 0.f;
-      }
-      __syncthreads();
-      continue;
-    }
-    const float alpha = -copysignf(sqrtf(sigma), x0);
-    const float v0 = x0 - alpha;
-    const float bj = 2.0f / (tail + v0 * v0);
+    // reflector H = I - bj v v^T with v = x - alpha e_1; a column already in tridiagonal form
+    // gets bj = 0 (H = I) and keeps its entries
+    const bool skip = !(tail > 1e-30f * sigma) || !(sigma > 0.f);
+    const float alpha = skip ? x0 : -copysignf(sqrtf(sigma), x0);
+    const float v0 = skip ? x0 : x0 - alpha;
+    const float bj = skip ? 0.f : 2.0f / (tail + v0 * v0);
     for (int r = tid; r < m; r += 512) {
       const float x = (r == 0) ? v0 : A[(j + 1 + r) * ld + j];
       vv[r] = x;
-      A[(j + 1 + r) * ld + j] = x;  // kept for the accumulation of Q
+      if (r == 0) A[(j + 1) * ld + j] = x;  // the column is kept for the accumulation of Q
     }
     if (tid == 0) {
+      dv[j] = A[j * ld + j];
       ev[j] = alpha;
       beta[j] = bj;
     }
     __syncthreads();
-    // p = beta * B v, one warp per row of the trailing block B = A[j+1.., j+1..]
+    float vreg[VR];
+#pragma unroll
+    for (int u = 0; u < VR; ++u) vreg[u] = (lane + 32 * u < m) ? vv[lane + 32 * u] : 0.f;
+    // p = bj * B v, one warp per row of the trailing block B = A[j+1.., j+1..]; v.p on the way
+    float vp_part = 0.f;
     for (int r = warp; r < m; r += 16) {
       const float* row = A + (j + 1 + r) * ld + j + 1;
       float acc = 0.f;
-      for (int c = lane; c < m; c += 32) acc = fmaf(row[c], vv[c], acc);
+#pragma unroll
+      for (int u = 0; u < VR; ++u)
+        if (lane + 32 * u < m) acc = fmaf(row[lane + 32 * u], vreg[u], acc);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (lane == 0) pv[r] = bj * acc;
+      if (lane == 0) {
+        const float pr = bj * acc;
+        pv[r] = pr;
+        vp_part = fmaf(vv[r], pr, vp_part);
+      }
     }
-    __syncthreads();
-    // K = beta/2 * v.p ;  w = p - K v  (every thread forms K itself from the same partial sums)
-    part = 0.f;
-    for (int r = tid; r < m; r += 512) part = fmaf(vv[r], pv[r], part);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    if (lane == 0) s_red[warp] = part;
+    if (lane == 0) s_red[warp] = vp_part;
     __syncthreads();
     float vp = 0.f;
 #pragma unroll
     for (int w = 0; w < 16; ++w) vp += s_red[w];
-    const float K = 0.5f * bj * vp;
-    __syncthreads();  // s_red is reused next step; pv is rewritten below
-    for (int r = tid; r < m; r += 512) pv[r] = fmaf(-K, vv[r], pv[r]);
-    __syncthreads();
-    // B -= v w^T + w v^T
+    const float K = 0.5f * bj * vp;  // w = p - K v
+    float wreg[VR];
+#pragma unroll
+    for (int u = 0; u < VR; ++u) wreg[u] = (lane + 32 * u < m) ? fmaf(-K, vreg[u], pv[lane + 32 * u]) : 0.f;
+    // B -= v w^T + w v^T ; the first column of the new B (below its top entry) is the next x
+    float sig_part = 0.f;
     for (int r = warp; r < m; r += 16) {
       float* row = A + (j + 1 + r) * ld + j + 1;
-      const float vr = vv[r], wr = pv[r];
-      for (int c = lane; c < m; c += 32) row[c] -= fmaf(vr, pv[c], wr * vv[c]);
+      const float vr = vv[r], wr = fmaf(-K, vr, pv[r]);
+#pragma unroll
+      for (int u = 0; u < VR; ++u) {
+        const int c = lane + 32 * u;
+        if (c < m) {
+          const float nv = row[c] - fmaf(vr, wreg[u], wr * vreg[u]);
+          row[c] = nv;
+          if (c == 0 && r >= 1) sig_part = fmaf(nv, nv, sig_part);
+        }
+      }
     }
+    if (lane == 0) s_sig[warp] = sig_part;
     __syncthreads();
   }
   if (tid == 0) {
@@ -805,8 +832,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         for (int r = r_lo; r < r_hi; ++r) A[r * ld + c] = fmaf(-bt, A[r * ld + j], A[r * ld + c]);
         if (g == 0) A[(j + 1) * ld + c] = -bt * A[(j + 1) * ld + j];
       }
-      __syncthreads();
-      // column j+1: H_j e_{j+1}
+      // column j+1: H_j e_{j+1} (touches no column the threads above work on)
       const float vj1 = A[(j + 1) * ld + j];
       for (int r = j + 2 + tid; r < n; r += 512) A[r * ld + j + 1] = -bj * A[r * ld + j] * vj1;
       if (tid == 0) A[(j + 1) * ld + j + 1] = 1.0f - bj * vj1 * vj1;
@@ -856,7 +882,37 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     const float pivmin = fmaxf(tn, 1e-30f) * 1e-12f;
     lo -= 2.4e-7f * tn + pivmin;
     hi += 2.4e-7f * tn + pivmin;
-    if (tid < n) {
+    if (3 * ((n + 9) / 10) * 10 <= 480 + 30 && n <= 160) {
+      // three lanes per eigenvalue, ten eigenvalues per warp: each round evaluates the Sturm
+      // count at the three quarter points of the bracket, which shrinks it four-fold
+      const int t = warp * 10 + lane / 3, jj = lane % 3;
+      const bool on = (lane < 30) && (t < n);
+      const int base = lane - jj;
+      float a = lo, bhi = hi;
+      for (int it = 0; it < 24; ++it) {
+        const float step = 0.25f * (bhi - a);
+        const float x = a + step * (float)(jj + 1);
+        int cnt = 0;
+        if (on) {
+          float q = dv[0] - x;
+          cnt = q < 0.f;
+          for (int i = 1; i < n; ++i) {
+            if (fabsf(q) < pivmin) q = -pivmin;
+            q = dv[i] - x - __fdividef(e2[i - 1], q);
+            cnt += q < 0.f;
+          }
+        }
+        const int c0 = __shfl_sync(0xffffffffu, cnt, base & 31);
+        const int c1 = __shfl_sync(0xffffffffu, cnt, (base + 1) & 31);
+        const int c2 = __shfl_sync(0xffffffffu, cnt, (base + 2) & 31);
+        const float x0 = a + step, x1 = a + 2.0f * step, x2 = a + 3.0f * step;
+        if (c0 > t) bhi = x0;
+        else if (c1 > t) { a = x0; bhi = x1; }
+        else if (c2 > t) { a = x1; bhi = x2; }
+        else a = x2;
+      }
+      if (on && jj == 0) lam[t] = 0.5f * (a + bhi);
+    } else if (tid < n) {
       // eigenvalue number tid (0 = smallest): count(x) = number of eigenvalues below x
       float a = lo, bhi = hi;
       for (int it = 0; it < 48; ++it) {
@@ -1085,8 +1141,8 @@ static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, i
                             float shift_rel, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_CHOL, st);
   const size_t blocked = (size_t)k * (k | 1) * sizeof(float);
-  // (the blocked kernel keeps up to 8 outputs per thread in registers in its last step)
-  if (blocked <= SMEM_LIMIT && (size_t)k * CNB <= 8 * 512) {
+  // (the blocked kernel keeps 2 x 4 outputs per thread in registers in its last step)
+  if (blocked <= SMEM_LIMIT && (size_t)k * (CNB / 4) <= 2 * 512) {
     cudaFuncSetAttribute((const void*)chol_inv_blocked_kernel,
                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)blocked);
     { chol_inv_blocked_kernel<<<batch, 512, blocked, st>>>(S, RinvT, k, shift_rel, status); note_launch(); }
