@@ -673,14 +673,15 @@ __global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ H
 //   in   H [n][n] symmetric (only its symmetric part is used)
 //   out  theta [n] eigenvalues (ascending), ZT [n][n] with ZT[p][i] = component i of
 //        eigenvector p (all zero for eigenvalues under a quarter of the rank cut-off)
-//   scratch u0, u1, u2, yv: [n][n] float each, per image
+//   scratch u0, u1, u2, yv, ml: [n][n] float each, per image
 // One block (16 warps) per image.
 // ==========================================================================================
 __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ ZTg,
                                                          float* __restrict__ theta, int n, float rank_tol,
                                                          float* __restrict__ u0g, float* __restrict__ u1g,
-                                                         float* __restrict__ u2g, float* yg,
+                                                         float* __restrict__ u2g, float* yg, float* __restrict__ mlg,
+                                                         size_t ml_stride,
                                                          int32_t* __restrict__ status) {
   extern __shared__ float sm[];
   const int ld = n | 1;
@@ -879,29 +880,55 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       hi = fmaxf(hi, reinterpret_cast<float*>(cs)[w]);
     }
     const float tn = fmaxf(fabsf(lo), fabsf(hi));
-    const float pivmin = fmaxf(tn, 1e-30f) * 1e-12f;
-    lo -= 2.4e-7f * tn + pivmin;
-    hi += 2.4e-7f * tn + pivmin;
-    if (3 * ((n + 9) / 10) * 10 <= 480 + 30 && n <= 160) {
-      // three lanes per eigenvalue, ten eigenvalues per warp: each round evaluates the Sturm
-      // count at the three quarter points of the bracket, which shrinks it four-fold
+    lo -= 2.4e-7f * tn + 1e-30f;
+    hi += 2.4e-7f * tn + 1e-30f;
+    // Sturm count in product form on T / |T| (no division on the serial chain):
+    //   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1};
+    // the number of sign changes along the sequence is the number of eigenvalues below x.
+    // Both running values are rescaled together whenever they leave [1e-10, 1e10].
+    float* dn = beta;  // beta is free once Q has been formed
+    const float itn = 1.0f / fmaxf(tn, 1e-30f);
+    for (int i = tid; i < n; i += 512) {
+      dn[i] = dv[i] * itn;
+      e2[i] = e2[i] * itn * itn;
+    }
+    __syncthreads();
+    auto sturm = [&](float x) {
+      float p0 = 1.f, p1 = dn[0] - x;
+      int cnt = p1 < 0.f;
+      bool neg = p1 < 0.f;
+      for (int i = 1; i < n; ++i) {
+        const float p2 = fmaf(dn[i] - x, p1, -e2[i - 1] * p0);
+        const bool neg2 = (p2 < 0.f) || (p2 == 0.f && !neg);  // an exact zero counts as a change
+        cnt += (neg2 != neg);
+        neg = neg2;
+        p0 = p1;
+        p1 = p2;
+        // entries of the scaled matrix can be as small as rounding noise (1e-7 and below), so
+        // the pair can shrink by that much in a single step: re-centre it every step
+        const float sc = fmaxf(fabsf(p0), fabsf(p1));
+        if (sc < 1e-10f) {
+          p0 *= 1e20f;
+          p1 *= 1e20f;
+        } else if (sc > 1e10f) {
+          p0 *= 1e-20f;
+          p1 *= 1e-20f;
+        }
+      }
+      return cnt;
+    };
+    const float lon = lo * itn, hin = hi * itn;
+    if (n <= 160) {
+      // three lanes per eigenvalue, ten eigenvalues per warp: each round evaluates the count at
+      // the three quarter points of the bracket, which shrinks it four-fold
       const int t = warp * 10 + lane / 3, jj = lane % 3;
       const bool on = (lane < 30) && (t < n);
       const int base = lane - jj;
-      float a = lo, bhi = hi;
+      float a = lon, bhi = hin;
       for (int it = 0; it < 24; ++it) {
         const float step = 0.25f * (bhi - a);
         const float x = a + step * (float)(jj + 1);
-        int cnt = 0;
-        if (on) {
-          float q = dv[0] - x;
-          cnt = q < 0.f;
-          for (int i = 1; i < n; ++i) {
-            if (fabsf(q) < pivmin) q = -pivmin;
-            q = dv[i] - x - __fdividef(e2[i - 1], q);
-            cnt += q < 0.f;
-          }
-        }
+        const int cnt = on ? sturm(x) : 0;
         const int c0 = __shfl_sync(0xffffffffu, cnt, base & 31);
         const int c1 = __shfl_sync(0xffffffffu, cnt, (base + 1) & 31);
         const int c2 = __shfl_sync(0xffffffffu, cnt, (base + 2) & 31);
@@ -911,23 +938,15 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         else if (c2 > t) { a = x1; bhi = x2; }
         else a = x2;
       }
-      if (on && jj == 0) lam[t] = 0.5f * (a + bhi);
+      if (on && jj == 0) lam[t] = 0.5f * (a + bhi) * tn;
     } else if (tid < n) {
-      // eigenvalue number tid (0 = smallest): count(x) = number of eigenvalues below x
-      float a = lo, bhi = hi;
+      float a = lon, bhi = hin;
       for (int it = 0; it < 48; ++it) {
         const float x = 0.5f * (a + bhi);
         if (!(x > a) || !(x < bhi)) break;
-        float q = dv[0] - x;
-        int cnt = q < 0.f;
-        for (int i = 1; i < n; ++i) {
-          if (fabsf(q) < pivmin) q = -pivmin;
-          q = dv[i] - x - __fdividef(e2[i - 1], q);
-          cnt += q < 0.f;
-        }
-        if (cnt > tid) bhi = x; else a = x;
+        if (sturm(x) > tid) bhi = x; else a = x;
       }
-      lam[tid] = 0.5f * (a + bhi);
+      lam[tid] = 0.5f * (a + bhi) * tn;
     }
     tnorm = tn;
   }
@@ -941,6 +960,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     float* u1 = u1g + img;
     float* u2 = u2g + img;
     float* y = yg + img;
+    float* ml = mlg + (size_t)b * ml_stride;
     if (tid < n) {
       const int t = tid;
       float x = lam[t];
@@ -951,58 +971,71 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       if (t > 0 && x - lam[t - 1] < sep) x = lam[t - 1] + sep * (float)(1 + (t & 3));
       const float tiny = fmaxf(tnorm, 1e-30f) * 1.1920929e-7f;
       if (wanted) {
-        for (int it = 0; it < 3; ++it) {
-          // forward: eliminate the sub-diagonal with row interchanges, the right-hand side with it
+        // factor T - x I once, with row interchanges (|multiplier| <= 1).  Stored per row: the
+        // reciprocal pivot, the two entries right of it, and the multiplier, to which 4 is
+        // added when the rows were swapped.
+        {
           float a = dv[0] - x, bb = (n > 1) ? ev[0] : 0.f, c = 0.f;
-          float r = (it == 0) ? 1.f : y[t];
-          for (int i0 = 0; i0 + 1 < n; i0 += 8) {
-            float rnx[8];
+          for (int i = 0; i + 1 < n; ++i) {
+            const float sub = ev[i], dnx = dv[i + 1] - x, en = (i + 2 < n) ? ev[i + 1] : 0.f;
+            const bool sw = fabsf(a) < fabsf(sub);
+            float piv = sw ? sub : a;
+            const float oth = sw ? a : sub;
+            if (fabsf(piv) < tiny) piv = copysignf(tiny, piv);
+            const float rp = 1.0f / piv;
+            const float mlt = oth * rp;
+            const float p1 = sw ? dnx : bb, p2 = sw ? en : c;
+            const float q1 = sw ? bb : dnx, q2 = sw ? c : en;
+            u0[(size_t)i * n + t] = rp;
+            u1[(size_t)i * n + t] = p1;
+            u2[(size_t)i * n + t] = p2;
+            ml[(size_t)i * n + t] = sw ? mlt + 4.0f : mlt;
+            a = fmaf(-mlt, p1, q1);
+            bb = fmaf(-mlt, p2, q2);
+            c = 0.f;
+          }
+          if (fabsf(a) < tiny) a = copysignf(tiny, a);
+          u0[(size_t)(n - 1) * n + t] = 1.0f / a;
+          u1[(size_t)(n - 1) * n + t] = 0.f;
+          u2[(size_t)(n - 1) * n + t] = 0.f;
+        }
+        float scale = 1.f, nrm = 0.f;
+        for (int it = 0; it < 3; ++it) {
+          if (it > 0) {
+            // apply the elimination to the right-hand side (the previous solution, rescaled)
+            float cur = y[t] * scale;
+            for (int i0 = 0; i0 + 1 < n; i0 += 8) {
+              float nx[8], me[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-              rnx[u] = (it != 0 && i0 + u + 1 < n) ? y[(size_t)(i0 + u + 1) * n + t] : 1.f;
+              for (int u = 0; u < 8; ++u)
+                if (i0 + u + 1 < n) {
+                  nx[u] = y[(size_t)(i0 + u + 1) * n + t] * scale;
+                  me[u] = ml[(size_t)(i0 + u) * n + t];
+                }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const int i = i0 + u;
-              if (i + 1 < n) {
-                const float sub = ev[i], dn = dv[i + 1] - x, en = (i + 2 < n) ? ev[i + 1] : 0.f;
-                const float rn = rnx[u];
-                if (fabsf(a) >= fabsf(sub)) {
-                  if (fabsf(a) < tiny) a = copysignf(tiny, a);
-                  const float mlt = sub / a;
-                  u0[(size_t)i * n + t] = a;
-                  u1[(size_t)i * n + t] = bb;
-                  u2[(size_t)i * n + t] = c;
-                  y[(size_t)i * n + t] = r;
-                  a = fmaf(-mlt, bb, dn);
-                  bb = fmaf(-mlt, c, en);
-                  c = 0.f;
-                  r = (it == 0) ? 1.f : fmaf(-mlt, r, rn);
-                } else {
-                  const float mlt = a / sub;
-                  u0[(size_t)i * n + t] = sub;
-                  u1[(size_t)i * n + t] = dn;
-                  u2[(size_t)i * n + t] = en;
-                  y[(size_t)i * n + t] = (it == 0) ? 1.f : rn;
-                  a = fmaf(-mlt, dn, bb);
-                  bb = fmaf(-mlt, en, c);
-                  c = 0.f;
-                  r = (it == 0) ? 1.f : fmaf(-mlt, rn, r);
+              for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u;
+                if (i + 1 < n) {
+                  const bool sw = me[u] > 2.0f;
+                  const float mlt = sw ? me[u] - 4.0f : me[u];
+                  const float hi_ = sw ? nx[u] : cur, lo_ = sw ? cur : nx[u];
+                  y[(size_t)i * n + t] = hi_;
+                  cur = fmaf(-mlt, hi_, lo_);
                 }
               }
             }
+            y[(size_t)(n - 1) * n + t] = cur;
           }
-          if (fabsf(a) < tiny) a = copysignf(tiny, a);
-          // backward substitution, keeping the largest entry for the scaling.  The four global
-          // vectors are read eight rows at a time so their latency is paid once per group.
-          float y1 = r / a, y2 = 0.f, big = fabsf(y1);
-          y[(size_t)(n - 1) * n + t] = y1;
-          for (int i1 = n - 2; i1 >= 0; i1 -= 8) {
+          // back substitution (first pass: right-hand side of ones), eight rows per group of loads
+          float y1 = 0.f, y2 = 0.f, big = 0.f;
+          nrm = 0.f;
+          for (int i1 = n - 1; i1 >= 0; i1 -= 8) {
             float rh[8], p0[8], p1[8], p2[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
               const int i = i1 - u;
               if (i >= 0) {
-                rh[u] = y[(size_t)i * n + t];
+                rh[u] = (it == 0) ? 1.f : y[(size_t)i * n + t];
                 p0[u] = u0[(size_t)i * n + t];
                 p1[u] = u1[(size_t)i * n + t];
                 p2[u] = u2[(size_t)i * n + t];
@@ -1012,50 +1045,38 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
             for (int u = 0; u < 8; ++u) {
               const int i = i1 - u;
               if (i >= 0) {
-                const float yi = (rh[u] - p1[u] * y1 - p2[u] * y2) / p0[u];
+                const float yi = (rh[u] - p1[u] * y1 - p2[u] * y2) * p0[u];
                 y[(size_t)i * n + t] = yi;
                 big = fmaxf(big, fabsf(yi));
+                nrm = fmaf(yi, yi, nrm);
                 y2 = y1;
                 y1 = yi;
               }
             }
           }
-          // scale to unit maximum (keeps the next solve in range); the last pass normalises
-          const float sc = 1.0f / fmaxf(big, 1e-30f);
-          float nrm = 0.f;
+          scale = 1.0f / fmaxf(big, 1e-30f);  // keeps the next right-hand side in range
+        }
+        {
+          // normalise; Rayleigh quotient on T
+          const float inv = rsqrtf(fmaxf(nrm * scale * scale, 1e-30f)) * scale;
+          float rq = 0.f, prev = 0.f;
           for (int i0 = 0; i0 < n; i0 += 8) {
             float v[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u)
-              if (i0 + u < n) v[u] = y[(size_t)(i0 + u) * n + t] * sc;
+              if (i0 + u < n) v[u] = y[(size_t)(i0 + u) * n + t] * inv;
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if (i0 + u < n) {
-                y[(size_t)(i0 + u) * n + t] = v[u];
-                nrm = fmaf(v[u], v[u], nrm);
-              }
-          }
-          if (it == 2) {
-            const float inv = rsqrtf(fmaxf(nrm, 1e-30f));
-            float rq = 0.f, prev = 0.f;
-            for (int i0 = 0; i0 < n; i0 += 8) {
-              float v[8];
-#pragma unroll
-              for (int u = 0; u < 8; ++u)
-                if (i0 + u < n) v[u] = y[(size_t)(i0 + u) * n + t] * inv;
-#pragma unroll
-              for (int u = 0; u < 8; ++u) {
-                const int i = i0 + u;
-                if (i < n) {
-                  y[(size_t)i * n + t] = v[u];
-                  rq = fmaf(dv[i] * v[u], v[u], rq);
-                  if (i > 0) rq = fmaf(2.0f * ev[i - 1] * prev, v[u], rq);
-                  prev = v[u];
-                }
+            for (int u = 0; u < 8; ++u) {
+              const int i = i0 + u;
+              if (i < n) {
+                y[(size_t)i * n + t] = v[u];
+                rq = fmaf(dv[i] * v[u], v[u], rq);
+                if (i > 0) rq = fmaf(2.0f * ev[i - 1] * prev, v[u], rq);
+                prev = v[u];
               }
             }
-            e2[t] = rq;  // Rayleigh quotient on T (e2 is free after the bisection)
           }
+          e2[t] = rq;  // e2 is free after the bisection
         }
       } else {
         for (int i = 0; i < n; ++i) y[(size_t)i * n + t] = 0.f;
@@ -1111,13 +1132,13 @@ constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared 
 
 static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
                           int max_sweeps, float rank_tol, float* scr1, float* scr2, float* scr3,
-                          int32_t* status, cudaStream_t st) {
+                          float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_JACOBI, st);
   {
     const size_t tri = ((size_t)n * (n | 1) + 9 * (size_t)n) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       cudaFuncSetAttribute((const void*)tridiag_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
-      { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, status); note_launch(); }
+      { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status); note_launch(); }
       return;
     }
   }
@@ -1249,7 +1270,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   float* theta = (float*)(ws + P.sigma) + (size_t)b0 * k;
 
   if (D.full) {
-    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, nullptr, nullptr, nullptr, img_status, st);
+    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, nullptr, nullptr, nullptr, nullptr, 0, img_status, st);
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<B, 256, 2 * (size_t)N * sizeof(float), st>>>(theta, ZT, C_out, sigma_out, rank_out,
                                                              img_status, N, N, q, D.rank_tol, 1); note_launch(); }
@@ -1291,7 +1312,8 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   // 4. Rayleigh-Ritz:  H = Q1^T G Q1
   gemm<float, float, false, false>(G, Y2, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);   // T = G Q1
   gemm<float, float, true, false>(Y2, Y1, Hm, k, k, N, k, k, k, sY, sY, sK, B, st);   // H = Q1^T T
-  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, Sm, Rinv, Hm, img_status, st);
+  // scratch of the solver: W, Sm, Rinv, Hm (k x k each) and the first k x k of each image's Y1 panel
+  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, Sm, Rinv, Hm, Y1, sY, img_status, st);
   // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]
   gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
   Scope scope_(KC_ICS, st);
