@@ -27,15 +27,15 @@ __device__ inline float ld_f32(const __half* p) { return __half2float(__ldg(p));
 constexpr int GEMM_SYM = 1;       // C is symmetric (A^T A): tiles below the diagonal are mirrored
 constexpr int GEMM_B_UPPER = 2;   // opB[k][n] = 0 for k > n: the K loop stops at the tile's edge
 
-template <typename TA, typename TB, bool TRA, bool TRB, int RM>
+template <typename TA, typename TB, bool TRA, bool TRB, int RM, int CN>
 __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
                                                   const TB* __restrict__ B, float* __restrict__ C,
                                                   int M, int N, int K, int lda, int ldb, int ldc,
                                                   size_t sA, size_t sB, size_t sC, int flags) {
-  // (64 RM) x 64 tile per block, 16-deep slices, (4 RM) x 4 outputs per thread.  The next slice
-  // is fetched into registers while the current one is multiplied out of shared memory, whose
-  // rows are read four floats at a time.
-  constexpr int BM = 64 * RM, BN = 64, BK = 16;
+  // (64 RM) x (16 CN) tile per block, 16-deep slices, (4 RM) x CN outputs per thread.  The next
+  // slice is fetched into registers while the current one is multiplied out of shared memory.
+  // CN = 4 gives 64-column tiles, CN = 3 gives 48-column tiles (for widths like 144 = 3 * 48).
+  constexpr int BM = 64 * RM, BN = 16 * CN, BK = 16;
   constexpr int LA = BM * BK / 256, LB = BN * BK / 256;
   __shared__ __align__(16) float As[BK][BM + 4];
   __shared__ __align__(16) float Bs[BK][BN + 4];
@@ -46,11 +46,11 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
   C += (size_t)blockIdx.z * sC;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int Kend = (flags & GEMM_B_UPPER) ? min(K, n0 + BN) : K;
-  float acc[4 * RM][4];
+  float acc[4 * RM][CN];
 #pragma unroll
   for (int i = 0; i < 4 * RM; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int j = 0; j < CN; ++j) acc[i][j] = 0.f;
   float ra[LA], rb[LB];
 
   auto fetch = [&](int k0) {
@@ -78,8 +78,8 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
         k = e & 15;
         n = e >> 4;
       } else {
-        n = e & 63;
-        k = e >> 6;
+        n = e % BN;
+        k = e / BN;
       }
       const int gn = n0 + n, gk = k0 + k;
       float v = 0.f;
@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
     for (int i = 0; i < LB; ++i) {
       const int e = tid + i * 256;
       if (TRB) Bs[e & 15][e >> 4] = rb[i];
-      else Bs[e >> 6][e & 63] = rb[i];
+      else Bs[e / BN][e % BN] = rb[i];
     }
   };
 
@@ -112,20 +112,28 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
       float4 av[RM];
 #pragma unroll
       for (int g = 0; g < RM; ++g) av[g] = *reinterpret_cast<const float4*>(&As[kk][g * 64 + ty * 4]);
-      const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-      const float bb[4] = {bv.x, bv.y, bv.z, bv.w};
+      float bb[CN];
+      if (CN == 4) {
+        const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+        bb[0] = bv.x; bb[1] = bv.y; bb[2] = bv.z; bb[CN - 1] = bv.w;
+      } else {
+#pragma unroll
+        for (int j = 0; j < CN; ++j) bb[j] = Bs[kk][tx * CN + j];
+      }
 #pragma unroll
       for (int g = 0; g < RM; ++g) {
         const float a[4] = {av[g].x, av[g].y, av[g].z, av[g].w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int j = 0; j < 4; ++j) acc[g * 4 + i][j] = fmaf(a[i], bb[j], acc[g * 4 + i][j]);
+          for (int j = 0; j < CN; ++j) acc[g * 4 + i][j] = fmaf(a[i], bb[j], acc[g * 4 + i][j]);
       }
     }
     __syncthreads();
   }
-  const bool mirror = (flags & GEMM_SYM) && (n0 >= m0 + BM);
+  // symmetric output: a tile writes its entries on or above the diagonal and their mirror
+  // images, so each pair is produced exactly once and C is symmetric bit for bit
+  const bool sym = (flags & GEMM_SYM) != 0;
 #pragma unroll
   for (int g = 0; g < RM; ++g)
 #pragma unroll
@@ -133,14 +141,22 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
       const int gm = m0 + g * 64 + ty * 4 + i;
       if (gm >= M) continue;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int gn = n0 + tx * 4 + j;
-        if (gn < N) {
+      for (int j = 0; j < CN; ++j) {
+        const int gn = n0 + tx * CN + j;
+        if (gn < N && (!sym || gn >= gm)) {
           C[(size_t)gm * ldc + gn] = acc[g * 4 + i][j];
-          if (mirror) C[(size_t)gn * ldc + gm] = acc[g * 4 + i][j];
+          if (sym && gn > gm) C[(size_t)gn * ldc + gm] = acc[g * 4 + i][j];
         }
       }
     }
+}
+
+template <typename TA, typename TB, bool TRA, bool TRB, int RM, int CN>
+static void gemm_launch(const TA* A, const TB* B, float* C, int M, int N, int K, int lda, int ldb,
+                        int ldc, size_t sA, size_t sB, size_t sC, int batch, cudaStream_t st,
+                        int flags) {
+  dim3 grid((N + 16 * CN - 1) / (16 * CN), (M + 64 * RM - 1) / (64 * RM), batch);
+  { gemm_kernel<TA, TB, TRA, TRB, RM, CN><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
 }
 
 template <typename TA, typename TB, bool TRA, bool TRB>
@@ -148,13 +164,14 @@ static void gemm(const TA* A, const TB* B, float* C, int M, int N, int K, int ld
                  int ldc, size_t sA, size_t sB, size_t sC, int batch, cudaStream_t st,
                  int cls = KC_GEMM, int flags = 0) {
   Scope scope_(cls, st);
-  // tall outputs take 128-row tiles; small square ones (k x k) keep 64 x 64 tiles
+  // column tiles of 48 when they pad the width less than tiles of 64 (e.g. 144 = 3 * 48)
+  const bool narrow = ((N + 47) / 48) * 48 < ((N + 63) / 64) * 64;
   if (M >= 256 && !(flags & GEMM_SYM)) {
-    dim3 grid((N + 63) / 64, (M + 127) / 128, batch);
-    { gemm_kernel<TA, TB, TRA, TRB, 2><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
+    if (narrow) gemm_launch<TA, TB, TRA, TRB, 2, 3>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, batch, st, flags);
+    else gemm_launch<TA, TB, TRA, TRB, 2, 4>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, batch, st, flags);
   } else {
-    dim3 grid((N + 63) / 64, (M + 63) / 64, batch);
-    { gemm_kernel<TA, TB, TRA, TRB, 1><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
+    if (narrow) gemm_launch<TA, TB, TRA, TRB, 1, 3>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, batch, st, flags);
+    else gemm_launch<TA, TB, TRA, TRB, 1, 4>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, batch, st, flags);
   }
 }
 
