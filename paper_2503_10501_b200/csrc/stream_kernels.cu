@@ -73,14 +73,14 @@ __global__ void attn_colsum_kernel(const T* __restrict__ A, float* __restrict__ 
     if (cg < ncg) {
       int r = r_begin + threadIdx.y;
       if (VECTOR) {
-        // four independent 16-byte loads in flight per thread
-        for (; r + 3 * by < r_end; r += 4 * by) {
-          uint4 v[4];
+        // eight independent 16-byte loads in flight per thread
+        for (; r + 7 * by < r_end; r += 8 * by) {
+          uint4 v[8];
 #pragma unroll
-          for (int u = 0; u < 4; ++u)
+          for (int u = 0; u < 8; ++u)
             v[u] = __ldg(reinterpret_cast<const uint4*>(Ab + (size_t)(r + u * by) * N) + cg);
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < 8; ++u) {
             float f[8];
             Vec16<T>::unpack(v[u], f);
 #pragma unroll
