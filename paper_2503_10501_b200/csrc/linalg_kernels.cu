@@ -51,9 +51,57 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
   for (int i = 0; i < 4 * RM; ++i)
 #pragma unroll
     for (int j = 0; j < CN; ++j) acc[i][j] = 0.f;
-  float ra[LA], rb[LB];
+  // Slices are fetched as 16-byte vectors along the contiguous direction of each operand when
+  // every address involved is 16-byte aligned (float32 operands, leading dimensions, sizes and
+  // batch strides multiples of four); otherwise element by element.
+  constexpr bool F32 = (sizeof(TA) == 4) && (sizeof(TB) == 4);
+  const bool vec = F32 && ((lda | ldb | M | N | K) & 3) == 0 && ((sA | sB) & 3) == 0 &&
+                   ((((uintptr_t)A) | ((uintptr_t)B)) & 15) == 0;
+  constexpr int VA = LA / 4, VB = (LB + 3) / 4;  // vectors per thread (B: some threads idle)
+  float ra[LA], rb[VB * 4];
 
   auto fetch = [&](int k0) {
+    if (vec) {
+#pragma unroll
+      for (int i = 0; i < VA; ++i) {
+        const int e = tid + i * 256;  // vector index inside the A slice
+        int m, k;
+        if (TRA) {  // stored [k][m]: vectors run along m
+          m = (e % (BM / 4)) * 4;
+          k = e / (BM / 4);
+        } else {  // stored [m][k]: vectors run along k
+          k = (e & 3) * 4;
+          m = e >> 2;
+        }
+        const int gm = m0 + m, gk = k0 + k;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (gm < M && gk < Kend)
+          v = __ldg(reinterpret_cast<const float4*>(
+              TRA ? (const float*)A + (size_t)gk * lda + gm : (const float*)A + (size_t)gm * lda + gk));
+        ra[4 * i] = v.x; ra[4 * i + 1] = v.y; ra[4 * i + 2] = v.z; ra[4 * i + 3] = v.w;
+      }
+#pragma unroll
+      for (int i = 0; i < VB; ++i) {
+        const int e = tid + i * 256;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e < BN * BK / 4) {
+          int n, k;
+          if (TRB) {  // stored [n][k]: vectors run along k
+            k = (e & 3) * 4;
+            n = e >> 2;
+          } else {  // stored [k][n]: vectors run along n
+            n = (e % (BN / 4)) * 4;
+            k = e / (BN / 4);
+          }
+          const int gn = n0 + n, gk = k0 + k;
+          if (gn < N && gk < Kend)
+            v = __ldg(reinterpret_cast<const float4*>(
+                TRB ? (const float*)B + (size_t)gn * ldb + gk : (const float*)B + (size_t)gk * ldb + gn));
+        }
+        rb[4 * i] = v.x; rb[4 * i + 1] = v.y; rb[4 * i + 2] = v.z; rb[4 * i + 3] = v.w;
+      }
+      return;
+    }
 #pragma unroll
     for (int i = 0; i < LA; ++i) {
       const int e = tid + i * 256;
@@ -88,6 +136,35 @@ __global__ void __launch_bounds__(256) gemm_kernel(const TA* __restrict__ A,
     }
   };
   auto stash = [&]() {
+    if (vec) {
+#pragma unroll
+      for (int i = 0; i < VA; ++i) {
+        const int e = tid + i * 256;
+        if (TRA) {
+          const int m = (e % (BM / 4)) * 4, k = e / (BM / 4);
+          *reinterpret_cast<float4*>(&As[k][m]) = make_float4(ra[4 * i], ra[4 * i + 1], ra[4 * i + 2], ra[4 * i + 3]);
+        } else {
+          const int k = (e & 3) * 4, m = e >> 2;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) As[k + u][m] = ra[4 * i + u];
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < VB; ++i) {
+        const int e = tid + i * 256;
+        if (e < BN * BK / 4) {
+          if (TRB) {
+            const int k = (e & 3) * 4, n = e >> 2;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) Bs[k + u][n] = rb[4 * i + u];
+          } else {
+            const int n = (e % (BN / 4)) * 4, k = e / (BN / 4);
+            *reinterpret_cast<float4*>(&Bs[k][n]) = make_float4(rb[4 * i], rb[4 * i + 1], rb[4 * i + 2], rb[4 * i + 3]);
+          }
+        }
+      }
+      return;
+    }
 #pragma unroll
     for (int i = 0; i < LA; ++i) {
       const int e = tid + i * 256;
