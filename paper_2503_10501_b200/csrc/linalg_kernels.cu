@@ -287,6 +287,47 @@ __global__ void sketch_kernel(const T* __restrict__ O, float* __restrict__ Y, in
   Y[((size_t)b * N + x) * k + j] = acc;
 }
 
+// The same sketch with 16-byte loads, for k a multiple of the vector length L (8 halves or 4
+// floats): columns are taken in groups of L, group g goes to bucket group g mod (k / L), column
+// i of the group to bucket i of that bucket group.  block (k / L, rows), grid (N / rows, B).
+template <typename T, int L>
+__global__ void sketch_vec_kernel(const T* __restrict__ O, float* __restrict__ Y, int N, int d, int k) {
+  extern __shared__ float sgn[];  // [d]
+  const int kg = blockDim.x, tx = threadIdx.x, ty = threadIdx.y;
+  const int b = blockIdx.y, x = blockIdx.x * blockDim.y + ty;
+  for (int c = ty * kg + tx; c < d; c += kg * blockDim.y) sgn[c] = hash_sign((uint32_t)c);
+  __syncthreads();
+  if (x >= N) return;
+  const uint4* row = reinterpret_cast<const uint4*>(O + ((size_t)b * N + x) * d);
+  const int ng = d / L;
+  float acc[L];
+#pragma unroll
+  for (int i = 0; i < L; ++i) acc[i] = 0.f;
+  int g = tx;
+  for (; g + 3 * kg < ng; g += 4 * kg) {
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = __ldg(row + g + u * kg);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const T* e = reinterpret_cast<const T*>(&v[u]);
+      const float* sg = sgn + (size_t)(g + u * kg) * L;
+#pragma unroll
+      for (int i = 0; i < L; ++i) acc[i] = fmaf(sg[i], (float)e[i], acc[i]);
+    }
+  }
+  for (; g < ng; g += kg) {
+    const uint4 v = __ldg(row + g);
+    const T* e = reinterpret_cast<const T*>(&v);
+    const float* sg = sgn + (size_t)g * L;
+#pragma unroll
+    for (int i = 0; i < L; ++i) acc[i] = fmaf(sg[i], (float)e[i], acc[i]);
+  }
+  float* out = Y + ((size_t)b * N + x) * k + tx * L;
+#pragma unroll
+  for (int i = 0; i < L; ++i) out[i] = acc[i];
+}
+
 // ==========================================================================================
 // Cholesky factor of S (+ shift) and its inverse.  One block per image.
 //   S [k][k] symmetric in;  RinvT [k][k] out, RinvT[c][m] = (R^{-1})[m][c] for m <= c, else 0,
@@ -1380,12 +1421,24 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   // 1. sketch of the column space of O
   {
     Scope scope_(KC_SKETCH, st);
-    dim3 grid(N, B);
-    const int threads = (k + 31) / 32 * 32;
-    if (D.f16)
-      { sketch_kernel<__half><<<grid, threads, 0, st>>>((const __half*)O, Y0, N, D.d, k); note_launch(); }
-    else
-      { sketch_kernel<float><<<grid, threads, 0, st>>>((const float*)O, Y0, N, D.d, k); note_launch(); }
+    const int L = D.f16 ? 8 : 4;
+    if (k % L == 0 && k / L <= 256 && (size_t)D.d * sizeof(float) <= 48 * 1024) {
+      const int kg = k / L;
+      const int rows = max(1, 256 / kg);
+      dim3 block(kg, rows), grid((N + rows - 1) / rows, B);
+      const size_t smem = (size_t)D.d * sizeof(float);
+      if (D.f16)
+        { sketch_vec_kernel<__half, 8><<<grid, block, smem, st>>>((const __half*)O, Y0, N, D.d, k); note_launch(); }
+      else
+        { sketch_vec_kernel<float, 4><<<grid, block, smem, st>>>((const float*)O, Y0, N, D.d, k); note_launch(); }
+    } else {
+      dim3 grid(N, B);
+      const int threads = (k + 31) / 32 * 32;
+      if (D.f16)
+        { sketch_kernel<__half><<<grid, threads, 0, st>>>((const __half*)O, Y0, N, D.d, k); note_launch(); }
+      else
+        { sketch_kernel<float><<<grid, threads, 0, st>>>((const float*)O, Y0, N, D.d, k); note_launch(); }
+    }
   }
   // one Cholesky-QR pass: dst = src R^{-1},  R^T R = src^T src (+ shift)
   auto cholqr_pass = [&](const float* src, float* dst, float shift_rel) {
