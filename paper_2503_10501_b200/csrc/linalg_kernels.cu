@@ -840,23 +840,25 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   __syncthreads();
 
   // ---------------- Householder tridiagonalisation ----------------
-  // Three block barriers per column.  |x|^2 of the next column is gathered while the trailing
-  // block is updated; v and w live in registers (lane l keeps entries l, l + 32, ...).
-  constexpr int VR = 8;  // n <= 256
+  // Four block barriers per column and no warp reductions inside the O(m^2) parts: a thread owns
+  // one column c of the trailing block and a range of its rows (the block is symmetric, so the
+  // column sum over that range is a partial of (B v)_c); the ranges are combined through shared
+  // memory.  |x|^2 of the next column is gathered while the trailing block is updated.
   __shared__ float s_sig[16];
+  float* part = reinterpret_cast<float*>(cs);  // [<= 4][n] partial products (cs is free here)
   {
-    float part = 0.f;
+    float ps = 0.f;
     for (int r = tid; r + 1 < n; r += 512) {
       const float x = A[(1 + r) * ld];
-      part = fmaf(x, x, part);
+      ps = fmaf(x, x, ps);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    if (lane == 0) s_sig[warp] = part;
+    for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+    if (lane == 0) s_sig[warp] = ps;
     __syncthreads();
   }
   for (int j = 0; j + 2 < n; ++j) {
-    const int m = n - j - 1;  // length of the column below the diagonal
+    const int m = n - j - 1;  // order of the trailing block B = A[j+1.., j+1..]
     float sigma = 0.f;
 #pragma unroll
     for (int w = 0; w < 16; ++w) sigma += s_sig[w];
@@ -879,49 +881,54 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       beta[j] = bj;
     }
     __syncthreads();
-    float vreg[VR];
-#pragma unroll
-    for (int u = 0; u < VR; ++u) vreg[u] = (lane + 32 * u < m) ? vv[lane + 32 * u] : 0.f;
-    // p = bj * B v, one warp per row of the trailing block B = A[j+1.., j+1..]; v.p on the way
-    float vp_part = 0.f;
-    for (int r = warp; r < m; r += 16) {
-      const float* row = A + (j + 1 + r) * ld + j + 1;
-      float acc = 0.f;
-#pragma unroll
-      for (int u = 0; u < VR; ++u)
-        if (lane + 32 * u < m) acc = fmaf(row[lane + 32 * u], vreg[u], acc);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (lane == 0) {
-        const float pr = bj * acc;
-        pv[r] = pr;
-        vp_part = fmaf(vv[r], pr, vp_part);
+    // thread layout of this step: cw warps cover the m columns, G row ranges side by side
+    const int cw = (m + 31) >> 5;
+    const int G = min(4, 16 / cw);
+    const int g = warp / cw, c = (warp - g * cw) * 32 + lane;
+    const bool on = (g < G) && (c < m);
+    const int per = (m + G - 1) / G;
+    const int r_lo = g * per, r_hi = min(m, r_lo + per);
+    float* colp = A + (j + 1) * ld + j + 1 + c;  // B[0][c]; rows are ld apart
+    if (on) {
+      float a0 = 0.f, a1 = 0.f;
+      int r = r_lo;
+      for (; r + 1 < r_hi; r += 2) {
+        a0 = fmaf(colp[r * ld], vv[r], a0);
+        a1 = fmaf(colp[(r + 1) * ld], vv[r + 1], a1);
       }
+      if (r < r_hi) a0 = fmaf(colp[r * ld], vv[r], a0);
+      part[g * n + c] = a0 + a1;
     }
-    if (lane == 0) s_red[warp] = vp_part;
+    __syncthreads();
+    // p = bj * B v ; v.p
+    float vpp = 0.f;
+    if (g == 0 && c < m) {
+      float t = 0.f;
+      for (int q = 0; q < G; ++q) t += part[q * n + c];
+      const float pc = bj * t;
+      pv[c] = pc;
+      vpp = vv[c] * pc;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) vpp += __shfl_xor_sync(0xffffffffu, vpp, o);
+    if (lane == 0) s_red[warp] = vpp;
     __syncthreads();
     float vp = 0.f;
 #pragma unroll
     for (int w = 0; w < 16; ++w) vp += s_red[w];
     const float K = 0.5f * bj * vp;  // w = p - K v
-    float wreg[VR];
-#pragma unroll
-    for (int u = 0; u < VR; ++u) wreg[u] = (lane + 32 * u < m) ? fmaf(-K, vreg[u], pv[lane + 32 * u]) : 0.f;
-    // B -= v w^T + w v^T ; the first column of the new B (below its top entry) is the next x
+    // B -= v w^T + w v^T ; column 0 of the new B, below its top entry, is the next x
     float sig_part = 0.f;
-    for (int r = warp; r < m; r += 16) {
-      float* row = A + (j + 1 + r) * ld + j + 1;
-      const float vr = vv[r], wr = fmaf(-K, vr, pv[r]);
-#pragma unroll
-      for (int u = 0; u < VR; ++u) {
-        const int c = lane + 32 * u;
-        if (c < m) {
-          const float nv = row[c] - fmaf(vr, wreg[u], wr * vreg[u]);
-          row[c] = nv;
-          if (c == 0 && r >= 1) sig_part = fmaf(nv, nv, sig_part);
-        }
+    if (on) {
+      const float vc = vv[c], wc = fmaf(-K, vc, pv[c]);
+      for (int r = r_lo; r < r_hi; ++r) {
+        const float vr = vv[r], wr = fmaf(-K, vr, pv[r]);
+        const float nv = colp[r * ld] - fmaf(vr, wc, wr * vc);
+        colp[r * ld] = nv;
+        if (c == 0 && r >= 1) sig_part = fmaf(nv, nv, sig_part);
       }
     }
+    // only lane 0 of the first warp of each range holds a non-zero partial
     if (lane == 0) s_sig[warp] = sig_part;
     __syncthreads();
   }
