@@ -223,3 +223,41 @@ def test_cfg5_sweep_corners(T, keep):
 def test_cfg4_anyres():
     cfg = inputs.CONFIGS["cfg4_anyres_f16"]
     check_config(cfg, [2])
+
+
+# ------------------------------------------------------------------ launch modes
+def test_image_groups_and_graph_replay_do_not_change_results():
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=6)
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    d = {k: dev(v) for k, v in batch.items()}
+    ws = tcb.workspace(p)
+    outs = []
+    for groups in (1, 2, 4, 8):
+        tcb.tc_set_groups(groups)
+        o = tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)
+        torch.cuda.synchronize()
+        outs.append([host(t) for t in o])
+    # the same call captured into a CUDA graph (its internal fork/join becomes graph edges)
+    tcb.tc_set_groups(4)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)          # warm-up on the side stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    held = tcb._outputs(p, d["O"].device, True) + (
+        torch.zeros(p.batch, p.keep, dtype=torch.int32, device="cuda"),
+        torch.zeros(p.batch, dtype=torch.int32, device="cuda"))
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws, held)
+    for t in held:
+        t.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    outs.append([host(t) for t in held])
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert np.array_equal(a, b)
+    assert not outs[0][4].any()
