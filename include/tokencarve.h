@@ -143,8 +143,11 @@ tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void*
 
 /*
  * tc_carve for callers whose tensors live in HOST memory (pinned for the copies to be
- * asynchronous).  O, A, X, K, V, Xo, Ko, Vo, kept_idx and img_status are host pointers; the
- * inputs are copied to the device, carved, and the results copied back, all on `stream`.
+ * asynchronous).  O, A, X, K, V, Xo, Ko, Vo, kept_idx and img_status are host pointers.  The
+ * batch is cut into up to four chunks: the upload of the next chunk and the download of the
+ * previous one run on two internal copy streams while the current chunk is carved on `stream`;
+ * everything is forked from `stream` and joined back into it, so work enqueued on `stream`
+ * afterwards sees the results in host memory once it runs.
  * `ws` is device memory of at least tc_workspace_bytes_host() bytes (staging + scratch).
  */
 tc_status tc_workspace_bytes_host(const tc_params* p, size_t* bytes);

@@ -352,6 +352,54 @@ tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void*
 }
 
 // ---- host-buffer variant: device staging lives at the front of the workspace ---------------
+constexpr int kHostChunks = 4;
+struct HostStreams {
+  bool ready = false;
+  cudaStream_t cin, cout;
+  cudaEvent_t fork, out, in[kHostChunks], done[kHostChunks];
+};
+static std::mutex g_host_mu;
+static HostStreams g_host[64];
+
+// scratch that covers the whole batch in one call as well as any of the chunks it is cut into
+static size_t host_scratch_bytes(const tc_params* p, const Dims& D) {
+  size_t need = make_plan(D).total;
+  const int nchunk = D.B < kHostChunks ? D.B : kHostChunks;
+  tc_params pc = *p;
+  pc.batch = (D.B + nchunk - 1) / nchunk;
+  Dims Dc;
+  if (make_dims(&pc, &Dc) == TC_OK) {
+    const size_t c = make_plan(Dc).total;
+    if (c > need) need = c;
+  }
+  if (D.B / nchunk >= 1 && D.B / nchunk != pc.batch) {
+    pc.batch = D.B / nchunk;
+    if (make_dims(&pc, &Dc) == TC_OK) {
+      const size_t c = make_plan(Dc).total;
+      if (c > need) need = c;
+    }
+  }
+  return need;
+}
+
+static HostStreams* host_streams() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostStreams& h = g_host[dev];
+  if (!h.ready) {
+    if (cudaStreamCreateWithFlags(&h.cin, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&h.cout, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&h.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&h.out, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    for (int i = 0; i < kHostChunks; ++i) {
+      if (cudaEventCreateWithFlags(&h.in[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&h.done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    h.ready = true;
+  }
+  return &h;
+}
+
 struct HostPlan {
   size_t O, A, X, K, V, Xo, Ko, Vo, kept, status, scratch, total;
 };
@@ -385,7 +433,7 @@ tc_status tc_workspace_bytes_host(const tc_params* p, size_t* bytes) {
   tc_status s = make_dims(p, &D);
   if (s != TC_OK) return s;
   if (bytes == nullptr) return TC_ERR_INVALID_ARG;
-  *bytes = make_host_plan(D, make_plan(D).total).total;
+  *bytes = make_host_plan(D, host_scratch_bytes(p, D)).total;
   return TC_OK;
 }
 
@@ -396,7 +444,7 @@ tc_status tc_carve_host(const tc_params* p, const void* O, const void* A, const 
   Dims D;
   tc_status s = make_dims(p, &D);
   if (s != TC_OK) return s;
-  const size_t scratch = make_plan(D).total;
+  const size_t scratch = host_scratch_bytes(p, D);
   HostPlan h = make_host_plan(D, scratch);
   if (ws == nullptr || misaligned(ws)) return TC_ERR_INVALID_ARG;
   if (ws_bytes < h.total) return TC_ERR_WORKSPACE;
@@ -405,30 +453,67 @@ tc_status tc_carve_host(const tc_params* p, const void* O, const void* A, const 
   if (kv != (V != nullptr) || kv != (Ko != nullptr) || kv != (Vo != nullptr)) return TC_ERR_INVALID_ARG;
   char* w = (char*)ws;
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t B = D.B, e = D.esz;
-  const size_t bO = B * D.N * D.d * e, bA = B * D.H * D.T * (size_t)D.N * e;
-  const size_t bKV = B * D.H * D.N * (size_t)D.dh * e;
-  const size_t bXo = B * D.keep * (size_t)D.d * e, bKVo = B * D.H * D.keep * (size_t)D.dh * e;
+  const size_t e = D.esz;
+  // bytes per image
+  const size_t iO = (size_t)D.N * D.d * e, iA = (size_t)D.H * D.T * D.N * e;
+  const size_t iKV = (size_t)D.H * D.N * D.dh * e;
+  const size_t iXo = (size_t)D.keep * D.d * e, iKVo = (size_t)D.H * D.keep * D.dh * e;
+  // The batch goes through in a few chunks: the upload of chunk c + 1 (copy-in stream) and the
+  // download of chunk c - 1 (copy-out stream) run while chunk c is carved on `stream`.
+  std::lock_guard<std::mutex> lk(g_host_mu);
+  HostStreams* hs = host_streams();
+  const int nchunk = (hs == nullptr) ? 1 : (D.B < kHostChunks ? D.B : kHostChunks);
+  cudaStream_t cin = nchunk > 1 ? hs->cin : st, cout = nchunk > 1 ? hs->cout : st;
   bool ok = true;
-  ok &= cudaMemcpyAsync(w + h.O, O, bO, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(w + h.A, A, bA, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(w + h.X, X, bO, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (kv) {
-    ok &= cudaMemcpyAsync(w + h.K, K, bKV, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(w + h.V, V, bKV, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (nchunk > 1) {
+    ok &= cudaEventRecord(hs->fork, st) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(cin, hs->fork, 0) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(cout, hs->fork, 0) == cudaSuccess;
+  }
+  const int base = D.B / nchunk, extra = D.B % nchunk;
+  int b0 = 0;
+  for (int c = 0; c < nchunk; ++c) {
+    const size_t nb = base + (c < extra ? 1 : 0), o = b0;
+    ok &= cudaMemcpyAsync(w + h.O + o * iO, (const char*)O + o * iO, nb * iO, cudaMemcpyHostToDevice, cin) == cudaSuccess;
+    ok &= cudaMemcpyAsync(w + h.A + o * iA, (const char*)A + o * iA, nb * iA, cudaMemcpyHostToDevice, cin) == cudaSuccess;
+    ok &= cudaMemcpyAsync(w + h.X + o * iO, (const char*)X + o * iO, nb * iO, cudaMemcpyHostToDevice, cin) == cudaSuccess;
+    if (kv) {
+      ok &= cudaMemcpyAsync(w + h.K + o * iKV, (const char*)K + o * iKV, nb * iKV, cudaMemcpyHostToDevice, cin) == cudaSuccess;
+      ok &= cudaMemcpyAsync(w + h.V + o * iKV, (const char*)V + o * iKV, nb * iKV, cudaMemcpyHostToDevice, cin) == cudaSuccess;
+    }
+    if (nchunk > 1) ok &= cudaEventRecord(hs->in[c], cin) == cudaSuccess;
+    b0 += (int)nb;
   }
   if (!ok) return TC_ERR_CUDA;
-  s = tc_carve(p, w + h.O, w + h.A, w + h.X, kv ? w + h.K : nullptr, kv ? w + h.V : nullptr,
-               w + h.Xo, kv ? w + h.Ko : nullptr, kv ? w + h.Vo : nullptr,
-               (int32_t*)(w + h.kept), (int32_t*)(w + h.status), w + h.scratch, scratch, stream);
-  if (s != TC_OK) return s;
-  ok &= cudaMemcpyAsync(Xo, w + h.Xo, bXo, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (kv) {
-    ok &= cudaMemcpyAsync(Ko, w + h.Ko, bKVo, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(Vo, w + h.Vo, bKVo, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  b0 = 0;
+  for (int c = 0; c < nchunk; ++c) {
+    const size_t nb = base + (c < extra ? 1 : 0), o = b0;
+    if (nchunk > 1) ok &= cudaStreamWaitEvent(st, hs->in[c], 0) == cudaSuccess;
+    tc_params pc = *p;
+    pc.batch = (int32_t)nb;
+    s = tc_carve(&pc, w + h.O + o * iO, w + h.A + o * iA, w + h.X + o * iO,
+                 kv ? w + h.K + o * iKV : nullptr, kv ? w + h.V + o * iKV : nullptr,
+                 w + h.Xo + o * iXo, kv ? w + h.Ko + o * iKVo : nullptr,
+                 kv ? w + h.Vo + o * iKVo : nullptr, (int32_t*)(w + h.kept) + o * D.keep,
+                 (int32_t*)(w + h.status) + o, w + h.scratch, scratch, stream);
+    if (s != TC_OK) return s;
+    if (nchunk > 1) {
+      ok &= cudaEventRecord(hs->done[c], st) == cudaSuccess;
+      ok &= cudaStreamWaitEvent(cout, hs->done[c], 0) == cudaSuccess;
+    }
+    ok &= cudaMemcpyAsync((char*)Xo + o * iXo, w + h.Xo + o * iXo, nb * iXo, cudaMemcpyDeviceToHost, cout) == cudaSuccess;
+    if (kv) {
+      ok &= cudaMemcpyAsync((char*)Ko + o * iKVo, w + h.Ko + o * iKVo, nb * iKVo, cudaMemcpyDeviceToHost, cout) == cudaSuccess;
+      ok &= cudaMemcpyAsync((char*)Vo + o * iKVo, w + h.Vo + o * iKVo, nb * iKVo, cudaMemcpyDeviceToHost, cout) == cudaSuccess;
+    }
+    ok &= cudaMemcpyAsync(kept_idx + o * D.keep, (int32_t*)(w + h.kept) + o * D.keep, nb * D.keep * 4, cudaMemcpyDeviceToHost, cout) == cudaSuccess;
+    ok &= cudaMemcpyAsync(img_status + o, (int32_t*)(w + h.status) + o, nb * 4, cudaMemcpyDeviceToHost, cout) == cudaSuccess;
+    b0 += (int)nb;
   }
-  ok &= cudaMemcpyAsync(kept_idx, w + h.kept, B * D.keep * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(img_status, w + h.status, B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (nchunk > 1) {
+    ok &= cudaEventRecord(hs->out, cout) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(st, hs->out, 0) == cudaSuccess;
+  }
   return ok ? TC_OK : TC_ERR_CUDA;
 }
 

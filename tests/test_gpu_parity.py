@@ -261,3 +261,21 @@ def test_image_groups_and_graph_replay_do_not_change_results():
         for a, b in zip(outs[0], o):
             assert np.array_equal(a, b)
     assert not outs[0][4].any()
+
+
+def test_host_entry_point_matches_the_device_one():
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=6)       # chunks of 2, 2, 1, 1 images
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    d = {k: dev(v) for k, v in batch.items()}
+    ref = [host(t) for t in tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"])]
+    hin = {k: torch.from_numpy(v).pin_memory() for k, v in batch.items()}
+    hout = tuple(torch.empty(r.shape, dtype=torch.from_numpy(r).dtype).pin_memory() for r in ref)
+    ws = tcb.workspace(p, host=True)
+    for _ in range(2):                                             # the second call reuses the streams
+        for t in hout:
+            t.zero_()
+        tcb.tc_carve_host(p, hin["O"], hin["A"], hin["X"], hin["K"], hin["V"], hout, ws)
+        torch.cuda.synchronize()
+        for a, b in zip(ref, hout):
+            assert np.array_equal(a, b.numpy())
