@@ -258,36 +258,45 @@ def run_ours(args):
     nbytes = lambda ts: int(sum(t.numel() * t.element_size() for t in ts))
     pk = peaks()
 
-    # roofline of the kernel class that takes the most device time
+    # roofline of the kernel that takes the most device time per step (each profile class is one
+    # kernel; the float32 GEMM is three classes, one per kind of product)
     top = max(prof.items(), key=lambda kv: kv[1][0])
     top_name, (top_ms, top_launches) = top
     per_launch_s = top_ms * 1e-3 / max(top_launches, 1)
     k = p.rank_cap if p.rank_cap else p.n_tokens
+    N = cfg.n_tokens
     alg_bytes_img = algorithmic_bytes_per_image(cfg, P)
-    if top_name == "eig":
+    alu_peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+    # DRAM bytes per image from the ncu capture of the current kernels at B=16
+    # (profiles/ncu_full_kernels_cfg5_B16.md); they grow in proportion to the batch
+    ncu_dram_per_image = {"eig": 1.405e6 / 16, "chol_inv": 1.405e6 / 16, "gram": (75.58e6 + 4.85e6) / 16,
+                          "attn_colsum": (75.51e6 + 1.88e6) / 16, "compact": (75.56e6 + 18.57e6) / 16,
+                          "sketch": (75.51e6 + 2.40e6) / 16}
+    flops_per_launch = {
         # Householder tridiagonalisation 4/3 k^3, accumulation of Q 4/3 k^3, Z = Q Y 2 k^3
-        flops = cfg.batch * (14.0 / 3.0) * k ** 3
-        peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
-        roof = {"kernel": top_name, "bound": "alu", "achieved": flops / per_launch_s / 1e12,
-                "peak": peak, "unit": "TFLOP/s", "traffic": None}
-    elif top_name in ("gram",):
-        flops = cfg.batch * 2.0 * cfg.n_tokens ** 2 * cfg.d_model
+        "eig": cfg.batch * (14.0 / 3.0) * k ** 3,
+        "chol_inv": cfg.batch * (2.0 / 3.0) * k ** 3,
+        "gemm_f32_GQ": cfg.batch * 2.0 * N * N * k,
+        "gemm_f32_YtY": cfg.batch * 2.0 * N * k * k,
+        "gemm_f32_YRinv": cfg.batch * 2.0 * N * k * k,
+    }
+    if top_name in flops_per_launch:
+        roof = {"kernel": top_name, "bound": "alu", "achieved": flops_per_launch[top_name] / per_launch_s / 1e12,
+                "peak": alu_peak, "unit": "TFLOP/s"}
+    elif top_name == "gram":
+        flops = cfg.batch * 2.0 * N ** 2 * cfg.d_model
         roof = {"kernel": top_name, "bound": "tensor", "achieved": flops / per_launch_s / 1e12,
-                "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "traffic": None}
-    elif top_name == "gemm_f32":
-        N = cfg.n_tokens
-        # two products with G (2 N^2 k each) and ten N x k x k products per carve
-        flops = cfg.batch * (2 * 2.0 * N * N * k + 10 * 2.0 * N * k * k) / max(top_launches / args.steps, 1)
-        peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
-        roof = {"kernel": top_name, "bound": "alu", "achieved": flops / per_launch_s / 1e12,
-                "peak": peak, "unit": "TFLOP/s", "traffic": None}
+                "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s"}
     else:
         e = 2
-        per = {"attn_colsum": cfg.n_heads * cfg.n_query * cfg.n_tokens * e,
+        per = {"attn_colsum": cfg.n_heads * cfg.n_query * N * e,
                "compact": (P + cfg.keep) * (cfg.d_model + 2 * cfg.n_heads * cfg.head_dim) * e,
-               "sketch": cfg.n_tokens * cfg.d_model * e}.get(top_name, alg_bytes_img)
+               "sketch": N * cfg.d_model * e}.get(top_name, alg_bytes_img)
         roof = {"kernel": top_name, "bound": "hbm", "achieved": cfg.batch * per / per_launch_s / 1e9,
-                "peak": pk["hbm_gbs"], "unit": "GB/s", "traffic": None}
+                "peak": pk["hbm_gbs"], "unit": "GB/s"}
+    same_shape = (cfg.n_tokens, cfg.d_model, cfg.n_query, cfg.keep, k) == (576, 4096, 128, 128, 144)
+    roof["traffic"] = (ncu_dram_per_image[top_name] * cfg.batch
+                       if same_shape and top_name in ncu_dram_per_image else None)
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = pk["source"]
     # the whole path against the slower of its HBM bytes and its Gram flops

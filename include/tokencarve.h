@@ -208,7 +208,7 @@ tc_status tc_set_groups(int32_t groups);
  * milliseconds and the number of launches, in the HOST arrays ms[n], launches[n]
  * (n >= TC_N_KERNEL_CLASSES).  Not thread-safe against concurrent carve calls.
  */
-#define TC_N_KERNEL_CLASSES 13
+#define TC_N_KERNEL_CLASSES 15
 int32_t tc_profile_begin(void);
 int32_t tc_profile_end(double* ms, int64_t* launches, int32_t n);
 const char* tc_kernel_class_name(int32_t cls);

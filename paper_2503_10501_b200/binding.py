@@ -290,7 +290,7 @@ def tc_launch_count() -> int:
     return lib().tc_launch_count()
 
 
-N_KERNEL_CLASSES = 13
+N_KERNEL_CLASSES = 15
 
 
 def tc_profile_begin() -> None:

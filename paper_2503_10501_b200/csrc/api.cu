@@ -578,9 +578,9 @@ int32_t tc_profile_end(double* ms, int64_t* launches, int32_t n) {
 }
 
 const char* tc_kernel_class_name(int32_t cls) {
-  static const char* names[] = {"fill", "attn_colsum", "gram", "sketch", "gemm_f32", "chol_inv",
+  static const char* names[] = {"fill", "attn_colsum", "gram", "sketch", "gemm_f32_YRinv", "chol_inv",
                                 "eig", "ics", "combine", "prune", "match", "merge_select",
-                                "compact"};
+                                "compact", "gemm_f32_GQ", "gemm_f32_YtY"};
   return (cls >= 0 && cls < (int)tc::KC_COUNT) ? names[cls] : "?";
 }
 

@@ -1449,7 +1449,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   }
   // one Cholesky-QR pass: dst = src R^{-1},  R^T R = src^T src (+ shift)
   auto cholqr_pass = [&](const float* src, float* dst, float shift_rel) {
-    gemm<float, float, true, false>(src, src, Sm, k, k, N, k, k, k, sY, sY, sK, B, st, KC_GEMM, GEMM_SYM);
+    gemm<float, float, true, false>(src, src, Sm, k, k, N, k, k, k, sY, sY, sK, B, st, KC_GEMM_TN, GEMM_SYM);
     launch_chol_inv(Sm, Rinv, W, k, B, shift_rel, img_status, st);
     gemm<float, float, false, true>(src, Rinv, dst, N, k, k, k, k, k, sY, sK, sY, B, st, KC_GEMM, GEMM_B_UPPER);
   };
@@ -1459,13 +1459,13 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   cholqr_pass(Y0, Y1, kShift);
   { float* t = Y0; Y0 = Y1; Y1 = t; }  // Q0 in Y0
   // 3. one multiplication by G sharpens the subspace:  Y1 = G Q0, then orthonormalise
-  gemm<float, float, false, false>(G, Y0, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);
+  gemm<float, float, false, false>(G, Y0, Y1, N, k, N, N, k, k, sG, sY, sY, B, st, KC_GEMM_GQ);
   cholqr_pass(Y1, Y2, kShift);
   cholqr_pass(Y2, Y1, kShift);
   cholqr_pass(Y1, Y2, 0.f);  // Q1 in Y2
   // 4. Rayleigh-Ritz:  H = Q1^T G Q1
-  gemm<float, float, false, false>(G, Y2, Y1, N, k, N, N, k, k, sG, sY, sY, B, st);   // T = G Q1
-  gemm<float, float, true, false>(Y2, Y1, Hm, k, k, N, k, k, k, sY, sY, sK, B, st);   // H = Q1^T T
+  gemm<float, float, false, false>(G, Y2, Y1, N, k, N, N, k, k, sG, sY, sY, B, st, KC_GEMM_GQ);   // T = G Q1
+  gemm<float, float, true, false>(Y2, Y1, Hm, k, k, N, k, k, k, sY, sY, sK, B, st, KC_GEMM_TN);   // H = Q1^T T
   // scratch of the solver: W, Sm, Rinv, Hm (k x k each) and the first k x k of each image's Y1 panel
   launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, Sm, Rinv, Hm, Y1, sY, img_status, st);
   // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]

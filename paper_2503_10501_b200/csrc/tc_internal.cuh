@@ -50,7 +50,7 @@ void note_launch(int n = 1);
 // Kernel classes for the optional event profile (tc_profile_begin / tc_profile_end).
 enum KernelClass {
   KC_FILL = 0, KC_ATTN, KC_GRAM, KC_SKETCH, KC_GEMM, KC_CHOL, KC_JACOBI, KC_ICS, KC_COMBINE,
-  KC_PRUNE, KC_MATCH, KC_MSEL, KC_COMPACT, KC_COUNT
+  KC_PRUNE, KC_MATCH, KC_MSEL, KC_COMPACT, KC_GEMM_GQ, KC_GEMM_TN, KC_COUNT
 };
 // While a profile is open, brackets the launches made in its lifetime with two CUDA events
 // on `st`; otherwise does nothing.
