@@ -1060,28 +1060,10 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       return cnt;
     };
     const float lon = lo * itn, hin = hi * itn;
-    if (n <= 160) {
-      // three lanes per eigenvalue, ten eigenvalues per warp: each round evaluates the count at
-      // the three quarter points of the bracket, which shrinks it four-fold
-      const int t = warp * 10 + lane / 3, jj = lane % 3;
-      const bool on = (lane < 30) && (t < n);
-      const int base = lane - jj;
-      float a = lon, bhi = hin;
-      for (int it = 0; it < 24; ++it) {
-        const float step = 0.25f * (bhi - a);
-        const float x = a + step * (float)(jj + 1);
-        const int cnt = on ? sturm(x) : 0;
-        const int c0 = __shfl_sync(0xffffffffu, cnt, base & 31);
-        const int c1 = __shfl_sync(0xffffffffu, cnt, (base + 1) & 31);
-        const int c2 = __shfl_sync(0xffffffffu, cnt, (base + 2) & 31);
-        const float x0 = a + step, x1 = a + 2.0f * step, x2 = a + 3.0f * step;
-        if (c0 > t) bhi = x0;
-        else if (c1 > t) { a = x0; bhi = x1; }
-        else if (c2 > t) { a = x1; bhi = x2; }
-        else a = x2;
-      }
-      if (on && jj == 0) lam[t] = 0.5f * (a + bhi) * tn;
-    } else if (tid < n) {
+    if (tid < n) {
+      // eigenvalue number tid (0 = smallest): plain bisection, one thread per eigenvalue (the
+      // counts are bound by instruction issue, so evaluating several points per round on
+      // neighbouring lanes costs more than the rounds it saves)
       float a = lon, bhi = hin;
       for (int it = 0; it < 48; ++it) {
         const float x = 0.5f * (a + bhi);
