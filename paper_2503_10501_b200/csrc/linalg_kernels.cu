@@ -826,7 +826,8 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   float* vv = ev + n;                  // [n] Householder vector of the current step
   float* pv = vv + n;                  // [n] work vector
   float* beta = pv + n;                // [n] reflector scales
-  float2* cs = reinterpret_cast<float2*>(beta + n);  // [2][n] rotation batches
+  float2* cs = reinterpret_cast<float2*>(beta + n);  // [4 n floats] partial sums of the reduction
+  float* qf = reinterpret_cast<float*>(cs) + 4 * n;    // [16 n] reflector block and partial products
   __shared__ float s_red[16];
   __shared__ int s_fail;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -945,40 +946,100 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   __syncthreads();
 
   // ---------------- Q = H_0 H_1 ... H_{n-3}, accumulated backwards, in place ----------------
-  // Reflector j sits in A[j+1.., j]; column c >= j+2 of A, rows >= j+2, already holds the
-  // product of the later reflectors; row j+1 of those columns counts as zero.
+  // Reflector j sits in A[j+1.., j].  Reflectors are applied four at a time in the compact WY
+  // form  H_{j0} ... H_{j1} = I - V T V^T  (T upper triangular), so a block costs three barriers
+  // and two passes over the rows instead of two barriers and two passes per reflector.
+  // Before a block, columns c >= j1+2 of A (rows >= j1+2) hold the product of the later
+  // reflectors; everything else of Q is still the identity, which the block first writes out.
   {
-    const int cw = (n + 31) / 32;            // warps needed to cover the columns
-    const int groups = max(1, 16 / cw);      // row ranges worked on side by side
-    const int g = warp / cw;                 // this thread's row range
-    const int cl = (warp % cw) * 32 + lane;  // this thread's column, relative to j+2
-    float* tbuf = reinterpret_cast<float*>(cs);  // [<=4][n] partial dots (cs is free here)
-    const int gmax = min(groups, 4);
-    for (int j = n - 3; j >= 0; --j) {
-      const float bj = beta[j];
-      const int m = n - j - 1;       // rows j+1 .. n-1
-      const int ncol = m - 1;        // columns j+2 .. n-1
-      const int rows = m - 1;        // rows j+2 .. n-1 take part in the dots
-      const int per = (rows + gmax - 1) / gmax;
-      const int r_lo = j + 2 + g * per, r_hi = min(n, r_lo + per);
-      const bool active = (g < gmax) && (cl < ncol);
-      const int c = j + 2 + cl;
-      float tsum = 0.f;
-      if (active && bj != 0.f)
-        for (int r = r_lo; r < r_hi; ++r) tsum = fmaf(A[r * ld + j], A[r * ld + c], tsum);
-      if (g < gmax && cl < n) tbuf[g * n + cl] = tsum;
-      __syncthreads();
-      if (active) {
-        float t = 0.f;
-        for (int q = 0; q < gmax; ++q) t += tbuf[q * n + cl];
-        const float bt = bj * t;
-        for (int r = r_lo; r < r_hi; ++r) A[r * ld + c] = fmaf(-bt, A[r * ld + j], A[r * ld + c]);
-        if (g == 0) A[(j + 1) * ld + c] = -bt * A[(j + 1) * ld + j];
+    constexpr int NBQ = 4;
+    float* Vb = qf;              // [NBQ][n]  Vb[i][r] = entry r of reflector j0+i (0 above its support)
+    float* Wp = qf + NBQ * n;    // [3][NBQ][n] partial products V^T Q per row range
+    __shared__ float s_vv[NBQ][NBQ];  // v_a . v_b for a < b
+    __shared__ float s_T[NBQ][NBQ];
+    for (int j1 = n - 3; j1 >= 0; j1 -= NBQ) {
+      const int j0 = max(0, j1 - NBQ + 1), nbk = j1 - j0 + 1;
+      // (1) copy the block's reflectors out of the columns that are about to be overwritten
+      for (int idx = tid; idx < nbk * n; idx += 512) {
+        const int i = idx / n, r = idx - i * n, jj = j0 + i;
+        Vb[i * n + r] = (r >= jj + 1) ? A[r * ld + jj] : 0.f;
       }
-      // column j+1: H_j e_{j+1} (touches no column the threads above work on)
-      const float vj1 = A[(j + 1) * ld + j];
-      for (int r = j + 2 + tid; r < n; r += 512) A[r * ld + j + 1] = -bj * A[r * ld + j] * vj1;
-      if (tid == 0) A[(j + 1) * ld + j + 1] = 1.0f - bj * vj1 * vj1;
+      __syncthreads();
+      // (2) identity columns j0+1 .. j1+1, zero rows j0+1 .. j1+1 right of them; v_a . v_b
+      for (int idx = tid; idx < (n - j0 - 1) * nbk; idx += 512) {
+        const int r = j0 + 1 + idx / nbk, c = j0 + 1 + idx % nbk;
+        A[r * ld + c] = (r == c) ? 1.f : 0.f;
+      }
+      for (int idx = tid; idx < nbk * (n - j1 - 2); idx += 512) {
+        const int r = j0 + 1 + idx / (n - j1 - 2), c = j1 + 2 + idx % (n - j1 - 2);
+        A[r * ld + c] = 0.f;
+      }
+      if (warp < NBQ * NBQ) {
+        const int a2 = warp / NBQ, b2 = warp % NBQ;
+        if (a2 < b2 && b2 < nbk) {
+          float d2 = 0.f;
+          for (int r = lane; r < n; r += 32) d2 = fmaf(Vb[a2 * n + r], Vb[b2 * n + r], d2);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) d2 += __shfl_xor_sync(0xffffffffu, d2, o);
+          if (lane == 0) s_vv[a2][b2] = d2;
+        }
+      }
+      __syncthreads();
+      if (tid == 0) {
+        // T_ii = beta_i ;  T[0:i, i] = -beta_i T[0:i, 0:i] (V[:, 0:i]^T v_i)
+        for (int i = 0; i < nbk; ++i) {
+          const float bi = beta[j0 + i];
+          for (int a2 = 0; a2 < i; ++a2) {
+            float acc = 0.f;
+            for (int l = a2; l < i; ++l) acc = fmaf(s_T[a2][l], s_vv[l][i], acc);
+            s_T[a2][i] = -bi * acc;
+          }
+          s_T[i][i] = bi;
+        }
+      }
+      // (3) W = V^T Q on the columns c >= j0+1, rows split into up to three ranges
+      const int ncols = n - j0 - 1;
+      const int cw = (ncols + 31) >> 5;
+      const int G = min(3, 16 / cw);
+      const int g = warp / cw, c = j0 + 1 + (warp - g * cw) * 32 + lane;
+      const bool on = (g < G) && (c < n);
+      const int per = (ncols + G - 1) / G;
+      const int r_lo = j0 + 1 + g * per, r_hi = min(n, r_lo + per);
+      if (on) {
+        float acc[NBQ] = {0.f, 0.f, 0.f, 0.f};
+        for (int r = r_lo; r < r_hi; ++r) {
+          const float qv = A[r * ld + c];
+#pragma unroll
+          for (int i = 0; i < NBQ; ++i) acc[i] = fmaf(Vb[i * n + r], qv, acc[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < NBQ; ++i) Wp[(g * NBQ + i) * n + c] = acc[i];
+      }
+      __syncthreads();
+      // (4) T W, (5) Q -= V (T W)
+      if (on) {
+        float w[NBQ], tw[NBQ];
+#pragma unroll
+        for (int i = 0; i < NBQ; ++i) {
+          float t = 0.f;
+          for (int q = 0; q < G; ++q) t += Wp[(q * NBQ + i) * n + c];
+          w[i] = (i < nbk) ? t : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < NBQ; ++i) {
+          float t = 0.f;
+#pragma unroll
+          for (int l = 0; l < NBQ; ++l)
+            if (l >= i && l < nbk && i < nbk) t = fmaf(s_T[i][l], w[l], t);
+          tw[i] = t;
+        }
+        for (int r = r_lo; r < r_hi; ++r) {
+          float qv = A[r * ld + c];
+#pragma unroll
+          for (int i = 0; i < NBQ; ++i) qv = fmaf(-Vb[i * n + r], tw[i], qv);
+          A[r * ld + c] = qv;
+        }
+      }
       __syncthreads();
     }
     // first row and column of Q are e_0
@@ -1259,7 +1320,7 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
                           float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_JACOBI, st);
   {
-    const size_t tri = ((size_t)n * (n | 1) + 9 * (size_t)n) * sizeof(float);
+    const size_t tri = ((size_t)n * (n | 1) + 25 * (size_t)n) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       cudaFuncSetAttribute((const void*)tridiag_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
       { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status); note_launch(); }
