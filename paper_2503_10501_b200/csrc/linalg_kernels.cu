@@ -1088,7 +1088,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     // Sturm count in product form on T / |T| (no division on the serial chain):
     //   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1};
     // the number of sign changes along the sequence is the number of eigenvalues below x.
-    // Both running values are rescaled together whenever they leave [1e-10, 1e10].
+    // Both running values are rescaled together whenever they leave [1e-8, 1e8].
     float* dn = beta;  // beta is free once Q has been formed
     const float itn = 1.0f / fmaxf(tn, 1e-30f);
     for (int i = tid; i < n; i += 512) {
@@ -1097,26 +1097,36 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     }
     __syncthreads();
     auto sturm = [&](float x) {
+      // two steps per trip: the diagonal and off-diagonal entries of both are loaded up front,
+      // and the pair is re-centred once per trip (entries can be as small as rounding noise,
+      // 1e-7 of the largest, so it can shrink by 1e-14 in a trip: the thresholds leave room)
       float p0 = 1.f, p1 = dn[0] - x;
-      int cnt = p1 < 0.f;
       bool neg = p1 < 0.f;
-      for (int i = 1; i < n; ++i) {
-        const float p2 = fmaf(dn[i] - x, p1, -e2[i - 1] * p0);
-        const bool neg2 = (p2 < 0.f) || (p2 == 0.f && !neg);  // an exact zero counts as a change
-        cnt += (neg2 != neg);
-        neg = neg2;
-        p0 = p1;
-        p1 = p2;
-        // entries of the scaled matrix can be as small as rounding noise (1e-7 and below), so
-        // the pair can shrink by that much in a single step: re-centre it every step
+      int cnt = neg;
+      int i = 1;
+      for (; i + 1 < n; i += 2) {
+        const float da = dn[i] - x, db = dn[i + 1] - x, ea = e2[i - 1], eb = e2[i];
+        const float pa = fmaf(da, p1, -ea * p0);
+        const float pb = fmaf(db, pa, -eb * p1);
+        const bool na = (pa < 0.f) || (pa == 0.f && !neg);  // an exact zero counts as a change
+        const bool nb2 = (pb < 0.f) || (pb == 0.f && !na);
+        cnt += (na != neg) + (nb2 != na);
+        neg = nb2;
+        p0 = pa;
+        p1 = pb;
         const float sc = fmaxf(fabsf(p0), fabsf(p1));
-        if (sc < 1e-10f) {
-          p0 *= 1e20f;
-          p1 *= 1e20f;
-        } else if (sc > 1e10f) {
-          p0 *= 1e-20f;
-          p1 *= 1e-20f;
+        if (sc < 1e-8f) {
+          p0 *= 1e16f;
+          p1 *= 1e16f;
+        } else if (sc > 1e8f) {
+          p0 *= 1e-16f;
+          p1 *= 1e-16f;
         }
+      }
+      if (i < n) {
+        const float pa = fmaf(dn[i] - x, p1, -e2[i - 1] * p0);
+        const bool na = (pa < 0.f) || (pa == 0.f && !neg);
+        cnt += (na != neg);
       }
       return cnt;
     };
