@@ -329,10 +329,116 @@ def run_ours(args):
                 "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
                 "path_roofline": path,
                 "kernel_ms_per_step": {k_: round(v[0] / args.steps, 4) for k_, v in prof.items() if v[1]},
+                "kernel_roofline": kernel_fractions(cfg, P, k, prof, args.steps, pk),
                 "cpu_baseline": cpu}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- sweep
+def kernel_fractions(cfg, P, k, prof, steps, pk):
+    """Roofline fraction of every profiled kernel class: algorithmic bytes (or flops) per launch
+    over its event-timed duration, against the HBM, tensor or FP32-ALU peak that bounds it."""
+    e = 2 if cfg.dtype == "f16" else 4
+    B, N, d, H, dh, T = cfg.batch, cfg.n_tokens, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.n_query
+    alu_peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6  # flop/s
+    work = {  # class -> (amount per launch, peak per second, bound)
+        "attn_colsum": (B * H * T * N * e, pk["hbm_gbs"] * 1e9, "hbm"),
+        "sketch": (B * N * d * e, pk["hbm_gbs"] * 1e9, "hbm"),
+        "compact": (B * (P + cfg.keep) * (d + 2 * H * dh) * e, pk["hbm_gbs"] * 1e9, "hbm"),
+        "gram": (B * 2.0 * N * N * d, pk["bf16_tflops_sustained"] * 1e12, "tensor"),
+        "gemm_f32_GQ": (B * 2.0 * N * N * k, alu_peak, "alu"),
+        "gemm_f32_YtY": (B * 2.0 * N * k * k, alu_peak, "alu"),
+        "gemm_f32_YRinv": (B * 2.0 * N * k * k, alu_peak, "alu"),
+        "chol_inv": (B * (2.0 / 3.0) * k ** 3, alu_peak, "alu"),
+        "eig": (B * (14.0 / 3.0) * k ** 3, alu_peak, "alu"),
+    }
+    out = {}
+    for name, (ms_total, launches) in prof.items():
+        if not launches or name not in work:
+            continue
+        amount, peak, bound = work[name]
+        # a class launched several times per step (the GEMM products, chol_inv) does `amount`
+        # per launch; its time per launch is the class total over its launches
+        per_launch_s = ms_total * 1e-3 / launches
+        out[name] = {"bound": bound, "frac": round(amount / per_launch_s / peak, 4),
+                     "ms_per_step": round(ms_total / steps, 4)}
+    return out
+
+
+def run_sweep(args):
+    """One JSON line per point of the throughput sweep: text tokens T in {32,128,512} x keep in
+    {64,128,192,288} at the bench batch; images/s and the roofline fraction of every kernel."""
+    import torch
+    from paper_2503_10501_b200 import binding as tcb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the carve path")
+    torch.cuda.set_device(0)
+    tcb.lib()
+    groups = args.groups if args.groups else 4
+    tcb.tc_set_groups(groups)
+    pk = peaks()
+    base = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=args.batch)
+    if args.rank_cap:
+        base = base.with_(rank_cap=args.rank_cap)
+    dev = {k: torch.from_numpy(v).cuda() for k, v in inputs.make_batch(base, want="OXKV").items()}
+    for T in (32, 128, 512):
+        cfgT = base.with_(n_query=T)
+        A = torch.from_numpy(inputs.make_batch(cfgT, want="A")["A"]).cuda()
+        for keep in (64, 128, 192, 288):
+            cfg = cfgT.with_(keep=keep)
+            p = tcb.Params(batch=cfg.batch, n_tokens=cfg.n_tokens, d_model=cfg.d_model,
+                           n_heads=cfg.n_heads, head_dim=cfg.head_dim, n_query=T, keep=keep,
+                           rho=cfg.rho, lam=cfg.lam, rank_tol=cfg.rank_tol, dtype=cfg.dtype,
+                           rank_cap=cfg.rank_cap)
+            M, P, nA, nB = tcb.tc_counts(p)
+            dt = p.torch_dtype
+            mk = lambda *s, dtype=dt: torch.empty(*s, dtype=dtype, device="cuda")
+            out = (mk(p.batch, keep, p.d_model), mk(p.batch, p.n_heads, keep, p.head_dim),
+                   mk(p.batch, p.n_heads, keep, p.head_dim), mk(p.batch, keep, dtype=torch.int32),
+                   mk(p.batch, dtype=torch.int32))
+            ws = tcb.workspace(p)
+
+            def step():
+                tcb.tc_carve(p, dev["O"], A, dev["X"], dev["K"], dev["V"], ws, out)
+
+            for _ in range(args.warmup):
+                step()
+            torch.cuda.synchronize()
+            status = out[4].cpu().numpy()
+            if status.any():
+                raise SystemExit(f"T={T} keep={keep}: per-image status {status.tolist()}")
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                step()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            tcb.tc_set_groups(1)
+            step()
+            tcb.tc_profile_begin()
+            for _ in range(args.steps):
+                step()
+            prof = tcb.tc_profile_end()
+            tcb.tc_set_groups(groups)
+            k = p.rank_cap if p.rank_cap else p.n_tokens
+            alg = algorithmic_bytes_per_image(cfg, P)
+            t_roof = max(alg / (pk["hbm_gbs"] * 1e9),
+                         2.0 * cfg.n_tokens ** 2 * cfg.d_model / (pk["bf16_tflops_sustained"] * 1e12))
+            us_img = ms * 1e3 / (cfg.batch * args.steps)
+            print(json.dumps({
+                "sweep_point": {"T": T, "keep": keep, "P": P, "M": M, "batch": cfg.batch},
+                "images_per_s": round(cfg.batch * args.steps / (ms * 1e-3), 1),
+                "us_per_image": round(us_img, 3), "ms_per_step": round(ms / args.steps, 4),
+                "path_roofline_frac": round(t_roof * 1e6 / us_img, 4),
+                "algorithmic_bytes_per_image": alg, "peak_source": pk["source"],
+                "kernels": kernel_fractions(cfg, P, k, prof, args.steps, pk)}), flush=True)
+            del out, ws
+        del A
+        torch.cuda.empty_cache()
 
 
 def main():
@@ -350,8 +456,12 @@ def main():
     ap.add_argument("--groups", type=int, default=0, help="concurrent image groups (0 = library default)")
     ap.add_argument("--cpu-images", type=int, default=12,
                     help="images the CPU oracle is timed on (0 = skip)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="one line per point of the T x keep sweep instead of the bench line")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
