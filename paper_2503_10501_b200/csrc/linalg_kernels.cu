@@ -811,6 +811,11 @@ __global__ void __launch_bounds__(512) jacobi_kernel(const float* __restrict__ H
 //   scratch u0, u1, u2, yv, ml: [n][n] float each, per image
 // One block (16 warps) per image.
 // ==========================================================================================
+// Barrier among `count` threads (a multiple of 32) of the block, on hardware barrier `id` (1..15).
+__device__ __forceinline__ void bar_named(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
 __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ ZTg,
                                                          float* __restrict__ theta, int n, float rank_tol,
@@ -828,6 +833,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   float* beta = pv + n;                // [n] reflector scales
   float2* cs = reinterpret_cast<float2*>(beta + n);  // [4 n floats] partial sums of the reduction
   float* qf = reinterpret_cast<float*>(cs) + 4 * n;    // [16 n] reflector block and partial products
+  float* dn = qf + 16 * n;             // [n] diagonal of T / |T| for the Sturm counts
   __shared__ float s_red[16];
   __shared__ int s_fail;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -945,6 +951,14 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   }
   __syncthreads();
 
+  // From here the block works as two teams until Z = Q Y needs both results: the first
+  // ceil(n / 32) warps find the eigenpairs of T (one thread per eigenvalue; they only read the
+  // diagonals of T), the other warps accumulate Q.  Each team synchronises on its own barrier.
+  const int nbw = (n + 31) >> 5;           // warps of the eigenvalue team
+  const int ET = nbw * 32;                 // its threads
+  const int NQW = 16 - nbw, QT = NQW * 32; // warps and threads of the Q team
+  const int qt = tid - ET, qw = warp - nbw;
+  if (warp >= nbw) {
   // ---------------- Q = H_0 H_1 ... H_{n-3}, accumulated backwards, in place ----------------
   // Reflector j sits in A[j+1.., j].  Reflectors are applied four at a time in the compact WY
   // form  H_{j0} ... H_{j1} = I - V T V^T  (T upper triangular), so a block costs three barriers
@@ -960,23 +974,25 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     for (int j1 = n - 3; j1 >= 0; j1 -= NBQ) {
       const int j0 = max(0, j1 - NBQ + 1), nbk = j1 - j0 + 1;
       // (1) copy the block's reflectors out of the columns that are about to be overwritten
-      for (int idx = tid; idx < nbk * n; idx += 512) {
+      for (int idx = qt; idx < nbk * n; idx += QT) {
         const int i = idx / n, r = idx - i * n, jj = j0 + i;
         Vb[i * n + r] = (r >= jj + 1) ? A[r * ld + jj] : 0.f;
       }
-      __syncthreads();
+      bar_named(1, QT);
       // (2) identity columns j0+1 .. j1+1, zero rows j0+1 .. j1+1 right of them; v_a . v_b
-      for (int idx = tid; idx < (n - j0 - 1) * nbk; idx += 512) {
+      for (int idx = qt; idx < (n - j0 - 1) * nbk; idx += QT) {
         const int r = j0 + 1 + idx / nbk, c = j0 + 1 + idx % nbk;
         A[r * ld + c] = (r == c) ? 1.f : 0.f;
       }
-      for (int idx = tid; idx < nbk * (n - j1 - 2); idx += 512) {
+      for (int idx = qt; idx < nbk * (n - j1 - 2); idx += QT) {
         const int r = j0 + 1 + idx / (n - j1 - 2), c = j1 + 2 + idx % (n - j1 - 2);
         A[r * ld + c] = 0.f;
       }
-      if (warp < NBQ * NBQ) {
-        const int a2 = warp / NBQ, b2 = warp % NBQ;
-        if (a2 < b2 && b2 < nbk) {
+      if (qw < 6) {
+        // the six pairs a < b of a block of four, one warp each
+        const int a2 = (qw < 3) ? 0 : (qw < 5 ? 1 : 2);
+        const int b2 = (qw < 3) ? qw + 1 : (qw < 5 ? qw - 1 : 3);
+        if (b2 < nbk) {
           float d2 = 0.f;
           for (int r = lane; r < n; r += 32) d2 = fmaf(Vb[a2 * n + r], Vb[b2 * n + r], d2);
 #pragma unroll
@@ -984,8 +1000,8 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
           if (lane == 0) s_vv[a2][b2] = d2;
         }
       }
-      __syncthreads();
-      if (tid == 0) {
+      bar_named(1, QT);
+      if (qt == 0) {
         // T_ii = beta_i ;  T[0:i, i] = -beta_i T[0:i, 0:i] (V[:, 0:i]^T v_i)
         for (int i = 0; i < nbk; ++i) {
           const float bi = beta[j0 + i];
@@ -1000,8 +1016,8 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       // (3) W = V^T Q on the columns c >= j0+1, rows split into up to three ranges
       const int ncols = n - j0 - 1;
       const int cw = (ncols + 31) >> 5;
-      const int G = min(3, 16 / cw);
-      const int g = warp / cw, c = j0 + 1 + (warp - g * cw) * 32 + lane;
+      const int G = min(3, NQW / cw);
+      const int g = qw / cw, c = j0 + 1 + (qw - g * cw) * 32 + lane;
       const bool on = (g < G) && (c < n);
       const int per = (ncols + G - 1) / G;
       const int r_lo = j0 + 1 + g * per, r_hi = min(n, r_lo + per);
@@ -1015,7 +1031,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
 #pragma unroll
         for (int i = 0; i < NBQ; ++i) Wp[(g * NBQ + i) * n + c] = acc[i];
       }
-      __syncthreads();
+      bar_named(1, QT);
       // (4) T W, (5) Q -= V (T W)
       if (on) {
         float w[NBQ], tw[NBQ];
@@ -1040,17 +1056,17 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
           A[r * ld + c] = qv;
         }
       }
-      __syncthreads();
+      bar_named(1, QT);
     }
     // first row and column of Q are e_0
-    for (int i = tid; i < n; i += 512) {
+    for (int i = qt; i < n; i += QT) {
       A[i * ld] = (i == 0) ? 1.f : 0.f;
       A[i] = (i == 0) ? 1.f : 0.f;
     }
-    if (n == 2 && tid == 0) {  // no reflector at all: Q = I
+    if (n == 2 && qt == 0) {  // no reflector at all: Q = I
       A[ld + 1] = 1.f;
     }
-    __syncthreads();
+  }
   }
 
   // ---------------- eigenvalues of T by bisection ----------------
@@ -1058,9 +1074,9 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   float* e2 = vv;
   float* lam = pv;
   float tnorm = 0.f;
-  {
+  if (warp < nbw) {
     float lo = 3.0e38f, hi = -3.0e38f;
-    for (int i = tid; i < n; i += 512) {
+    for (int i = tid; i < n; i += ET) {
       const float el = (i > 0) ? fabsf(ev[i - 1]) : 0.f, er = (i + 1 < n) ? fabsf(ev[i]) : 0.f;
       lo = fminf(lo, dv[i] - el - er);
       hi = fmaxf(hi, dv[i] + el + er);
@@ -1075,10 +1091,10 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       s_red[warp] = lo;
       reinterpret_cast<float*>(cs)[warp] = hi;
     }
-    __syncthreads();
+    bar_named(2, ET);
     lo = s_red[0];
     hi = reinterpret_cast<float*>(cs)[0];
-    for (int w = 1; w < 16; ++w) {
+    for (int w = 1; w < nbw; ++w) {
       lo = fminf(lo, s_red[w]);
       hi = fmaxf(hi, reinterpret_cast<float*>(cs)[w]);
     }
@@ -1089,13 +1105,12 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     //   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1};
     // the number of sign changes along the sequence is the number of eigenvalues below x.
     // Both running values are rescaled together whenever they leave [1e-8, 1e8].
-    float* dn = beta;  // beta is free once Q has been formed
     const float itn = 1.0f / fmaxf(tn, 1e-30f);
-    for (int i = tid; i < n; i += 512) {
+    for (int i = tid; i < n; i += ET) {
       dn[i] = dv[i] * itn;
       e2[i] = e2[i] * itn * itn;
     }
-    __syncthreads();
+    bar_named(2, ET);
     auto sturm = [&](float x) {
       // two steps per trip: the diagonal and off-diagonal entries of both are loaded up front,
       // and the pair is re-centred once per trip (entries can be as small as rounding noise,
@@ -1144,8 +1159,8 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       lam[tid] = 0.5f * (a + bhi) * tn;
     }
     tnorm = tn;
+    bar_named(2, ET);
   }
-  __syncthreads();
 
   // ---------------- eigenvectors of T by inverse iteration ----------------
   const float keep_floor = 0.25f * rank_tol * rank_tol * tnorm;
@@ -1330,7 +1345,7 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
                           float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_JACOBI, st);
   {
-    const size_t tri = ((size_t)n * (n | 1) + 25 * (size_t)n) * sizeof(float);
+    const size_t tri = ((size_t)n * (n | 1) + 26 * (size_t)n) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       cudaFuncSetAttribute((const void*)tridiag_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
       { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status); note_launch(); }
