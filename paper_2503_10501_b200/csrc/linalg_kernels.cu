@@ -823,17 +823,19 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ u2g, float* yg, float* __restrict__ mlg,
                                                          size_t ml_stride,
                                                          int32_t* __restrict__ status) {
-  extern __shared__ float sm[];
+  extern __shared__ __align__(16) float sm[];
   const int ld = n | 1;
-  float* A = sm;                       // [n][ld]
-  float* dv = A + (size_t)n * ld;      // [n] diagonal
-  float* ev = dv + n;                  // [n] sub-diagonal (ev[i] couples i and i+1)
-  float* vv = ev + n;                  // [n] Householder vector of the current step
-  float* pv = vv + n;                  // [n] work vector
-  float* beta = pv + n;                // [n] reflector scales
-  float2* cs = reinterpret_cast<float2*>(beta + n);  // [4 n floats] partial sums of the reduction
-  float* qf = reinterpret_cast<float*>(cs) + 4 * n;    // [16 n] reflector block and partial products
-  float* dn = qf + 16 * n;             // [n] diagonal of T / |T| for the Sturm counts
+  const int n4 = (n + 3) & ~3;         // the vectors start on 16-byte boundaries
+  float* dv = sm;                      // [n] diagonal
+  float* ev = dv + n4;                 // [n] sub-diagonal (ev[i] couples i and i+1)
+  float* vv = ev + n4;                 // [n] Householder vector of the current step
+  float* vv2 = vv + n4;                // [n] ... of the next step (the two alternate)
+  float* pv = vv2 + n4;                // [n] work vector
+  float* beta = pv + n4;               // [n] reflector scales
+  float* dn = beta + n4;               // [n] diagonal of T / |T| for the Sturm counts
+  float2* cs = reinterpret_cast<float2*>(dn + n4);     // [4 n floats] partial sums of the reduction
+  float* qf = reinterpret_cast<float*>(cs) + 4 * n4;   // [16 n] reflector block and partial products
+  float* A = qf + 16 * n4;             // [n][ld]
   __shared__ float s_red[16];
   __shared__ int s_fail;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -847,16 +849,20 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   __syncthreads();
 
   // ---------------- Householder tridiagonalisation ----------------
-  // Four block barriers per column and no warp reductions inside the O(m^2) parts: a thread owns
-  // one column c of the trailing block and a range of its rows (the block is symmetric, so the
-  // column sum over that range is a partial of (B v)_c); the ranges are combined through shared
-  // memory.  |x|^2 of the next column is gathered while the trailing block is updated.
+  // Three block barriers per column and no warp reductions inside the O(m^2) parts: a thread
+  // owns one column c of the trailing block and a range of its rows (the block is symmetric, so
+  // the column sum over that range is a partial of (B v)_c); the ranges are combined through
+  // shared memory.  While the trailing block is updated, the thread that owns its first column
+  // also writes that column out as the next step's vector and gathers its |x|^2, so a step
+  // starts with everything it needs except the square root, which every thread takes itself.
+  // Vector entries are read four at a time (one broadcast load per four rows).
   __shared__ float s_sig[16];
   float* part = reinterpret_cast<float*>(cs);  // [<= 4][n] partial products (cs is free here)
   {
     float ps = 0.f;
     for (int r = tid; r + 1 < n; r += 512) {
       const float x = A[(1 + r) * ld];
+      vv[r] = x;
       ps = fmaf(x, x, ps);
     }
 #pragma unroll
@@ -864,12 +870,15 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     if (lane == 0) s_sig[warp] = ps;
     __syncthreads();
   }
+  int cw = 0, G = 1, g = 0, c = 0;  // thread layout: cw warps cover the columns, G row ranges
   for (int j = 0; j + 2 < n; ++j) {
     const int m = n - j - 1;  // order of the trailing block B = A[j+1.., j+1..]
+    float* vc = (j & 1) ? vv2 : vv;  // x of this step (v is x with v_0 in place of its entry 0)
+    float* vn = (j & 1) ? vv : vv2;  // x of the next step
     float sigma = 0.f;
 #pragma unroll
     for (int w = 0; w < 16; ++w) sigma += s_sig[w];
-    const float x0 = A[(j + 1) * ld + j];
+    const float x0 = vc[0];
     const float tail = sigma - x0 * x0;  // |x|^2 without its first entry
     // reflector H = I - bj v v^T with v = x - alpha e_1; a column already in tridiagonal form
     // gets bj = 0 (H = I) and keeps its entries
@@ -877,34 +886,34 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     const float alpha = skip ? x0 : -copysignf(sqrtf(sigma), x0);
     const float v0 = skip ? x0 : x0 - alpha;
     const float bj = skip ? 0.f : 2.0f / (tail + v0 * v0);
-    for (int r = tid; r < m; r += 512) {
-      const float x = (r == 0) ? v0 : A[(j + 1 + r) * ld + j];
-      vv[r] = x;
-      if (r == 0) A[(j + 1) * ld + j] = x;  // the column is kept for the accumulation of Q
-    }
     if (tid == 0) {
       dv[j] = A[j * ld + j];
       ev[j] = alpha;
       beta[j] = bj;
     }
-    __syncthreads();
-    // thread layout of this step: cw warps cover the m columns, G row ranges side by side
-    const int cw = (m + 31) >> 5;
-    const int G = min(4, 16 / cw);
-    const int g = warp / cw, c = (warp - g * cw) * 32 + lane;
+    if (((m + 31) >> 5) != cw) {
+      cw = (m + 31) >> 5;
+      G = min(4, 16 / cw);
+      g = warp / cw;
+      c = (warp - g * cw) * 32 + lane;
+    }
     const bool on = (g < G) && (c < m);
-    const int per = (m + G - 1) / G;
+    const int per = ((G == 4 ? (m + 3) >> 2 : (m + G - 1) / G) + 3) & ~3;  // a multiple of four
     const int r_lo = g * per, r_hi = min(m, r_lo + per);
     float* colp = A + (j + 1) * ld + j + 1 + c;  // B[0][c]; rows are ld apart
     if (on) {
-      float a0 = 0.f, a1 = 0.f;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       int r = r_lo;
-      for (; r + 1 < r_hi; r += 2) {
-        a0 = fmaf(colp[r * ld], vv[r], a0);
-        a1 = fmaf(colp[(r + 1) * ld], vv[r + 1], a1);
+      for (; r + 3 < r_hi; r += 4) {
+        float4 v4 = *reinterpret_cast<const float4*>(vc + r);
+        if (r == 0) v4.x = v0;
+        a0 = fmaf(colp[r * ld], v4.x, a0);
+        a1 = fmaf(colp[(r + 1) * ld], v4.y, a1);
+        a2 = fmaf(colp[(r + 2) * ld], v4.z, a2);
+        a3 = fmaf(colp[(r + 3) * ld], v4.w, a3);
       }
-      if (r < r_hi) a0 = fmaf(colp[r * ld], vv[r], a0);
-      part[g * n + c] = a0 + a1;
+      for (; r < r_hi; ++r) a0 = fmaf(colp[r * ld], (r == 0) ? v0 : vc[r], a0);
+      part[g * n + c] = (a0 + a1) + (a2 + a3);
     }
     __syncthreads();
     // p = bj * B v ; v.p
@@ -914,8 +923,10 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       for (int q = 0; q < G; ++q) t += part[q * n + c];
       const float pc = bj * t;
       pv[c] = pc;
-      vpp = vv[c] * pc;
+      vpp = ((c == 0) ? v0 : vc[c]) * pc;
     }
+    // the column is kept for the accumulation of Q (everyone has read its x_0 by now)
+    if (tid == 0) A[(j + 1) * ld + j] = v0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) vpp += __shfl_xor_sync(0xffffffffu, vpp, o);
     if (lane == 0) s_red[warp] = vpp;
@@ -927,12 +938,34 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     // B -= v w^T + w v^T ; column 0 of the new B, below its top entry, is the next x
     float sig_part = 0.f;
     if (on) {
-      const float vc = vv[c], wc = fmaf(-K, vc, pv[c]);
-      for (int r = r_lo; r < r_hi; ++r) {
-        const float vr = vv[r], wr = fmaf(-K, vr, pv[r]);
-        const float nv = colp[r * ld] - fmaf(vr, wc, wr * vc);
+      const bool first = (c == 0);
+      const float vcc = first ? v0 : vc[c], wc = fmaf(-K, vcc, pv[c]);
+      int r = r_lo;
+      for (; r + 3 < r_hi; r += 4) {
+        float4 v4 = *reinterpret_cast<const float4*>(vc + r);
+        if (r == 0) v4.x = v0;
+        const float4 p4 = *reinterpret_cast<const float4*>(pv + r);
+        const float vr[4] = {v4.x, v4.y, v4.z, v4.w};
+        const float pr[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float wr = fmaf(-K, vr[u], pr[u]);
+          const float nv = colp[(r + u) * ld] - fmaf(vr[u], wc, wr * vcc);
+          colp[(r + u) * ld] = nv;
+          if (first && r + u >= 1) {
+            vn[r + u - 1] = nv;
+            sig_part = fmaf(nv, nv, sig_part);
+          }
+        }
+      }
+      for (; r < r_hi; ++r) {
+        const float vr = (r == 0) ? v0 : vc[r], wr = fmaf(-K, vr, pv[r]);
+        const float nv = colp[r * ld] - fmaf(vr, wc, wr * vcc);
         colp[r * ld] = nv;
-        if (c == 0 && r >= 1) sig_part = fmaf(nv, nv, sig_part);
+        if (first && r >= 1) {
+          vn[r - 1] = nv;
+          sig_part = fmaf(nv, nv, sig_part);
+        }
       }
     }
     // only lane 0 of the first warp of each range holds a non-zero partial
@@ -1296,24 +1329,58 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     __syncthreads();
     for (int p = tid; p < n; p += 512) theta[(size_t)b * n + p] = fmaxf(e2[p], 0.f);
     // ---------------- Z = Q Y:  ZT[p][i] = sum_j Q[i][j] Y[j][p] ----------------
-    // thread = (eigenvector p, group of 8 rows i); Q rows are broadcast reads from shared memory
+    // thread = (four eigenvectors p, twelve rows i): per j one 16-byte load of Y (coalesced over
+    // p) and twelve broadcast reads of Q from shared memory feed 48 multiply-adds
     float* out = ZTg + img;
-    const int ngrp = (n + 7) / 8;
-    for (int w = tid; w < n * ngrp; w += 512) {
-      const int grp = w / n, p = w - grp * n;
-      const int i0 = grp * 8;
-      float acc[8];
+    const bool vec = (n & 3) == 0;
+    const int npg = (n + 3) >> 2, nrg = (n + 11) / 12;
+    for (int w = tid; w < npg * nrg; w += 512) {
+      const int rg = w / npg, pg = w - rg * npg;
+      const int p0 = pg * 4, i0 = rg * 12;
+      float acc[12][4];
+      const float* qrow[12];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) acc[u] = 0.f;
+      for (int u = 0; u < 12; ++u) {
+        qrow[u] = A + min(i0 + u, n - 1) * ld;  // rows past the end are computed and dropped
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = 0.f;
+      }
+#pragma unroll 4
       for (int j = 0; j < n; ++j) {
-        const float yv = __ldcg(y + (size_t)j * n + p);
+        float4 yv;
+        const float* yr = y + (size_t)j * n + p0;
+        if (vec) {
+          yv = __ldcg(reinterpret_cast<const float4*>(yr));
+        } else {
+          yv.x = __ldcg(yr);
+          yv.y = (p0 + 1 < n) ? __ldcg(yr + 1) : 0.f;
+          yv.z = (p0 + 2 < n) ? __ldcg(yr + 2) : 0.f;
+          yv.w = (p0 + 3 < n) ? __ldcg(yr + 3) : 0.f;
+        }
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-          if (i0 + u < n) acc[u] = fmaf(A[(i0 + u) * ld + j], yv, acc[u]);
+        for (int u = 0; u < 12; ++u) {
+          const float a = qrow[u][j];
+          acc[u][0] = fmaf(a, yv.x, acc[u][0]);
+          acc[u][1] = fmaf(a, yv.y, acc[u][1]);
+          acc[u][2] = fmaf(a, yv.z, acc[u][2]);
+          acc[u][3] = fmaf(a, yv.w, acc[u][3]);
+        }
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if (i0 + u < n) out[(size_t)p * n + i0 + u] = acc[u];
+      for (int v = 0; v < 4; ++v) {
+        if (p0 + v >= n) continue;
+        float* orow = out + (size_t)(p0 + v) * n + i0;
+        if (vec && i0 + 12 <= n) {
+#pragma unroll
+          for (int u = 0; u < 12; u += 4)
+            *reinterpret_cast<float4*>(orow + u) =
+                make_float4(acc[u][v], acc[u + 1][v], acc[u + 2][v], acc[u + 3][v]);
+        } else {
+#pragma unroll
+          for (int u = 0; u < 12; ++u)
+            if (i0 + u < n) orow[u] = acc[u][v];
+        }
+      }
     }
   }
   if (tid == 0 && s_fail) atomicMax(&status[b], (int)TC_ERR_NOT_CONVERGED);
@@ -1345,7 +1412,7 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
                           float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_JACOBI, st);
   {
-    const size_t tri = ((size_t)n * (n | 1) + 26 * (size_t)n) * sizeof(float);
+    const size_t tri = ((size_t)n * (n | 1) + 27 * (size_t)((n + 3) & ~3)) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       cudaFuncSetAttribute((const void*)tridiag_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
       { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status); note_launch(); }
