@@ -1122,14 +1122,14 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     }
     if (lane == 0) {
       s_red[warp] = lo;
-      reinterpret_cast<float*>(cs)[warp] = hi;
+      s_sig[warp] = hi;
     }
     bar_named(2, ET);
     lo = s_red[0];
-    hi = reinterpret_cast<float*>(cs)[0];
+    hi = s_sig[0];
     for (int w = 1; w < nbw; ++w) {
       lo = fminf(lo, s_red[w]);
-      hi = fmaxf(hi, reinterpret_cast<float*>(cs)[w]);
+      hi = fmaxf(hi, s_sig[w]);
     }
     const float tn = fmaxf(fabsf(lo), fabsf(hi));
     lo -= 2.4e-7f * tn + 1e-30f;
@@ -1144,22 +1144,26 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       e2[i] = e2[i] * itn * itn;
     }
     bar_named(2, ET);
+    // the entries of two steps side by side, one 16-byte load per trip of the count below
+    float4* tq = reinterpret_cast<float4*>(cs);
+    const int ntrip = (n - 1) >> 1;
+    for (int t = tid; t < ntrip; t += ET)
+      tq[t] = make_float4(dn[2 * t + 1], e2[2 * t], dn[2 * t + 2], e2[2 * t + 1]);
+    bar_named(2, ET);
     auto sturm = [&](float x) {
-      // two steps per trip: the diagonal and off-diagonal entries of both are loaded up front,
-      // and the pair is re-centred once per trip (entries can be as small as rounding noise,
-      // 1e-7 of the largest, so it can shrink by 1e-14 in a trip: the thresholds leave room)
+      // two steps per trip, and the pair is re-centred once per trip (entries can be as small as
+      // rounding noise, 1e-7 of the largest, so it can shrink by 1e-14 in a trip: the thresholds
+      // leave room).  A sign change is a difference of sign bits; a zero takes the sign of its
+      // bit, which gives the same total because the value after it has the opposite sign of the
+      // one before it.
       float p0 = 1.f, p1 = dn[0] - x;
-      bool neg = p1 < 0.f;
-      int cnt = neg;
-      int i = 1;
-      for (; i + 1 < n; i += 2) {
-        const float da = dn[i] - x, db = dn[i + 1] - x, ea = e2[i - 1], eb = e2[i];
-        const float pa = fmaf(da, p1, -ea * p0);
-        const float pb = fmaf(db, pa, -eb * p1);
-        const bool na = (pa < 0.f) || (pa == 0.f && !neg);  // an exact zero counts as a change
-        const bool nb2 = (pb < 0.f) || (pb == 0.f && !na);
-        cnt += (na != neg) + (nb2 != na);
-        neg = nb2;
+      unsigned cnt = __float_as_uint(p1) >> 31;
+      for (int t = 0; t < ntrip; ++t) {
+        const float4 q = tq[t];
+        const float pa = fmaf(q.x - x, p1, -q.y * p0);
+        const float pb = fmaf(q.z - x, pa, -q.w * p1);
+        cnt += ((__float_as_uint(pa) ^ __float_as_uint(p1)) >> 31) +
+               ((__float_as_uint(pb) ^ __float_as_uint(pa)) >> 31);
         p0 = pa;
         p1 = pb;
         const float sc = fmaxf(fabsf(p0), fabsf(p1));
@@ -1171,19 +1175,40 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
           p1 *= 1e-16f;
         }
       }
-      if (i < n) {
-        const float pa = fmaf(dn[i] - x, p1, -e2[i - 1] * p0);
-        const bool na = (pa < 0.f) || (pa == 0.f && !neg);
-        cnt += (na != neg);
+      if (!(n & 1)) {  // one step left
+        const float pa = fmaf(dn[n - 1] - x, p1, -e2[n - 2] * p0);
+        cnt += (__float_as_uint(pa) ^ __float_as_uint(p1)) >> 31;
       }
-      return cnt;
+      return (int)cnt;
     };
     const float lon = lo * itn, hin = hi * itn;
+    // First round, shared by all eigenvalues: counts at n points spaced geometrically from the
+    // top of the spectrum down to a little under the smallest eigenvalue that can pass the rank
+    // cut-off.  Each eigenvalue starts its own bisection from the two points around it.
+    int* gcnt = reinterpret_cast<int*>(pv);
+    const float glo = fmaxf(0.06f * rank_tol * rank_tol, 1e-9f);
+    const bool use_grid = hin > 2.0f * glo;
+    const float lr = use_grid ? log2f(glo / hin) / (float)n : 0.f;
+    auto grid = [&](int t) { return hin * exp2f(lr * (float)(n - t)); };
+    if (use_grid) {
+      if (tid < n) gcnt[tid] = sturm(grid(tid));
+      bar_named(2, ET);
+    }
+    float a = lon, bhi = hin;
+    if (use_grid && tid < n) {
+      int tl = -1, th = n;  // the count is 0 at lon (t = -1) and n at hin (t = n)
+      while (th - tl > 1) {
+        const int mid = (tl + th) >> 1;
+        if (gcnt[mid] > tid) th = mid; else tl = mid;
+      }
+      if (tl >= 0) a = fmaxf(lon, grid(tl));
+      if (th < n) bhi = fminf(hin, grid(th));
+    }
+    bar_named(2, ET);  // the counts are overwritten by the eigenvalues below
     if (tid < n) {
       // eigenvalue number tid (0 = smallest): plain bisection, one thread per eigenvalue (the
       // counts are bound by instruction issue, so evaluating several points per round on
       // neighbouring lanes costs more than the rounds it saves)
-      float a = lon, bhi = hin;
       for (int it = 0; it < 48; ++it) {
         const float x = 0.5f * (a + bhi);
         if (!(x > a) || !(x < bhi)) break;
