@@ -1,3 +1,4 @@
+#include <type_traits>
 // Dense linear algebra behind Eq. 3-5 / 3-6: the eigen-decomposition of the Gram matrix
 // G = O O^T = U Sigma^2 U^T, which yields the singular values and the rows of U Sigma that the
 // information contribution score sums.
@@ -856,36 +857,47 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   // also writes that column out as the next step's vector and gathers its |x|^2, so a step
   // starts with everything it needs except the square root, which every thread takes itself.
   // Vector entries are read four at a time (one broadcast load per four rows).
+  // The scalar parts of a step are repeated by every warp, four warps to a scheduler, so what
+  // counts there is the number of instructions: sums come as one or two 16-byte loads, the
+  // square root and the reciprocal as a Newton step on the hardware approximations.
   __shared__ float s_sig[16];
+  __shared__ __align__(16) float s_sig4[4];  // |x|^2 of the next column, one partial per row range
+  __shared__ __align__(16) float s_red8[8];  // v.p, one partial per warp of the first row range
   float* part = reinterpret_cast<float*>(cs);  // [<= 4][n] partial products (cs is free here)
-  {
+  if (warp == 0) {
     float ps = 0.f;
-    for (int r = tid; r + 1 < n; r += 512) {
+    for (int r = lane; r + 1 < n; r += 32) {
       const float x = A[(1 + r) * ld];
       vv[r] = x;
       ps = fmaf(x, x, ps);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
-    if (lane == 0) s_sig[warp] = ps;
-    __syncthreads();
+    if (lane < 4) s_sig4[lane] = (lane == 0) ? ps : 0.f;
   }
+  __syncthreads();
   int cw = 0, G = 1, g = 0, c = 0;  // thread layout: cw warps cover the columns, G row ranges
+  bool lead = false;                // this warp holds column 0 of its row range
   for (int j = 0; j + 2 < n; ++j) {
     const int m = n - j - 1;  // order of the trailing block B = A[j+1.., j+1..]
     float* vc = (j & 1) ? vv2 : vv;  // x of this step (v is x with v_0 in place of its entry 0)
     float* vn = (j & 1) ? vv : vv2;  // x of the next step
-    float sigma = 0.f;
-#pragma unroll
-    for (int w = 0; w < 16; ++w) sigma += s_sig[w];
+    const float4 s4 = *reinterpret_cast<const float4*>(s_sig4);
+    const float sigma = (s4.x + s4.y) + (s4.z + s4.w);
     const float x0 = vc[0];
     const float tail = sigma - x0 * x0;  // |x|^2 without its first entry
     // reflector H = I - bj v v^T with v = x - alpha e_1; a column already in tridiagonal form
     // gets bj = 0 (H = I) and keeps its entries
     const bool skip = !(tail > 1e-30f * sigma) || !(sigma > 0.f);
-    const float alpha = skip ? x0 : -copysignf(sqrtf(sigma), x0);
+    const float rs = rsqrtf(sigma);
+    float nrm = sigma * rs;
+    nrm = fmaf(fmaf(-nrm, nrm, sigma), 0.5f * rs, nrm);
+    const float alpha = skip ? x0 : -copysignf(nrm, x0);
     const float v0 = skip ? x0 : x0 - alpha;
-    const float bj = skip ? 0.f : 2.0f / (tail + v0 * v0);
+    const float den = tail + v0 * v0;
+    float rc = __fdividef(2.0f, den);
+    rc = fmaf(fmaf(-den, rc, 2.0f), 0.5f * rc, rc);
+    const float bj = skip ? 0.f : rc;
     if (tid == 0) {
       dv[j] = A[j * ld + j];
       ev[j] = alpha;
@@ -896,21 +908,25 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       G = min(4, 16 / cw);
       g = warp / cw;
       c = (warp - g * cw) * 32 + lane;
+      lead = (warp == g * cw);
     }
     const bool on = (g < G) && (c < m);
-    const int per = ((G == 4 ? (m + 3) >> 2 : (m + G - 1) / G) + 3) & ~3;  // a multiple of four
+    // rows per range, a multiple of four (G is 2, 3 or 4; the multiplication is a division by 3)
+    const int per0 = (G == 4) ? (m + 3) >> 2 : (G == 3) ? ((m + 2) * 21846) >> 16 : (m + 1) >> 1;
+    const int per = (per0 + 3) & ~3;
     const int r_lo = g * per, r_hi = min(m, r_lo + per);
     float* colp = A + (j + 1) * ld + j + 1 + c;  // B[0][c]; rows are ld apart
     if (on) {
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       int r = r_lo;
-      for (; r + 3 < r_hi; r += 4) {
+      const float* bp = colp + r_lo * ld;
+      for (; r + 3 < r_hi; r += 4, bp += 4 * ld) {
         float4 v4 = *reinterpret_cast<const float4*>(vc + r);
         if (r == 0) v4.x = v0;
-        a0 = fmaf(colp[r * ld], v4.x, a0);
-        a1 = fmaf(colp[(r + 1) * ld], v4.y, a1);
-        a2 = fmaf(colp[(r + 2) * ld], v4.z, a2);
-        a3 = fmaf(colp[(r + 3) * ld], v4.w, a3);
+        a0 = fmaf(bp[0], v4.x, a0);
+        a1 = fmaf(bp[ld], v4.y, a1);
+        a2 = fmaf(bp[2 * ld], v4.z, a2);
+        a3 = fmaf(bp[3 * ld], v4.w, a3);
       }
       for (; r < r_hi; ++r) a0 = fmaf(colp[r * ld], (r == 0) ? v0 : vc[r], a0);
       part[g * n + c] = (a0 + a1) + (a2 + a3);
@@ -919,29 +935,33 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     // p = bj * B v ; v.p
     float vpp = 0.f;
     if (g == 0 && c < m) {
-      float t = 0.f;
-      for (int q = 0; q < G; ++q) t += part[q * n + c];
-      const float pc = bj * t;
+      const float t0 = part[c], t1 = part[n + c];
+      const float t2 = (G > 2) ? part[2 * n + c] : 0.f, t3 = (G > 3) ? part[3 * n + c] : 0.f;
+      const float pc = bj * ((t0 + t1) + (t2 + t3));
       pv[c] = pc;
       vpp = ((c == 0) ? v0 : vc[c]) * pc;
     }
     // the column is kept for the accumulation of Q (everyone has read its x_0 by now)
     if (tid == 0) A[(j + 1) * ld + j] = v0;
+    if (warp < 8) {  // the first row range is at most seven warps; the others hold zero
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) vpp += __shfl_xor_sync(0xffffffffu, vpp, o);
-    if (lane == 0) s_red[warp] = vpp;
+      for (int o = 16; o > 0; o >>= 1) vpp += __shfl_xor_sync(0xffffffffu, vpp, o);
+      if (lane == 0) s_red8[warp] = vpp;
+    }
     __syncthreads();
-    float vp = 0.f;
-#pragma unroll
-    for (int w = 0; w < 16; ++w) vp += s_red[w];
+    const float4 ra = *reinterpret_cast<const float4*>(s_red8);
+    const float4 rb = *reinterpret_cast<const float4*>(s_red8 + 4);
+    const float vp = ((ra.x + ra.y) + (ra.z + ra.w)) + ((rb.x + rb.y) + (rb.z + rb.w));
     const float K = 0.5f * bj * vp;  // w = p - K v
     // B -= v w^T + w v^T ; column 0 of the new B, below its top entry, is the next x
     float sig_part = 0.f;
-    if (on) {
-      const bool first = (c == 0);
-      const float vcc = first ? v0 : vc[c], wc = fmaf(-K, vcc, pv[c]);
+    auto update = [&](auto tag) {
+      constexpr bool LEAD = decltype(tag)::value;  // this warp's lane 0 owns column 0
+      const bool first = LEAD && (lane == 0);
+      const float vcc = (c == 0) ? v0 : vc[c], wc = fmaf(-K, vcc, pv[c]);
       int r = r_lo;
-      for (; r + 3 < r_hi; r += 4) {
+      float* bp = colp + r_lo * ld;
+      for (; r + 3 < r_hi; r += 4, bp += 4 * ld) {
         float4 v4 = *reinterpret_cast<const float4*>(vc + r);
         if (r == 0) v4.x = v0;
         const float4 p4 = *reinterpret_cast<const float4*>(pv + r);
@@ -950,11 +970,13 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const float wr = fmaf(-K, vr[u], pr[u]);
-          const float nv = colp[(r + u) * ld] - fmaf(vr[u], wc, wr * vcc);
-          colp[(r + u) * ld] = nv;
-          if (first && r + u >= 1) {
-            vn[r + u - 1] = nv;
-            sig_part = fmaf(nv, nv, sig_part);
+          const float nv = bp[u * ld] - fmaf(vr[u], wc, wr * vcc);
+          bp[u * ld] = nv;
+          if (LEAD) {
+            if (first && r + u >= 1) {
+              vn[r + u - 1] = nv;
+              sig_part = fmaf(nv, nv, sig_part);
+            }
           }
         }
       }
@@ -962,14 +984,18 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         const float vr = (r == 0) ? v0 : vc[r], wr = fmaf(-K, vr, pv[r]);
         const float nv = colp[r * ld] - fmaf(vr, wc, wr * vcc);
         colp[r * ld] = nv;
-        if (first && r >= 1) {
-          vn[r - 1] = nv;
-          sig_part = fmaf(nv, nv, sig_part);
+        if (LEAD) {
+          if (first && r >= 1) {
+            vn[r - 1] = nv;
+            sig_part = fmaf(nv, nv, sig_part);
+          }
         }
       }
+    };
+    if (on) {
+      if (lead) update(std::true_type{}); else update(std::false_type{});
     }
-    // only lane 0 of the first warp of each range holds a non-zero partial
-    if (lane == 0) s_sig[warp] = sig_part;
+    if (lead && lane == 0 && g < 4) s_sig4[g] = sig_part;  // zero from a range that is not in use
     __syncthreads();
   }
   if (tid == 0) {
