@@ -126,9 +126,10 @@ Plan make_plan(const Dims& D) {
     P.Y0 = take(B * N * k * 4);
     P.Y1 = take(B * N * k * 4);
     P.Y2 = take(B * N * k * 4);
-    P.Sm = take(B * k * k * 4);
+    const size_t parts = (size_t)tn_parts(D.k);  // k x k products arrive in this many parts
+    P.Sm = take(B * k * k * 4 * parts);
     P.Rinv = take(B * k * k * 4);
-    P.Hm = take(B * k * k * 4);
+    P.Hm = take(B * k * k * 4 * parts);
   }
   P.W = take(B * k * k * 4);
   P.ZT = take(B * k * k * 4);

@@ -253,6 +253,139 @@ static void gemm(const TA* A, const TB* B, float* C, int M, int N, int K, int ld
   }
 }
 
+// ==========================================================================================
+// C = A^T B for tall operands with few columns (n <= 144, n a multiple of 4), where C is known
+// to be symmetric (A = B, or B = G A with G symmetric): only the entries on or above the
+// diagonal are computed and each is written to both places.
+//   A, B [K][n] row-major;  C parts: [nparts][n][n] per image, part s = the sum over the s-th
+//   chunk of K.  The consumer adds the parts (in order, so the result is deterministic).
+// One block per (chunk, image): 192 threads.  The columns are split in a low and a high half;
+// thread (ty, tx), tx >= ty, of the triangular grid holds rows {4 ty.., half + 4 ty..} x columns
+// {4 tx.., half + 4 tx..}: four 4 x 4 blocks, of which three lie on or above the diagonal and the
+// fourth is the mirror image of a block no thread of the triangle holds.  A 16-deep slice costs
+// four 16-byte reads of shared memory (neighbouring threads read neighbouring vectors) per 64
+// multiply-adds.
+// ==========================================================================================
+constexpr int TN_MAX = 144, TN_LD = 152, TN_PARTS = 4;
+
+template <bool SAME>
+__global__ void __launch_bounds__(192) gemm_tn_upper_kernel(const float* __restrict__ A,
+                                                           const float* __restrict__ B,
+                                                           float* __restrict__ C, int n, int K,
+                                                           int chunk, size_t sA, size_t sB,
+                                                           size_t sC) {
+  __shared__ __align__(16) float As[16][TN_LD];
+  __shared__ __align__(16) float Bs[SAME ? 1 : 16][TN_LD];
+  const int tid = threadIdx.x, s = blockIdx.x, img = blockIdx.y;
+  A += (size_t)img * sA;
+  B += (size_t)img * sB;
+  C += (size_t)img * sC + (size_t)s * n * n;
+  const int k_lo = s * chunk, k_hi = min(K, k_lo + chunk);
+  const int nt = (n + 7) >> 3;  // tiles per side; the high half starts at column 4 nt
+  const int half = 4 * nt;
+  int ty = 0, rem = tid;
+  while (ty < nt && rem >= nt - ty) {
+    rem -= nt - ty;
+    ++ty;
+  }
+  const bool active = ty < nt;
+  const int tx = ty + rem;
+  const int nv = n >> 2;                 // 16-byte vectors per row
+  const int nvec = 16 * nv;              // per slice
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+  float4 ra[3], rb[3];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      const int e = tid + i * 192;
+      const int kr = e / nv, cv = e - kr * nv;
+      float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
+      if (e < nvec && k0 + kr < k_hi) {
+        va = __ldg(reinterpret_cast<const float4*>(A + (size_t)(k0 + kr) * n) + cv);
+        if (!SAME) vb = __ldg(reinterpret_cast<const float4*>(B + (size_t)(k0 + kr) * n) + cv);
+      }
+      ra[i] = va;
+      rb[i] = vb;
+    }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      const int e = tid + i * 192;
+      const int kr = e / nv, cv = e - kr * nv;
+      if (e < nvec) {
+        *reinterpret_cast<float4*>(&As[kr][cv * 4]) = ra[i];
+        if (!SAME) *reinterpret_cast<float4*>(&Bs[kr][cv * 4]) = rb[i];
+      }
+    }
+  };
+  const float(*Bt)[TN_LD] = SAME ? As : Bs;
+  fetch(k_lo);
+  for (int k0 = k_lo; k0 < k_hi; k0 += 16) {
+    stash();
+    __syncthreads();
+    if (k0 + 16 < k_hi) fetch(k0 + 16);
+    if (active) {
+#pragma unroll
+      for (int kk = 0; kk < 16; ++kk) {
+        const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+        const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][half + ty * 4]);
+        const float4 b0 = *reinterpret_cast<const float4*>(&Bt[kk][tx * 4]);
+        const float4 b1 = *reinterpret_cast<const float4*>(&Bt[kk][half + tx * 4]);
+        const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+        const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+      }
+    }
+    __syncthreads();
+  }
+  if (!active) return;
+  // every unordered pair {r, c} is produced by exactly one thread and written to both places
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = (i < 4) ? ty * 4 + i : half + ty * 4 + i - 4;
+    if (r >= n) continue;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int c = (j < 4) ? tx * 4 + j : half + tx * 4 + j - 4;
+      if (c >= n) continue;
+      if (c >= r || tx > ty) {
+        C[(size_t)r * n + c] = acc[i][j];
+        if (c != r) C[(size_t)c * n + r] = acc[i][j];
+      }
+    }
+  }
+}
+
+// Number of parts the k x k products A^T B are delivered in (1 = the general kernel).
+int tn_parts(int k) { return (k <= TN_MAX && (k & 3) == 0 && k >= 8) ? TN_PARTS : 1; }
+
+// C (nparts parts per image, image stride nparts * n * n) = A^T B, symmetric.
+static void gemm_tn_sym(const float* A, const float* B, float* C, int n, int K, size_t sA, size_t sB,
+                        int batch, cudaStream_t st, int cls) {
+  const int parts = tn_parts(n);
+  if (parts == 1) {
+    gemm<float, float, true, false>(A, B, C, n, n, K, n, n, n, sA, sB, (size_t)n * n, batch, st, cls,
+                                    A == B ? GEMM_SYM : 0);
+    return;
+  }
+  Scope scope_(cls, st);
+  const int chunk = ((K + parts - 1) / parts + 15) / 16 * 16;
+  dim3 grid(parts, batch);
+  const size_t sC = (size_t)parts * n * n;
+  if (A == B)
+    { gemm_tn_upper_kernel<true><<<grid, 192, 0, st>>>(A, B, C, n, K, chunk, sA, sB, sC); note_launch(); }
+  else
+    { gemm_tn_upper_kernel<false><<<grid, 192, 0, st>>>(A, B, C, n, K, chunk, sA, sB, sC); note_launch(); }
+}
+
 // G = O O^T for float32 inputs (and, until the tensor-core kernel takes over, float16 ones).
 tc_status launch_gram_simt(const Dims& D, const void* O, float* G, cudaStream_t st) {
   const size_t sO = (size_t)D.N * D.d, sG = (size_t)D.N * D.N;
@@ -425,7 +558,8 @@ constexpr int CNB = 16;
 __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __restrict__ S,
                                                               float* __restrict__ RinvT, int k,
                                                               float shift_rel,
-                                                              int32_t* __restrict__ status) {
+                                                              int32_t* __restrict__ status,
+                                                              int nparts) {
   extern __shared__ float A[];  // [k][ld], ld odd: rows and columns both walk all banks
   __shared__ float s_red[16];
   __shared__ float s_row[2][CNB];
@@ -433,10 +567,14 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ld = k | 1;
   const size_t kk = (size_t)k * k;
-  const float* Sb = S + b * kk;
+  const float* Sb = S + (size_t)b * nparts * kk;  // S arrives as nparts parts to be added up
 
   float md = 0.f;
-  for (int i = tid; i < k; i += 512) md = fmaxf(md, Sb[(size_t)i * k + i]);
+  for (int i = tid; i < k; i += 512) {
+    float dsum = 0.f;
+    for (int q = 0; q < nparts; ++q) dsum += __ldg(Sb + q * kk + (size_t)i * k + i);
+    md = fmaxf(md, dsum);
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, o));
   if (lane == 0) s_red[warp] = md;
@@ -446,9 +584,27 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
   for (int w = 1; w < 16; ++w) md = fmaxf(md, s_red[w]);
   const float shift = shift_rel * md;
   const float tiny = fmaxf(md, 1e-30f) * 1e-12f;
-  for (int e = tid; e < (int)kk; e += 512) {
-    const int r = e / k, c = e - r * k;
-    A[r * ld + c] = Sb[e] + (r == c ? shift : 0.f);
+  if (nparts == 4 && (k & 3) == 0) {
+    // four parts, sixteen bytes at a time: all the loads of a trip are in flight together
+    const float4* S4 = reinterpret_cast<const float4*>(Sb);
+    const int kv = k >> 2, nv = (int)(kk >> 2);
+    for (int e = tid; e < nv; e += 512) {
+      const float4 p0 = __ldg(S4 + e), p1 = __ldg(S4 + nv + e), p2 = __ldg(S4 + 2 * nv + e),
+                   p3 = __ldg(S4 + 3 * nv + e);
+      const int r = e / kv, c = (e - r * kv) * 4;
+      float* dst = A + r * ld + c;
+      dst[0] = ((p0.x + p1.x) + (p2.x + p3.x)) + (r == c ? shift : 0.f);
+      dst[1] = ((p0.y + p1.y) + (p2.y + p3.y)) + (r == c + 1 ? shift : 0.f);
+      dst[2] = ((p0.z + p1.z) + (p2.z + p3.z)) + (r == c + 2 ? shift : 0.f);
+      dst[3] = ((p0.w + p1.w) + (p2.w + p3.w)) + (r == c + 3 ? shift : 0.f);
+    }
+  } else {
+    for (int e = tid; e < (int)kk; e += 512) {
+      const int r = e / k, c = e - r * k;
+      float v = 0.f;
+      for (int q = 0; q < nparts; ++q) v += Sb[q * kk + e];
+      A[r * ld + c] = v + (r == c ? shift : 0.f);
+    }
   }
   __syncthreads();
 
@@ -823,7 +979,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ u0g, float* __restrict__ u1g,
                                                          float* __restrict__ u2g, float* yg, float* __restrict__ mlg,
                                                          size_t ml_stride,
-                                                         int32_t* __restrict__ status) {
+                                                         int32_t* __restrict__ status, int nparts) {
   extern __shared__ __align__(16) float sm[];
   const int ld = n | 1;
   const int n4 = (n + 3) & ~3;         // the vectors start on 16-byte boundaries
@@ -840,11 +996,33 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   __shared__ float s_red[16];
   __shared__ int s_fail;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* Hb = Hin + (size_t)b * n * n;
+  const float* Hb = Hin + (size_t)b * nparts * n * n;  // H arrives as nparts parts to be added up
 
-  for (int e = tid; e < n * n; e += 512) {
-    const int r = e / n, c = e - r * n;
-    A[r * ld + c] = 0.5f * (Hb[e] + Hb[(size_t)c * n + r]);
+  if (nparts == 4 && (n & 3) == 0) {
+    // the parts come from the kernel that writes every entry and its mirror image with the
+    // same bits, so their sum is symmetric as it stands
+    const float4* H4 = reinterpret_cast<const float4*>(Hb);
+    const int kv = n >> 2, nv = (n * n) >> 2;
+    for (int e = tid; e < nv; e += 512) {
+      const float4 p0 = __ldg(H4 + e), p1 = __ldg(H4 + nv + e), p2 = __ldg(H4 + 2 * nv + e),
+                   p3 = __ldg(H4 + 3 * nv + e);
+      const int r = e / kv, c = (e - r * kv) * 4;
+      float* dst = A + r * ld + c;
+      dst[0] = (p0.x + p1.x) + (p2.x + p3.x);
+      dst[1] = (p0.y + p1.y) + (p2.y + p3.y);
+      dst[2] = (p0.z + p1.z) + (p2.z + p3.z);
+      dst[3] = (p0.w + p1.w) + (p2.w + p3.w);
+    }
+  } else {
+    for (int e = tid; e < n * n; e += 512) {
+      const int r = e / n, c = e - r * n;
+      float h = 0.f, ht = 0.f;
+      for (int q = 0; q < nparts; ++q) {
+        h += Hb[(size_t)q * n * n + e];
+        ht += Hb[(size_t)q * n * n + (size_t)c * n + r];
+      }
+      A[r * ld + c] = 0.5f * (h + ht);
+    }
   }
   if (tid == 0) s_fail = 0;
   __syncthreads();
@@ -1253,7 +1431,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     float* u0 = u0g + img;
     float* u1 = u1g + img;
     float* u2 = u2g + img;
-    float* y = yg + img;
+    float* y = yg + img * nparts;
     float* ml = mlg + (size_t)b * ml_stride;
     if (tid < n) {
       const int t = tid;
@@ -1460,13 +1638,14 @@ constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared 
 
 static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
                           int max_sweeps, float rank_tol, float* scr1, float* scr2, float* scr3,
-                          float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st) {
+                          float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st,
+                          int nparts = 1) {
   Scope scope_(KC_JACOBI, st);
   {
     const size_t tri = ((size_t)n * (n | 1) + 27 * (size_t)((n + 3) & ~3)) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       cudaFuncSetAttribute((const void*)tridiag_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
-      { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status); note_launch(); }
+      { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts); note_launch(); }
       return;
     }
   }
@@ -1487,14 +1666,14 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
 }
 
 static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
-                            float shift_rel, int32_t* status, cudaStream_t st) {
+                            float shift_rel, int32_t* status, cudaStream_t st, int nparts) {
   Scope scope_(KC_CHOL, st);
   const size_t blocked = (size_t)k * (k | 1) * sizeof(float);
   // (the blocked kernel keeps 2 x 4 outputs per thread in registers in its last step)
   if (blocked <= SMEM_LIMIT && (size_t)k * (CNB / 4) <= 2 * 512) {
     cudaFuncSetAttribute((const void*)chol_inv_blocked_kernel,
                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)blocked);
-    { chol_inv_blocked_kernel<<<batch, 512, blocked, st>>>(S, RinvT, k, shift_rel, status); note_launch(); }
+    { chol_inv_blocked_kernel<<<batch, 512, blocked, st>>>(S, RinvT, k, shift_rel, status, nparts); note_launch(); }
     return;
   }
   const size_t need = 2 * (size_t)k * k * sizeof(float);
@@ -1607,9 +1786,10 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   float* Y0 = (float*)(ws + P.Y0) + b0 * sY;
   float* Y1 = (float*)(ws + P.Y1) + b0 * sY;
   float* Y2 = (float*)(ws + P.Y2) + b0 * sY;
-  float* Sm = (float*)(ws + P.Sm) + b0 * sK;
+  const int parts = tn_parts(k);  // the k x k products come in this many parts per image
+  float* Sm = (float*)(ws + P.Sm) + b0 * sK * parts;
   float* Rinv = (float*)(ws + P.Rinv) + b0 * sK;
-  float* Hm = (float*)(ws + P.Hm) + b0 * sK;
+  float* Hm = (float*)(ws + P.Hm) + b0 * sK * parts;
 
   // 1. sketch of the column space of O
   {
@@ -1635,8 +1815,8 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   }
   // one Cholesky-QR pass: dst = src R^{-1},  R^T R = src^T src (+ shift)
   auto cholqr_pass = [&](const float* src, float* dst, float shift_rel) {
-    gemm<float, float, true, false>(src, src, Sm, k, k, N, k, k, k, sY, sY, sK, B, st, KC_GEMM_TN, GEMM_SYM);
-    launch_chol_inv(Sm, Rinv, W, k, B, shift_rel, img_status, st);
+    gemm_tn_sym(src, src, Sm, k, N, sY, sY, B, st, KC_GEMM_TN);
+    launch_chol_inv(Sm, Rinv, W, k, B, shift_rel, img_status, st, parts);
     gemm<float, float, false, true>(src, Rinv, dst, N, k, k, k, k, k, sY, sK, sY, B, st, KC_GEMM, GEMM_B_UPPER);
   };
   const float kShift = 1e-6f;
@@ -1651,9 +1831,9 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   cholqr_pass(Y1, Y2, 0.f);  // Q1 in Y2
   // 4. Rayleigh-Ritz:  H = Q1^T G Q1
   gemm<float, float, false, false>(G, Y2, Y1, N, k, N, N, k, k, sG, sY, sY, B, st, KC_GEMM_GQ);   // T = G Q1
-  gemm<float, float, true, false>(Y2, Y1, Hm, k, k, N, k, k, k, sY, sY, sK, B, st, KC_GEMM_TN);   // H = Q1^T T
+  gemm_tn_sym(Y2, Y1, Hm, k, N, sY, sY, B, st, KC_GEMM_TN);   // H = Q1^T T (symmetric)
   // scratch of the solver: W, Sm, Rinv, Hm (k x k each) and the first k x k of each image's Y1 panel
-  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, Sm, Rinv, Hm, Y1, sY, img_status, st);
+  launch_jacobi(Hm, W, ZT, theta, k, B, D.max_sweeps, D.rank_tol, Sm, Rinv, Hm, Y1, sY, img_status, st, parts);
   // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]
   gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
   Scope scope_(KC_ICS, st);

@@ -32,7 +32,7 @@ struct Plan {
   size_t sigma;    // [B, k] f32 (unsorted eigenvalue norms theta)
   size_t G;        // [B, N, N] f32
   size_t Y0, Y1, Y2;  // [B, N, k] f32 each (subspace solve only)
-  size_t Sm, Rinv, Hm;  // [B, k, k] f32 each (subspace solve only)
+  size_t Sm, Rinv, Hm;  // [B, k, k] f32 each (subspace solve only; Sm, Hm: tn_parts(k) of them)
   size_t W, ZT;    // [B, k, k] f32: Jacobi work matrix and accumulated rotations (column-major)
   size_t setA, setB, best_val, best_dst, msrc, mdst, kept;  // int32 / f32 lists
   size_t rank;     // [B] int32
@@ -41,6 +41,10 @@ struct Plan {
 };
 
 Plan make_plan(const Dims& D);
+
+// Number of parts per image in which the k x k products of the subspace solve are stored
+// (partial sums over chunks of the long dimension, added up by the kernel that reads them).
+int tn_parts(int k);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
