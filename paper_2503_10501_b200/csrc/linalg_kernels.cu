@@ -237,11 +237,146 @@ static void gemm_launch(const TA* A, const TB* B, float* C, int M, int N, int K,
   { gemm_kernel<TA, TB, TRA, TRB, RM, CN><<<grid, 256, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
 }
 
+// ==========================================================================================
+// The same product for float32 operands whose output is 48 k columns wide (the subspace
+// dimension 144 = 3 * 48):  C[m][n] = sum_k A[m][k] * opB[k][n],  A row-major.
+// (64 RM) x 48 tile per block of 192 threads = 12 (columns, four each) x 16 (rows, four in each
+// of RM groups of 64): a 16-deep slice costs RM + 1 16-byte reads of shared memory per 16 RM
+// multiply-adds, against RM + 3 reads per 12 RM in the kernel above.  Needs every operand
+// address 16-byte aligned (the caller checks).
+// ==========================================================================================
+template <bool TRB, int RM>
+__global__ void __launch_bounds__(192, 2) gemm_tall_kernel(const float* __restrict__ A,
+                                                          const float* __restrict__ B,
+                                                          float* __restrict__ C, int M, int N, int K,
+                                                          int lda, int ldb, int ldc, size_t sA,
+                                                          size_t sB, size_t sC, int flags) {
+  constexpr int BM = 64 * RM, BN = 48, BK = 16;
+  constexpr int NVA = BM * BK / 4, VA = (NVA + 191) / 192;  // A vectors per slice, per thread
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  A += (size_t)blockIdx.z * sA;
+  B += (size_t)blockIdx.z * sB;
+  C += (size_t)blockIdx.z * sC;
+  const int tid = threadIdx.x, tx = tid % 12, ty = tid / 12;
+  const int Kend = (flags & GEMM_B_UPPER) ? min(K, n0 + BN) : K;
+  float acc[4 * RM][4];
+#pragma unroll
+  for (int i = 0; i < 4 * RM; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  float4 ra[VA], rb;
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int i = 0; i < VA; ++i) {
+      const int e = tid + i * 192;
+      const int k = (e & 3) * 4, m = e >> 2;  // stored [m][k]: vectors run along k
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (e < NVA && m0 + m < M && k0 + k < Kend)
+        v = __ldg(reinterpret_cast<const float4*>(A + (size_t)(m0 + m) * lda + k0 + k));
+      ra[i] = v;
+    }
+    {
+      int n, k;
+      if (TRB) {  // stored [n][k]: vectors run along k
+        k = (tid & 3) * 4;
+        n = tid >> 2;
+      } else {  // stored [k][n]: vectors run along n
+        n = (tid % 12) * 4;
+        k = tid / 12;
+      }
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (n0 + n < N && k0 + k < Kend)
+        v = __ldg(reinterpret_cast<const float4*>(
+            TRB ? B + (size_t)(n0 + n) * ldb + k0 + k : B + (size_t)(k0 + k) * ldb + n0 + n));
+      rb = v;
+    }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int i = 0; i < VA; ++i) {
+      const int e = tid + i * 192;
+      if (e < NVA) {
+        const int k = (e & 3) * 4, m = e >> 2;
+        As[k][m] = ra[i].x;
+        As[k + 1][m] = ra[i].y;
+        As[k + 2][m] = ra[i].z;
+        As[k + 3][m] = ra[i].w;
+      }
+    }
+    if (TRB) {
+      const int k = (tid & 3) * 4, n = tid >> 2;
+      Bs[k][n] = rb.x;
+      Bs[k + 1][n] = rb.y;
+      Bs[k + 2][n] = rb.z;
+      Bs[k + 3][n] = rb.w;
+    } else {
+      *reinterpret_cast<float4*>(&Bs[tid / 12][(tid % 12) * 4]) = rb;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < Kend; k0 += BK) {
+    stash();
+    __syncthreads();
+    if (k0 + BK < Kend) fetch(k0 + BK);
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+      for (int g = 0; g < RM; ++g) {
+        const float4 av = *reinterpret_cast<const float4*>(&As[kk][g * 64 + ty * 4]);
+        const float a[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[g * 4 + i][j] = fmaf(a[i], bb[j], acc[g * 4 + i][j]);
+      }
+    }
+    __syncthreads();
+  }
+  const int gn = n0 + tx * 4;
+  if (gn >= N) return;  // N is a multiple of four: a thread's four columns are in or out together
+#pragma unroll
+  for (int g = 0; g < RM; ++g)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int gm = m0 + g * 64 + ty * 4 + i;
+      if (gm < M)
+        *reinterpret_cast<float4*>(C + (size_t)gm * ldc + gn) =
+            make_float4(acc[g * 4 + i][0], acc[g * 4 + i][1], acc[g * 4 + i][2], acc[g * 4 + i][3]);
+    }
+}
+
+template <bool TRB>
+static bool gemm_tall(const float* A, const float* B, float* C, int M, int N, int K, int lda, int ldb,
+                      int ldc, size_t sA, size_t sB, size_t sC, int batch, cudaStream_t st, int flags) {
+  if (N % 48 != 0 || M < 128 && M != 144 || ((lda | ldb | ldc | K) & 3) != 0 ||
+      ((sA | sB | sC) & 3) != 0 || ((((uintptr_t)A) | ((uintptr_t)B) | ((uintptr_t)C)) & 15) != 0)
+    return false;
+  // rows per tile: 192 unless 128 wastes less of the last tile
+  const bool three = ((M + 191) / 192) * 192 <= ((M + 127) / 128) * 128;
+  if (three) {
+    dim3 grid(N / 48, (M + 191) / 192, batch);
+    { gemm_tall_kernel<TRB, 3><<<grid, 192, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
+  } else {
+    dim3 grid(N / 48, (M + 127) / 128, batch);
+    { gemm_tall_kernel<TRB, 2><<<grid, 192, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
+  }
+  return true;
+}
+
 template <typename TA, typename TB, bool TRA, bool TRB>
 static void gemm(const TA* A, const TB* B, float* C, int M, int N, int K, int lda, int ldb,
                  int ldc, size_t sA, size_t sB, size_t sC, int batch, cudaStream_t st,
                  int cls = KC_GEMM, int flags = 0) {
   Scope scope_(cls, st);
+  if constexpr (std::is_same<TA, float>::value && std::is_same<TB, float>::value && !TRA) {
+    if (!(flags & GEMM_SYM) &&
+        gemm_tall<TRB>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, batch, st, flags))
+      return;
+  }
   // column tiles of 48 when they pad the width less than tiles of 64 (e.g. 144 = 3 * 48)
   const bool narrow = ((N + 47) / 48) * 48 < ((N + 63) / 64) * 64;
   if (M >= 256 && !(flags & GEMM_SYM)) {
