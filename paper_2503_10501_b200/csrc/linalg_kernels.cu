@@ -15,6 +15,18 @@
 
 namespace tc {
 
+// 16-byte asynchronous copy global -> shared; `bytes` = 16, or 0 to write zeros instead.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int bytes) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+
 // ==========================================================================================
 // Batched float32 GEMM on the plain ALUs:  C[m][n] = sum_k opA[m][k] * opB[k][n].
 //   opA[m][k] = TRA ? A[k * lda + m] : A[m * lda + k]
@@ -349,6 +361,100 @@ __global__ void __launch_bounds__(192, 2) gemm_tall_kernel(const float* __restri
     }
 }
 
+// The same tile for opB = B (stored [k][n]), the product with the long inner dimension (G Q):
+// both operands keep their global layout in shared memory, so slices arrive by asynchronous
+// 16-byte copies, TALL_STAGES of them in flight, with one barrier per slice.  A is held as
+// [m][16] with the four vectors of a row permuted by (m / 4) mod 4, which spreads the rows a
+// warp reads at once over the banks.
+constexpr int TALL_STAGES = 4;
+
+template <int RM>
+__global__ void __launch_bounds__(192, 2) gemm_tall_nn_kernel(const float* __restrict__ A,
+                                                             const float* __restrict__ B,
+                                                             float* __restrict__ C, int M, int N, int K,
+                                                             int lda, int ldb, int ldc, size_t sA,
+                                                             size_t sB, size_t sC) {
+  constexpr int BM = 64 * RM, BN = 48, BK = 16;
+  constexpr int ATILE = BM * BK, STAGE = ATILE + BK * BN;
+  extern __shared__ __align__(16) float tall_smem[];  // [stage][A: BM x 16 | B: 16 x 48]
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  A += (size_t)blockIdx.z * sA;
+  B += (size_t)blockIdx.z * sB;
+  C += (size_t)blockIdx.z * sC;
+  const int tid = threadIdx.x, tx = tid % 12, ty = tid / 12;
+  const int nslice = (K + BK - 1) / BK;
+  float acc[4 * RM][4];
+#pragma unroll
+  for (int i = 0; i < 4 * RM; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  auto issue = [&](int slice) {
+    if (slice < nslice) {
+      float* st = tall_smem + (slice % TALL_STAGES) * STAGE;
+      const int k0 = slice * BK;
+#pragma unroll
+      for (int i = 0; i < (BM * 4 + 191) / 192; ++i) {
+        const int e = tid + i * 192;  // vector e: row m = e / 4, vector c = e % 4 of the row
+        if (e < BM * 4) {
+          const int m = e >> 2, c = e & 3;
+          const bool ok = (m0 + m < M) && (k0 + c * 4 < K);
+          const float* src = ok ? A + (size_t)(m0 + m) * lda + k0 + c * 4 : A;
+          cp_async16(st + m * BK + ((c ^ ((m >> 2) & 3)) << 2), src, ok ? 16 : 0);
+        }
+      }
+      {
+        const int kr = tid / 12, cvn = (tid % 12) * 4;
+        const bool ok = (k0 + kr < K) && (n0 + cvn < N);
+        const float* src = ok ? B + (size_t)(k0 + kr) * ldb + n0 + cvn : B;
+        cp_async16(st + ATILE + kr * BN + cvn, src, ok ? 16 : 0);
+      }
+    }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int p = 0; p < TALL_STAGES - 1; ++p) issue(p);
+  const int sw = ty & 3;
+  for (int slice = 0; slice < nslice; ++slice) {
+    cp_async_wait<TALL_STAGES - 2>();
+    __syncthreads();
+    issue(slice + TALL_STAGES - 1);
+    const float* As = tall_smem + (slice % TALL_STAGES) * STAGE;
+    const float* Bs = As + ATILE;
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4) {
+      float4 bv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) bv[u] = *reinterpret_cast<const float4*>(Bs + (k4 * 4 + u) * BN + tx * 4);
+#pragma unroll
+      for (int g = 0; g < RM; ++g)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 av = *reinterpret_cast<const float4*>(As + (g * 64 + ty * 4 + i) * BK + ((k4 ^ sw) << 2));
+          const float a[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            acc[g * 4 + i][0] = fmaf(a[u], bv[u].x, acc[g * 4 + i][0]);
+            acc[g * 4 + i][1] = fmaf(a[u], bv[u].y, acc[g * 4 + i][1]);
+            acc[g * 4 + i][2] = fmaf(a[u], bv[u].z, acc[g * 4 + i][2]);
+            acc[g * 4 + i][3] = fmaf(a[u], bv[u].w, acc[g * 4 + i][3]);
+          }
+        }
+    }
+  }
+  cp_async_wait<0>();
+  const int gn = n0 + tx * 4;
+  if (gn >= N) return;
+#pragma unroll
+  for (int g = 0; g < RM; ++g)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int gm = m0 + g * 64 + ty * 4 + i;
+      if (gm < M)
+        *reinterpret_cast<float4*>(C + (size_t)gm * ldc + gn) =
+            make_float4(acc[g * 4 + i][0], acc[g * 4 + i][1], acc[g * 4 + i][2], acc[g * 4 + i][3]);
+    }
+}
+
 template <bool TRB>
 static bool gemm_tall(const float* A, const float* B, float* C, int M, int N, int K, int lda, int ldb,
                       int ldc, size_t sA, size_t sB, size_t sC, int batch, cudaStream_t st, int flags) {
@@ -359,6 +465,12 @@ static bool gemm_tall(const float* A, const float* B, float* C, int M, int N, in
   const bool three = ((M + 191) / 192) * 192 <= ((M + 127) / 128) * 128;
   if (three) {
     dim3 grid(N / 48, (M + 191) / 192, batch);
+    if (!TRB && !(flags & GEMM_B_UPPER)) {
+      const size_t smem = (size_t)TALL_STAGES * (192 * 16 + 16 * 48) * sizeof(float);
+      cudaFuncSetAttribute((const void*)gemm_tall_nn_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      { gemm_tall_nn_kernel<3><<<grid, 192, smem, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC); note_launch(); }
+      return true;
+    }
     { gemm_tall_kernel<TRB, 3><<<grid, 192, 0, st>>>(A, B, C, M, N, K, lda, ldb, ldc, sA, sB, sC, flags); note_launch(); }
   } else {
     dim3 grid(N / 48, (M + 127) / 128, batch);
@@ -403,19 +515,22 @@ static void gemm(const TA* A, const TB* B, float* C, int M, int N, int K, int ld
 // ==========================================================================================
 constexpr int TN_MAX = 144, TN_LD = 152, TN_PARTS = 4;
 
+constexpr int TN_STAGES = 4;  // slices in flight (asynchronous copies straight into shared memory)
+
 template <bool SAME>
 __global__ void __launch_bounds__(192) gemm_tn_upper_kernel(const float* __restrict__ A,
                                                            const float* __restrict__ B,
                                                            float* __restrict__ C, int n, int K,
                                                            int chunk, size_t sA, size_t sB,
                                                            size_t sC) {
-  __shared__ __align__(16) float As[16][TN_LD];
-  __shared__ __align__(16) float Bs[SAME ? 1 : 16][TN_LD];
+  extern __shared__ __align__(16) float tn_smem[];  // [stage][A, B][16][TN_LD]
+  constexpr int TILE = 16 * TN_LD, STAGE = (SAME ? 1 : 2) * TILE;
   const int tid = threadIdx.x, s = blockIdx.x, img = blockIdx.y;
   A += (size_t)img * sA;
   B += (size_t)img * sB;
   C += (size_t)img * sC + (size_t)s * n * n;
   const int k_lo = s * chunk, k_hi = min(K, k_lo + chunk);
+  const int nslice = (k_hi > k_lo) ? (k_hi - k_lo + 15) >> 4 : 0;
   const int nt = (n + 7) >> 3;  // tiles per side; the high half starts at column 4 nt
   const int half = 4 * nt;
   int ty = 0, rem = tid;
@@ -432,45 +547,44 @@ __global__ void __launch_bounds__(192) gemm_tn_upper_kernel(const float* __restr
   for (int i = 0; i < 8; ++i)
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-  float4 ra[3], rb[3];
-  auto fetch = [&](int k0) {
+  // this thread's (at most three) vectors of a slice: row kr[i] of the slice, vector cv[i]
+  int kr[3], cv[3];
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      const int e = tid + i * 192;
-      const int kr = e / nv, cv = e - kr * nv;
-      float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
-      if (e < nvec && k0 + kr < k_hi) {
-        va = __ldg(reinterpret_cast<const float4*>(A + (size_t)(k0 + kr) * n) + cv);
-        if (!SAME) vb = __ldg(reinterpret_cast<const float4*>(B + (size_t)(k0 + kr) * n) + cv);
-      }
-      ra[i] = va;
-      rb[i] = vb;
-    }
-  };
-  auto stash = [&]() {
+  for (int i = 0; i < 3; ++i) {
+    const int e = tid + i * 192;
+    kr[i] = (e < nvec) ? e / nv : -1;
+    cv[i] = (e < nvec) ? e - kr[i] * nv : 0;
+  }
+  auto issue = [&](int slice) {
+    if (slice < nslice) {
+      float* st = tn_smem + (slice % TN_STAGES) * STAGE;
+      const int k0 = k_lo + slice * 16;
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      const int e = tid + i * 192;
-      const int kr = e / nv, cv = e - kr * nv;
-      if (e < nvec) {
-        *reinterpret_cast<float4*>(&As[kr][cv * 4]) = ra[i];
-        if (!SAME) *reinterpret_cast<float4*>(&Bs[kr][cv * 4]) = rb[i];
+      for (int i = 0; i < 3; ++i) {
+        if (kr[i] < 0) continue;
+        const bool ok = k0 + kr[i] < k_hi;
+        const size_t off = (size_t)(ok ? k0 + kr[i] : k_lo) * n + cv[i] * 4;
+        cp_async16(st + kr[i] * TN_LD + cv[i] * 4, A + off, ok ? 16 : 0);
+        if (!SAME) cp_async16(st + TILE + kr[i] * TN_LD + cv[i] * 4, B + off, ok ? 16 : 0);
       }
     }
+    cp_async_commit();  // (an empty group keeps the count of groups in step with the slices)
   };
-  const float(*Bt)[TN_LD] = SAME ? As : Bs;
-  fetch(k_lo);
-  for (int k0 = k_lo; k0 < k_hi; k0 += 16) {
-    stash();
-    __syncthreads();
-    if (k0 + 16 < k_hi) fetch(k0 + 16);
+#pragma unroll
+  for (int p = 0; p < TN_STAGES - 1; ++p) issue(p);
+  for (int slice = 0; slice < nslice; ++slice) {
+    cp_async_wait<TN_STAGES - 2>();  // this thread's copies of `slice` have landed
+    __syncthreads();                 // everyone's have, and everyone is done with slice - 1
+    issue(slice + TN_STAGES - 1);    // into the buffer slice - 1 used
     if (active) {
+      const float* As = tn_smem + (slice % TN_STAGES) * STAGE;
+      const float* Bt = SAME ? As : As + TILE;
 #pragma unroll
       for (int kk = 0; kk < 16; ++kk) {
-        const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
-        const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][half + ty * 4]);
-        const float4 b0 = *reinterpret_cast<const float4*>(&Bt[kk][tx * 4]);
-        const float4 b1 = *reinterpret_cast<const float4*>(&Bt[kk][half + tx * 4]);
+        const float4 a0 = *reinterpret_cast<const float4*>(As + kk * TN_LD + ty * 4);
+        const float4 a1 = *reinterpret_cast<const float4*>(As + kk * TN_LD + half + ty * 4);
+        const float4 b0 = *reinterpret_cast<const float4*>(Bt + kk * TN_LD + tx * 4);
+        const float4 b1 = *reinterpret_cast<const float4*>(Bt + kk * TN_LD + half + tx * 4);
         const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
         const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
@@ -479,8 +593,8 @@ __global__ void __launch_bounds__(192) gemm_tn_upper_kernel(const float* __restr
           for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
       }
     }
-    __syncthreads();
   }
+  cp_async_wait<0>();
   if (!active) return;
   // every unordered pair {r, c} is produced by exactly one thread and written to both places
 #pragma unroll
@@ -515,10 +629,15 @@ static void gemm_tn_sym(const float* A, const float* B, float* C, int n, int K, 
   const int chunk = ((K + parts - 1) / parts + 15) / 16 * 16;
   dim3 grid(parts, batch);
   const size_t sC = (size_t)parts * n * n;
-  if (A == B)
-    { gemm_tn_upper_kernel<true><<<grid, 192, 0, st>>>(A, B, C, n, K, chunk, sA, sB, sC); note_launch(); }
-  else
-    { gemm_tn_upper_kernel<false><<<grid, 192, 0, st>>>(A, B, C, n, K, chunk, sA, sB, sC); note_launch(); }
+  if (A == B) {
+    const size_t smem = (size_t)TN_STAGES * 16 * TN_LD * sizeof(float);
+    cudaFuncSetAttribute((const void*)gemm_tn_upper_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    { gemm_tn_upper_kernel<true><<<grid, 192, smem, st>>>(A, B, C, n, K, chunk, sA, sB, sC); note_launch(); }
+  } else {
+    const size_t smem = (size_t)TN_STAGES * 2 * 16 * TN_LD * sizeof(float);
+    cudaFuncSetAttribute((const void*)gemm_tn_upper_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    { gemm_tn_upper_kernel<false><<<grid, 192, smem, st>>>(A, B, C, n, K, chunk, sA, sB, sC); note_launch(); }
+  }
 }
 
 // G = O O^T for float32 inputs (and, until the tensor-core kernel takes over, float16 ones).
