@@ -1050,6 +1050,255 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
 }
 
 // ==========================================================================================
+// The same job for k a multiple of 16, laid out so that no step waits on a chain of dependent
+// shared-memory reads and no warp reads a bank twice:
+//   * the warp that factors a diagonal block R_JJ also inverts it (reciprocal square roots are
+//     kept, nothing divides); D_J = R_JJ^{-1} then does the rest as products:
+//   * block row     R[J, c]  = D_J^T S[J, c]                 (512 threads: column x 4 outputs)
+//   * trailing      S[r, c] -= sum_i R[i, r] R[i, c]         (a warp owns 4 rows x 32-column
+//     blocks on or right of the diagonal; lanes run along columns; the 4 row entries come as
+//     one 16-byte read from an aligned copy P of the block row)
+//   * inverse       X[0:j0, J] = -X[0:j0, 0:j0] (R[0:j0, J] D_J), the inner product unrolled by
+//     four so that its reads are in flight together.
+// ==========================================================================================
+__global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restrict__ S,
+                                                           float* __restrict__ RinvT, int k,
+                                                           float shift_rel,
+                                                           int32_t* __restrict__ status,
+                                                           int nparts) {
+  extern __shared__ __align__(16) float fsm[];
+  __shared__ float s_red[16];
+  __shared__ float s_row[2][CNB];
+  __shared__ int s_bad;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ld = k | 1;
+  const int nblk = k / CNB;
+  const int PW = k;                       // row length of P (k is a multiple of 16)
+  float* P = fsm;                          // [16][PW] block row, later [<= k][16] the product T
+  float* Dinv = P + CNB * PW;              // [nblk][16][16] inverses of the diagonal blocks
+  float* A = Dinv + nblk * CNB * CNB;      // [k][ld]
+  const size_t kk = (size_t)k * k;
+  const float* Sb = S + (size_t)b * nparts * kk;  // S arrives as nparts parts to be added up
+
+  float md = 0.f;
+  for (int i = tid; i < k; i += 512) {
+    float dsum = 0.f;
+    for (int q = 0; q < nparts; ++q) dsum += __ldg(Sb + q * kk + (size_t)i * k + i);
+    md = fmaxf(md, dsum);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, o));
+  if (lane == 0) s_red[warp] = md;
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  md = s_red[0];
+  for (int w = 1; w < 16; ++w) md = fmaxf(md, s_red[w]);
+  const float shift = shift_rel * md;
+  const float tiny = fmaxf(md, 1e-30f) * 1e-12f;
+  {
+    const float4* S4 = reinterpret_cast<const float4*>(Sb);
+    const int kv = k >> 2, nv = (int)(kk >> 2);
+    for (int e = tid; e < nv; e += 512) {
+      float4 v = __ldg(S4 + e);
+      for (int q = 1; q < nparts; ++q) {
+        const float4 p = __ldg(S4 + (size_t)q * nv + e);
+        v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+      }
+      const int r = e / kv, c = (e - r * kv) * 4;
+      float* dst = A + r * ld + c;
+      dst[0] = v.x + (r == c ? shift : 0.f);
+      dst[1] = v.y + (r == c + 1 ? shift : 0.f);
+      dst[2] = v.z + (r == c + 2 ? shift : 0.f);
+      dst[3] = v.w + (r == c + 3 ? shift : 0.f);
+    }
+  }
+  __syncthreads();
+
+  // ---------------- phase 1: Cholesky, R^T R = S + shift I ----------------
+  for (int jb = 0; jb < nblk; ++jb) {
+    const int j0 = jb * CNB, j1 = j0 + CNB, m = k - j1;
+    float* Dj = Dinv + jb * CNB * CNB;
+    if (warp == 0) {
+      // lane c (< 16) keeps column c of the diagonal block
+      float col[CNB], rd[CNB];
+      const int gc = j0 + (lane & 15);
+#pragma unroll
+      for (int r = 0; r < CNB; ++r) col[r] = (r <= (lane & 15)) ? A[(j0 + r) * ld + gc] : 0.f;
+#pragma unroll
+      for (int i = 0; i < CNB; ++i) {
+        float piv = __shfl_sync(0xffffffffu, col[i], i);
+        if (!(piv > 0.f)) {
+          piv = tiny;
+          if (lane == 0) s_bad = 1;
+        }
+        const float rinv = rsqrtf(piv);
+        rd[i] = rinv;  // 1 / R_ii, the same in every lane
+        if ((lane & 15) == i) col[i] = piv * rinv;
+        else if ((lane & 15) > i) col[i] = col[i] * rinv;
+        if (lane < CNB) s_row[i & 1][lane] = col[i];
+        __syncwarp();
+#pragma unroll
+        for (int r = i + 1; r < CNB; ++r) {
+          const float v = s_row[i & 1][r];
+          if ((lane & 15) >= r) col[r] = fmaf(-v, col[i], col[r]);
+        }
+      }
+      if (lane < CNB) {
+#pragma unroll
+        for (int r = 0; r < CNB; ++r)
+          if (r <= lane) A[(j0 + r) * ld + gc] = col[r];
+      }
+      __syncwarp();
+      // lane c solves R_JJ x = e_c by back substitution: x_c = 1/R_cc,
+      // x_i = -(1/R_ii) sum_{i < mm <= c} R[i][mm] x_mm.  Row entries are broadcast reads.
+      float x[CNB];
+#pragma unroll
+      for (int i = 0; i < CNB; ++i) x[i] = 0.f;
+      const int c = lane & 15;
+#pragma unroll
+      for (int i = CNB - 1; i >= 0; --i) {
+        float sacc = 0.f;
+#pragma unroll
+        for (int mm = i + 1; mm < CNB; ++mm) sacc = fmaf(A[(j0 + i) * ld + j0 + mm], x[mm], sacc);
+        x[i] = (i == c) ? rd[i] : ((i < c) ? -rd[i] * sacc : 0.f);
+      }
+      if (lane < CNB) {
+#pragma unroll
+        for (int i = 0; i < CNB; ++i) Dj[i * CNB + c] = x[i];
+      }
+    }
+    __syncthreads();
+    // block row: R[j0 + i][c] = sum_{mm <= i} D[mm][i] S[j0 + mm][c] for c >= j1.
+    // thread = (column, group ig of four outputs i = 4 ig ..); 128 columns per pass.
+    for (int cb = 0; cb < m; cb += 128) {
+      const int cl = cb + (tid & 127), ig = tid >> 7;
+      const bool on = cl < m;
+      float a[CNB], out[4] = {0.f, 0.f, 0.f, 0.f};
+      if (on) {
+#pragma unroll
+        for (int mm = 0; mm < CNB; ++mm)
+          a[mm] = (mm <= 4 * ig + 3) ? A[(j0 + mm) * ld + j1 + cl] : 0.f;
+#pragma unroll
+        for (int mm = 0; mm < CNB; ++mm) {
+          if (mm <= 4 * ig + 3) {
+            const float4 d4 = *reinterpret_cast<const float4*>(Dj + mm * CNB + 4 * ig);
+            out[0] = fmaf(d4.x, a[mm], out[0]);
+            out[1] = fmaf(d4.y, a[mm], out[1]);
+            out[2] = fmaf(d4.z, a[mm], out[2]);
+            out[3] = fmaf(d4.w, a[mm], out[3]);
+          }
+        }
+      }
+      __syncthreads();  // every input of this pass has been read
+      if (on) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          A[(j0 + 4 * ig + u) * ld + j1 + cl] = out[u];
+          P[(4 * ig + u) * PW + cl] = out[u];
+        }
+      }
+    }
+    __syncthreads();
+    // trailing update of the upper triangle
+    for (int s4 = warp; s4 * 4 < m; s4 += 16) {
+      const int r0 = 4 * s4;  // rows j1 + r0 .. + 3
+      for (int u = r0 >> 5; u * 32 < m; ++u) {
+        const int cl = u * 32 + lane;
+        const bool on = cl < m;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int i = 0; i < CNB; ++i) {
+          const float4 a4 = *reinterpret_cast<const float4*>(P + i * PW + r0);
+          const float bv = on ? P[i * PW + cl] : 0.f;
+          acc[0] = fmaf(a4.x, bv, acc[0]);
+          acc[1] = fmaf(a4.y, bv, acc[1]);
+          acc[2] = fmaf(a4.z, bv, acc[2]);
+          acc[3] = fmaf(a4.w, bv, acc[3]);
+        }
+#pragma unroll
+        for (int xx = 0; xx < 4; ++xx)
+          if (on && r0 + xx < m && cl >= r0 + xx) A[(j1 + r0 + xx) * ld + j1 + cl] -= acc[xx];
+      }
+    }
+    __syncthreads();
+  }
+  if (tid == 0 && s_bad) atomicMax(&status[b], (int)TC_ERR_BREAKDOWN);
+
+  // ---------------- phase 2: X = R^{-1}, in place ----------------
+  float* TB = P;  // [j0][16]
+  for (int jb = 0; jb < nblk; ++jb) {
+    const int j0 = jb * CNB;
+    const float* Dj = Dinv + jb * CNB * CNB;
+    if (j0 > 0) {
+      // T = R[0:j0, J] D_J
+      for (int rb = 0; rb < j0; rb += 128) {
+        const int r = rb + (tid >> 2), cg = tid & 3;
+        if (r < j0) {
+          float out[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int mm = 0; mm < CNB; ++mm) {
+            const float rv = A[r * ld + j0 + mm];
+            const float4 d4 = *reinterpret_cast<const float4*>(Dj + mm * CNB + 4 * cg);
+            out[0] = fmaf(rv, d4.x, out[0]);
+            out[1] = fmaf(rv, d4.y, out[1]);
+            out[2] = fmaf(rv, d4.z, out[2]);
+            out[3] = fmaf(rv, d4.w, out[3]);
+          }
+          *reinterpret_cast<float4*>(TB + r * CNB + 4 * cg) = make_float4(out[0], out[1], out[2], out[3]);
+        }
+      }
+      __syncthreads();
+      // X[r][J] = - sum_{mm = r}^{j0 - 1} X[r][mm] T[mm][:]
+      for (int rb = 0; rb < j0; rb += 128) {
+        const int r = rb + (tid >> 2), cg = tid & 3;
+        if (r < j0) {
+          float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
+          const float* xr = A + r * ld;
+          const float* tb = TB + 4 * cg;
+          int mm = r;
+          for (; mm + 3 < j0; mm += 4) {
+            const float x0 = xr[mm], x1 = xr[mm + 1], x2 = xr[mm + 2], x3 = xr[mm + 3];
+            const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
+            const float4 t1 = *reinterpret_cast<const float4*>(tb + (mm + 1) * CNB);
+            const float4 t2 = *reinterpret_cast<const float4*>(tb + (mm + 2) * CNB);
+            const float4 t3 = *reinterpret_cast<const float4*>(tb + (mm + 3) * CNB);
+            o0[0] = fmaf(x0, t0.x, o0[0]); o0[1] = fmaf(x0, t0.y, o0[1]);
+            o0[2] = fmaf(x0, t0.z, o0[2]); o0[3] = fmaf(x0, t0.w, o0[3]);
+            o1[0] = fmaf(x1, t1.x, o1[0]); o1[1] = fmaf(x1, t1.y, o1[1]);
+            o1[2] = fmaf(x1, t1.z, o1[2]); o1[3] = fmaf(x1, t1.w, o1[3]);
+            o0[0] = fmaf(x2, t2.x, o0[0]); o0[1] = fmaf(x2, t2.y, o0[1]);
+            o0[2] = fmaf(x2, t2.z, o0[2]); o0[3] = fmaf(x2, t2.w, o0[3]);
+            o1[0] = fmaf(x3, t3.x, o1[0]); o1[1] = fmaf(x3, t3.y, o1[1]);
+            o1[2] = fmaf(x3, t3.z, o1[2]); o1[3] = fmaf(x3, t3.w, o1[3]);
+          }
+          for (; mm < j0; ++mm) {
+            const float x0 = xr[mm];
+            const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
+            o0[0] = fmaf(x0, t0.x, o0[0]); o0[1] = fmaf(x0, t0.y, o0[1]);
+            o0[2] = fmaf(x0, t0.z, o0[2]); o0[3] = fmaf(x0, t0.w, o0[3]);
+          }
+          // columns J of A are not read in this step: the results can go straight in
+#pragma unroll
+          for (int u = 0; u < 4; ++u) A[r * ld + j0 + 4 * cg + u] = -(o0[u] + o1[u]);
+        }
+      }
+    }
+    // X_JJ = D_J
+    if (tid < CNB * CNB) {
+      const int i = tid >> 4, c = tid & 15;
+      A[(j0 + i) * ld + j0 + c] = Dj[i * CNB + c];
+    }
+    __syncthreads();
+  }
+  // RinvT[c][m] = X[m][c] for m <= c, zero otherwise
+  float* out = RinvT + b * kk;
+  for (int e = tid; e < (int)kk; e += 512) {
+    const int c = e / k, mrow = e - c * k;
+    out[e] = (mrow <= c) ? A[mrow * ld + c] : 0.f;
+  }
+}
+
+// ==========================================================================================
 // One-sided Jacobi eigen-solver for a symmetric positive semi-definite n x n matrix.
 // One block (16 warps) per image.  W (column-major) starts as the matrix, J as the identity;
 // each pair step rotates columns p, q of both so that the W columns become orthogonal.  At
@@ -1922,6 +2171,12 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
 static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
                             float shift_rel, int32_t* status, cudaStream_t st, int nparts) {
   Scope scope_(KC_CHOL, st);
+  const size_t fast = ((size_t)k * (k | 1) + (size_t)CNB * k + (size_t)(k / CNB) * CNB * CNB) * sizeof(float);
+  if (k % CNB == 0 && k >= CNB && fast <= SMEM_LIMIT) {
+    cudaFuncSetAttribute((const void*)chol_inv_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast);
+    { chol_inv_fast_kernel<<<batch, 512, fast, st>>>(S, RinvT, k, shift_rel, status, nparts); note_launch(); }
+    return;
+  }
   const size_t blocked = (size_t)k * (k | 1) * sizeof(float);
   // (the blocked kernel keeps 2 x 4 outputs per thread in registers in its last step)
   if (blocked <= SMEM_LIMIT && (size_t)k * (CNB / 4) <= 2 * 512) {
