@@ -1061,11 +1061,15 @@ __global__ void __launch_bounds__(512) chol_inv_blocked_kernel(const float* __re
 //   * inverse       X[0:j0, J] = -X[0:j0, 0:j0] (R[0:j0, J] D_J), the inner product unrolled by
 //     four so that its reads are in flight together.
 // ==========================================================================================
+// KT = k when it is known at compile time (every shared-memory address then folds into an
+// immediate offset, which halves the instruction count), 0 for any k.
+template <int KT>
 __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restrict__ S,
-                                                           float* __restrict__ RinvT, int k,
+                                                           float* __restrict__ RinvT, int k_rt,
                                                            float shift_rel,
                                                            int32_t* __restrict__ status,
                                                            int nparts) {
+  const int k = KT ? KT : k_rt;
   extern __shared__ __align__(16) float fsm[];
   __shared__ float s_red[16];
   __shared__ float s_row[2][CNB];
@@ -1096,20 +1100,42 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
   const float shift = shift_rel * md;
   const float tiny = fmaxf(md, 1e-30f) * 1e-12f;
   {
+    // parts are added in the order 0, 1, 2, 3; two trips' worth of loads are in flight together
     const float4* S4 = reinterpret_cast<const float4*>(Sb);
     const int kv = k >> 2, nv = (int)(kk >> 2);
-    for (int e = tid; e < nv; e += 512) {
-      float4 v = __ldg(S4 + e);
-      for (int q = 1; q < nparts; ++q) {
-        const float4 p = __ldg(S4 + (size_t)q * nv + e);
-        v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-      }
+    auto put = [&](int e, const float4& v) {
       const int r = e / kv, c = (e - r * kv) * 4;
       float* dst = A + r * ld + c;
       dst[0] = v.x + (r == c ? shift : 0.f);
       dst[1] = v.y + (r == c + 1 ? shift : 0.f);
       dst[2] = v.z + (r == c + 2 ? shift : 0.f);
       dst[3] = v.w + (r == c + 3 ? shift : 0.f);
+    };
+    if (nparts == 4) {
+      for (int e = tid; e < nv; e += 1024) {
+        const int e2 = e + 512;
+        const bool two = e2 < nv;
+        float4 p[4], q[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          p[i] = __ldg(S4 + (size_t)i * nv + e);
+          q[i] = two ? __ldg(S4 + (size_t)i * nv + e2) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        put(e, make_float4(((p[0].x + p[1].x) + p[2].x) + p[3].x, ((p[0].y + p[1].y) + p[2].y) + p[3].y,
+                           ((p[0].z + p[1].z) + p[2].z) + p[3].z, ((p[0].w + p[1].w) + p[2].w) + p[3].w));
+        if (two)
+          put(e2, make_float4(((q[0].x + q[1].x) + q[2].x) + q[3].x, ((q[0].y + q[1].y) + q[2].y) + q[3].y,
+                              ((q[0].z + q[1].z) + q[2].z) + q[3].z, ((q[0].w + q[1].w) + q[2].w) + q[3].w));
+      }
+    } else {
+      for (int e = tid; e < nv; e += 512) {
+        float4 v = __ldg(S4 + e);
+        for (int q = 1; q < nparts; ++q) {
+          const float4 pp = __ldg(S4 + (size_t)q * nv + e);
+          v.x += pp.x; v.y += pp.y; v.z += pp.z; v.w += pp.w;
+        }
+        put(e, v);
+      }
     }
   }
   __syncthreads();
@@ -1476,13 +1502,15 @@ __device__ __forceinline__ void bar_named(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
+template <int NT>  // n when it is known at compile time (addresses fold into immediates), else 0
 __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ ZTg,
-                                                         float* __restrict__ theta, int n, float rank_tol,
+                                                         float* __restrict__ theta, int n_rt, float rank_tol,
                                                          float* __restrict__ u0g, float* __restrict__ u1g,
                                                          float* __restrict__ u2g, float* yg, float* __restrict__ mlg,
                                                          size_t ml_stride,
                                                          int32_t* __restrict__ status, int nparts) {
+  const int n = NT ? NT : n_rt;
   extern __shared__ __align__(16) float sm[];
   const int ld = n | 1;
   const int n4 = (n + 3) & ~3;         // the vectors start on 16-byte boundaries
@@ -1506,15 +1534,31 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     // same bits, so their sum is symmetric as it stands
     const float4* H4 = reinterpret_cast<const float4*>(Hb);
     const int kv = n >> 2, nv = (n * n) >> 2;
-    for (int e = tid; e < nv; e += 512) {
-      const float4 p0 = __ldg(H4 + e), p1 = __ldg(H4 + nv + e), p2 = __ldg(H4 + 2 * nv + e),
-                   p3 = __ldg(H4 + 3 * nv + e);
-      const int r = e / kv, c = (e - r * kv) * 4;
-      float* dst = A + r * ld + c;
-      dst[0] = (p0.x + p1.x) + (p2.x + p3.x);
-      dst[1] = (p0.y + p1.y) + (p2.y + p3.y);
-      dst[2] = (p0.z + p1.z) + (p2.z + p3.z);
-      dst[3] = (p0.w + p1.w) + (p2.w + p3.w);
+    for (int e = tid; e < nv; e += 1024) {  // two trips' worth of loads in flight together
+      const int e2 = e + 512;
+      const bool two = e2 < nv;
+      float4 p[4], q[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        p[i] = __ldg(H4 + (size_t)i * nv + e);
+        q[i] = two ? __ldg(H4 + (size_t)i * nv + e2) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      {
+        const int r = e / kv, c = (e - r * kv) * 4;
+        float* dst = A + r * ld + c;
+        dst[0] = (p[0].x + p[1].x) + (p[2].x + p[3].x);
+        dst[1] = (p[0].y + p[1].y) + (p[2].y + p[3].y);
+        dst[2] = (p[0].z + p[1].z) + (p[2].z + p[3].z);
+        dst[3] = (p[0].w + p[1].w) + (p[2].w + p[3].w);
+      }
+      if (two) {
+        const int r = e2 / kv, c = (e2 - r * kv) * 4;
+        float* dst = A + r * ld + c;
+        dst[0] = (q[0].x + q[1].x) + (q[2].x + q[3].x);
+        dst[1] = (q[0].y + q[1].y) + (q[2].y + q[3].y);
+        dst[2] = (q[0].z + q[1].z) + (q[2].z + q[3].z);
+        dst[3] = (q[0].w + q[1].w) + (q[2].w + q[3].w);
+      }
     }
   } else {
     for (int e = tid; e < n * n; e += 512) {
@@ -2147,8 +2191,17 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
   {
     const size_t tri = ((size_t)n * (n | 1) + 27 * (size_t)((n + 3) & ~3)) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
-      cudaFuncSetAttribute((const void*)tridiag_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
-      { tridiag_eig_kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts); note_launch(); }
+      auto go = [&](auto kernel) {
+        cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
+        { kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts); note_launch(); }
+      };
+      switch (n) {
+        case 128: go(tridiag_eig_kernel<128>); break;
+        case 144: go(tridiag_eig_kernel<144>); break;
+        case 160: go(tridiag_eig_kernel<160>); break;
+        case 192: go(tridiag_eig_kernel<192>); break;
+        default: go(tridiag_eig_kernel<0>); break;
+      }
       return;
     }
   }
@@ -2173,8 +2226,17 @@ static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, i
   Scope scope_(KC_CHOL, st);
   const size_t fast = ((size_t)k * (k | 1) + (size_t)CNB * k + (size_t)(k / CNB) * CNB * CNB) * sizeof(float);
   if (k % CNB == 0 && k >= CNB && fast <= SMEM_LIMIT) {
-    cudaFuncSetAttribute((const void*)chol_inv_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast);
-    { chol_inv_fast_kernel<<<batch, 512, fast, st>>>(S, RinvT, k, shift_rel, status, nparts); note_launch(); }
+    auto go = [&](auto kernel) {
+      cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast);
+      { kernel<<<batch, 512, fast, st>>>(S, RinvT, k, shift_rel, status, nparts); note_launch(); }
+    };
+    switch (k) {
+      case 128: go(chol_inv_fast_kernel<128>); break;
+      case 144: go(chol_inv_fast_kernel<144>); break;
+      case 160: go(chol_inv_fast_kernel<160>); break;
+      case 192: go(chol_inv_fast_kernel<192>); break;
+      default: go(chol_inv_fast_kernel<0>); break;
+    }
     return;
   }
   const size_t blocked = (size_t)k * (k | 1) * sizeof(float);
