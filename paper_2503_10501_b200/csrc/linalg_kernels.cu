@@ -2267,24 +2267,27 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
                                                  int32_t* __restrict__ rank_out,
                                                  int32_t* __restrict__ status, int N, int k, int q,
                                                  float rank_tol, int full) {
+  // grid (token chunks of 256, images): every block ranks the k singular values again (k^2
+  // comparisons, cheap) and sums Eq. 3-6 for its own tokens; chunk 0 writes sigma and the rank.
   extern __shared__ float sig[];  // [k] sigma, then [k] weights (sigma or 0)
   float* wgt = sig + k;
-  __shared__ float s_red[256];
-  __shared__ int s_cnt[256];
-  const int b = blockIdx.x, tid = threadIdx.x;
+  __shared__ float s_red[8];
+  __shared__ int s_cnt[8];
+  const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool writer = blockIdx.x == 0;
   float mx = 0.f;
   for (int p = tid; p < k; p += 256) {
     const float s = sqrtf(fmaxf(theta[(size_t)b * k + p], 0.f));
     sig[p] = s;
     mx = fmaxf(mx, s);
   }
-  s_red[tid] = mx;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) s_red[warp] = mx;
   __syncthreads();
-  for (int s = 128; s > 0; s >>= 1) {
-    if (tid < s) s_red[tid] = fmaxf(s_red[tid], s_red[tid + s]);
-    __syncthreads();
-  }
-  const float smax = s_red[0];
+  float smax = s_red[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) smax = fmaxf(smax, s_red[w]);
   const float cut = rank_tol * smax;
   // O has at most q = min(N, d) non-zero singular values: only the q largest eigenvalues of G
   // can be one, whatever rounding left in the others.
@@ -2296,28 +2299,34 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
     const bool on = (s > cut) && (pos < q);
     wgt[p] = on ? s : 0.f;
     cnt += on;
-    if (sigma_sorted && pos < q) sigma_sorted[(size_t)b * q + pos] = s;
+    if (writer && sigma_sorted && pos < q) sigma_sorted[(size_t)b * q + pos] = s;
   }
-  if (sigma_sorted)
+  if (writer && sigma_sorted)
     for (int p = k + tid; p < q; p += 256) sigma_sorted[(size_t)b * q + p] = 0.f;
-  s_cnt[tid] = cnt;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if (lane == 0) s_cnt[warp] = cnt;
   __syncthreads();
-  for (int s = 128; s > 0; s >>= 1) {
-    if (tid < s) s_cnt[tid] += s_cnt[tid + s];
-    __syncthreads();
-  }
-  const int r = s_cnt[0];
-  if (tid == 0) {
+  if (writer && tid == 0) {
+    int r = 0;
+    for (int w = 0; w < 8; ++w) r += s_cnt[w];
     if (rank_out) rank_out[b] = r;
     if (!full && r > k - 8) atomicMax(&status[b], (int)TC_ERR_RANK_CAP);
   }
   const float* PTb = PT + (size_t)b * k * N;
-  for (int x = tid; x < N; x += 256) {
+  const int x = blockIdx.x * 256 + tid;
+  if (x < N) {
+    // terms in the order p = 0, 1, ...; eight loads in flight
     float acc = 0.f;
-    for (int p = 0; p < k; ++p) {
-      const float w = wgt[p];
-      if (w != 0.f) acc = fmaf(fabsf(PTb[(size_t)p * N + x]), w, acc);
+    int p = 0;
+    for (; p + 7 < k; p += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = PTb[(size_t)(p + u) * N + x];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc = fmaf(fabsf(v[u]), wgt[p + u], acc);
     }
+    for (; p < k; ++p) acc = fmaf(fabsf(PTb[(size_t)p * N + x]), wgt[p], acc);
     C[(size_t)b * N + x] = acc;
   }
 }
@@ -2350,8 +2359,8 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   if (D.full) {
     launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, nullptr, nullptr, nullptr, nullptr, 0, img_status, st);
     Scope scope_(KC_ICS, st);
-    { ics_kernel<<<B, 256, 2 * (size_t)N * sizeof(float), st>>>(theta, ZT, C_out, sigma_out, rank_out,
-                                                             img_status, N, N, q, D.rank_tol, 1); note_launch(); }
+    { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)N * sizeof(float), st>>>(
+          theta, ZT, C_out, sigma_out, rank_out, img_status, N, N, q, D.rank_tol, 1); note_launch(); }
     return;
   }
   float* Y0 = (float*)(ws + P.Y0) + b0 * sY;
@@ -2408,8 +2417,8 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]
   gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
   Scope scope_(KC_ICS, st);
-  { ics_kernel<<<B, 256, 2 * (size_t)k * sizeof(float), st>>>(theta, Y0, C_out, sigma_out, rank_out,
-                                                           img_status, N, k, q, D.rank_tol, 0); note_launch(); }
+  { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
+        theta, Y0, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0); note_launch(); }
 }
 
 }  // namespace tc

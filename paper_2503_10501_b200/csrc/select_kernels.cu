@@ -42,9 +42,12 @@ __device__ int block_excl_scan(int v, int* sh /* >= 9 ints */, int* total) {
 }
 
 // k-th largest key (k in 1..n) of keys[0..n): returns the key value `thr` and how many of the
-// keys equal to thr belong to the top k (`need_eq` >= 1).  MSB-first, 8 bits per pass.
+// keys equal to thr belong to the top k (`need_eq` >= 1).  MSB-first, 8 bits per pass; the bin
+// that holds the k-th key is found by a block-wide scan of the histogram from the top bin down
+// (thread t holds bin 255 - t), not by one thread walking it.
 __device__ void block_select_kth(const uint32_t* keys, int n, int kth, int* hist /*256*/,
-                                 uint32_t* sh_u /*2*/, uint32_t* thr, int* need_eq) {
+                                 uint32_t* sh_u /*2*/, int* sh_scan /*9*/, uint32_t* thr,
+                                 int* need_eq) {
   uint32_t prefix = 0, mask = 0;
   int remaining = kth;
   for (int shift = 24; shift >= 0; shift -= 8) {
@@ -55,14 +58,12 @@ __device__ void block_select_kth(const uint32_t* keys, int n, int kth, int* hist
       if ((kx & mask) == prefix) atomicAdd(&hist[(kx >> shift) & 255u], 1);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int acc = 0, bin = 255;
-      for (; bin > 0; --bin) {
-        if (acc + hist[bin] >= remaining) break;
-        acc += hist[bin];
-      }
-      sh_u[0] = (uint32_t)bin;
-      sh_u[1] = (uint32_t)(remaining - acc);
+    const int mine = hist[255 - threadIdx.x];
+    int tot;
+    const int above = block_excl_scan(mine, sh_scan, &tot);  // keys in higher bins
+    if (above < remaining && above + mine >= remaining) {      // exactly one thread
+      sh_u[0] = 255u - threadIdx.x;
+      sh_u[1] = (uint32_t)(remaining - above);
     }
     __syncthreads();
     prefix |= sh_u[0] << shift;
@@ -90,8 +91,8 @@ __global__ void __launch_bounds__(SEL_THREADS) prune_kernel(const float* __restr
   __syncthreads();
   uint32_t thrP, thrA = 0xffffffffu;
   int needP, needA = 0;
-  block_select_kth(keys, N, P, hist, sh_u, &thrP, &needP);
-  if (nA > 0) block_select_kth(keys, N, nA, hist, sh_u, &thrA, &needA);
+  block_select_kth(keys, N, P, hist, sh_u, sh_scan, &thrP, &needP);
+  if (nA > 0) block_select_kth(keys, N, nA, hist, sh_u, sh_scan, &thrA, &needA);
 
   const int chunk = (N + SEL_THREADS - 1) / SEL_THREADS;
   const int i0 = min(N, (int)threadIdx.x * chunk), i1 = min(N, i0 + chunk);
@@ -295,7 +296,7 @@ __global__ void __launch_bounds__(SEL_THREADS) merge_select_kernel(
   for (int j = threadIdx.x; j < nA; j += SEL_THREADS) flag[setA[(size_t)b * nA + j]] = 1;
   uint32_t thr = 0xffffffffu;
   int need = 0;
-  if (M > 0) block_select_kth(keys, nB, M, hist, sh_u, &thr, &need);
+  if (M > 0) block_select_kth(keys, nB, M, hist, sh_u, sh_scan, &thr, &need);
 
   int tot;
   {
