@@ -579,12 +579,20 @@ __global__ void __launch_bounds__(192) gemm_tn_upper_kernel(const float* __restr
     if (active) {
       const float* As = tn_smem + (slice % TN_STAGES) * STAGE;
       const float* Bt = SAME ? As : As + TILE;
+      // the operands of step kk + 1 are read before the multiply-adds of step kk are issued
+      float4 na0 = *reinterpret_cast<const float4*>(As + ty * 4);
+      float4 na1 = *reinterpret_cast<const float4*>(As + half + ty * 4);
+      float4 nb0 = *reinterpret_cast<const float4*>(Bt + tx * 4);
+      float4 nb1 = *reinterpret_cast<const float4*>(Bt + half + tx * 4);
 #pragma unroll
       for (int kk = 0; kk < 16; ++kk) {
-        const float4 a0 = *reinterpret_cast<const float4*>(As + kk * TN_LD + ty * 4);
-        const float4 a1 = *reinterpret_cast<const float4*>(As + kk * TN_LD + half + ty * 4);
-        const float4 b0 = *reinterpret_cast<const float4*>(Bt + kk * TN_LD + tx * 4);
-        const float4 b1 = *reinterpret_cast<const float4*>(Bt + kk * TN_LD + half + tx * 4);
+        const float4 a0 = na0, a1 = na1, b0 = nb0, b1 = nb1;
+        if (kk + 1 < 16) {
+          na0 = *reinterpret_cast<const float4*>(As + (kk + 1) * TN_LD + ty * 4);
+          na1 = *reinterpret_cast<const float4*>(As + (kk + 1) * TN_LD + half + ty * 4);
+          nb0 = *reinterpret_cast<const float4*>(Bt + (kk + 1) * TN_LD + tx * 4);
+          nb1 = *reinterpret_cast<const float4*>(Bt + (kk + 1) * TN_LD + half + tx * 4);
+        }
         const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
         const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
