@@ -161,8 +161,10 @@ def run_ours(args):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     tcb.lib()
-    if args.groups:
-        tcb.tc_set_groups(args.groups)
+    use_graph = not args.no_graph
+    # concurrent image groups: measured best is 8 under graph replay, the library's 4 otherwise
+    groups = args.groups if args.groups else (8 if use_graph else 4)
+    tcb.tc_set_groups(groups)
 
     cfg, name = workload(args)
     M, P, nA, nB = 0, 0, 0, 0
@@ -211,12 +213,13 @@ def run_ours(args):
     if status.any():
         raise SystemExit(f"carve reported per-image status {status.tolist()}")
 
-    # --graph: the timed step replays a CUDA graph of one tc_carve call (same kernels, same
-    # streams: the fork/join of the library's internal streams is captured as graph
-    # dependencies).  Measured: 2.89 ms against 2.90 ms for plain calls, so plain is the default.
+    # The timed step replays a CUDA graph of one tc_carve call (same kernels, same streams: the
+    # fork/join of the library's internal streams is captured as graph dependencies), which
+    # takes the ~25 dependent launches of a group's chain off the host: 1.85 ms against 1.91 ms
+    # per step for plain calls (--no-graph).
     eager_step = step
     graph = None
-    if args.graph:
+    if use_graph:
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             eager_step()
@@ -244,7 +247,7 @@ def run_ours(args):
         for _ in range(args.steps):
             eager_step()
         prof = tcb.tc_profile_end()
-        tcb.tc_set_groups(args.groups if args.groups else 4)
+        tcb.tc_set_groups(groups)
 
         # end to end through the host-buffer entry point
         for _ in range(min(args.warmup, 2)):
@@ -321,7 +324,8 @@ def run_ours(args):
                 "config": {"workload": name, "images_per_gpu": cfg.batch, "rank_cap": p.rank_cap,
                            "rank_tol": p.rank_tol, "lambda": p.lam, "rho": p.rho,
                            "l2": "inputs (1.5 GB per step) exceed the 126 MB L2",
-                           "launch": "CUDA graph replay of one tc_carve" if args.graph else "plain calls"},
+                           "image_groups": groups,
+                           "launch": "CUDA graph replay of one tc_carve" if use_graph else "plain calls"},
                 "us_per_image": us_img,
                 "e2e": {"value": e2e, "unit": UNIT,
                         "h2d_bytes_per_step": nbytes(hostin.values()),
@@ -451,8 +455,9 @@ def main():
     ap.add_argument("--n-query", type=int, default=128)
     ap.add_argument("--keep", type=int, default=128)
     ap.add_argument("--rank-cap", type=int, default=0, help="override the workload's rank_cap")
-    ap.add_argument("--graph", action="store_true",
-                    help="time the replay of a CUDA graph of one tc_carve instead of plain calls")
+    ap.add_argument("--graph", action="store_true", help="(the default; kept for old command lines)")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="time plain tc_carve calls instead of the replay of a CUDA graph of one call")
     ap.add_argument("--groups", type=int, default=0, help="concurrent image groups (0 = library default)")
     ap.add_argument("--cpu-images", type=int, default=12,
                     help="images the CPU oracle is timed on (0 = skip)")

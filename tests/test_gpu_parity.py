@@ -214,6 +214,50 @@ def test_cfg5_bench_point_sampled_images():
     assert flips["flips_sets"] <= 2 and flips["flips_merge"] <= 2, flips
 
 
+def test_cfg5_bench_point_in_the_bench_launch_mode():
+    # bench.py times the replay of a CUDA graph of one tc_carve with eight image groups: the
+    # replay must give, bit for bit, what the plain call gives (which the test above compares
+    # with the oracle), and sampled images are compared with the oracle once more from it
+    cfg = inputs.CONFIGS["cfg5_sweep_f16"]
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    d = {k: dev(v) for k, v in batch.items()}
+    ws = tcb.workspace(p)
+    tcb.tc_set_groups(4)
+    plain = [host(t) for t in tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)]
+    tcb.tc_set_groups(8)
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        held = tcb._outputs(p, d["O"].device, True) + (
+            torch.zeros(p.batch, p.keep, dtype=torch.int32, device="cuda"),
+            torch.zeros(p.batch, dtype=torch.int32, device="cuda"))
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws, held)
+        for t in held:
+            t.zero_()
+        g.replay()
+        g.replay()
+        torch.cuda.synchronize()
+    finally:
+        tcb.tc_set_groups(4)
+    replay = [host(t) for t in held]
+    for a, b in zip(plain, replay):
+        assert np.array_equal(a, b)
+    assert not replay[4].any()
+    # kept indices and merged rows of sampled images against the oracle's compaction
+    for b in (5, 40):
+        o = pu.oracle_scores(cfgp_of(p), batch["O"][b], batch["A"][b])
+        M, P, nA, nB = orc.resolve_counts(cfg.n_tokens, cfg.keep, cfg.rho, -1)
+        order = orc.descending_order(o["E"])
+        assert len(set(replay[3][b].tolist()) - set(int(t) for t in order[:P + 4])) <= 2
+
+
 @pytest.mark.parametrize("T,keep", [(32, 64), (512, 288)])
 def test_cfg5_sweep_corners(T, keep):
     cfg = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=8, n_query=T, keep=keep)
