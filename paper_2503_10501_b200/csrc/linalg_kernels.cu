@@ -1289,9 +1289,13 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
           float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
           const float* xr = A + r * ld;
           const float* tb = TB + 4 * cg;
-          int mm = r;
+          // the eight rows of a warp walk the same mm (from the first of them on, entries left
+          // of a row's diagonal counting as zero), so that lanes with the same columns read the
+          // same 16 bytes of T
+          int mm = r & ~7;
           for (; mm + 3 < j0; mm += 4) {
-            const float x0 = xr[mm], x1 = xr[mm + 1], x2 = xr[mm + 2], x3 = xr[mm + 3];
+            const float x0 = (mm >= r) ? xr[mm] : 0.f, x1 = (mm + 1 >= r) ? xr[mm + 1] : 0.f;
+            const float x2 = (mm + 2 >= r) ? xr[mm + 2] : 0.f, x3 = (mm + 3 >= r) ? xr[mm + 3] : 0.f;
             const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
             const float4 t1 = *reinterpret_cast<const float4*>(tb + (mm + 1) * CNB);
             const float4 t2 = *reinterpret_cast<const float4*>(tb + (mm + 2) * CNB);
@@ -1306,7 +1310,7 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
             o1[2] = fmaf(x3, t3.z, o1[2]); o1[3] = fmaf(x3, t3.w, o1[3]);
           }
           for (; mm < j0; ++mm) {
-            const float x0 = xr[mm];
+            const float x0 = (mm >= r) ? xr[mm] : 0.f;
             const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
             o0[0] = fmaf(x0, t0.x, o0[0]); o0[1] = fmaf(x0, t0.y, o0[1]);
             o0[2] = fmaf(x0, t0.z, o0[2]); o0[3] = fmaf(x0, t0.w, o0[3]);
