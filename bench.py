@@ -197,14 +197,17 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def timed(fn, steps):
+        """Milliseconds for `steps` calls between one pair of events (max over ranks), and this
+        rank's per-step times from an event after every call."""
         barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ev[0].record()
+        for i in range(steps):
             fn()
-        e1.record()
+            ev[i + 1].record()
         barrier()
-        return sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        return sharding.max_over_ranks(ev[0].elapsed_time(ev[steps]), device="cuda"), per
 
     for _ in range(args.warmup):
         step()
@@ -234,7 +237,7 @@ def run_ours(args):
     # nvidia-smi is sampled (every 0.2 s) over the timed region and the two passes after it,
     # which run the same kernels: one timed region alone is shorter than a sampling period
     with ClockSampler(local) as cs:
-        ms = timed(step, args.steps)
+        ms, per_step = timed(step, args.steps)
         launches0 = tcb.tc_launch_count()
         eager_step()
         launches = (tcb.tc_launch_count() - launches0) * args.steps  # same kernels per step
@@ -252,7 +255,7 @@ def run_ours(args):
         # end to end through the host-buffer entry point
         for _ in range(min(args.warmup, 2)):
             step_host()
-        ms_host = timed(step_host, args.steps)
+        ms_host, _ = timed(step_host, args.steps)
     clocks = cs.summary()
 
     images = cfg.batch * world * args.steps
@@ -327,6 +330,7 @@ def run_ours(args):
                            "image_groups": groups,
                            "launch": "CUDA graph replay of one tc_carve" if use_graph else "plain calls"},
                 "us_per_image": us_img,
+                "ms_per_step_median": float(np.median(per_step)), "ms_per_step_min": float(min(per_step)),
                 "e2e": {"value": e2e, "unit": UNIT,
                         "h2d_bytes_per_step": nbytes(hostin.values()),
                         "d2h_bytes_per_step": nbytes(hout)},
@@ -448,7 +452,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=64, help="images per GPU per step")

@@ -165,8 +165,17 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
   const float* pb = part + (size_t)b * chunks * N;
   float ls = 0.f, lc = 0.f;
   for (int x = threadIdx.x; x < N; x += 256) {
+    // chunk partials are added in chunk order, eight loads in flight at a time
     float s = 0.f;
-    for (int c = 0; c < chunks; ++c) s += pb[(size_t)c * N + x];
+    int c = 0;
+    for (; c + 7 < chunks; c += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = pb[(size_t)(c + u) * N + x];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) s += v[u];
+    }
+    for (; c < chunks; ++c) s += pb[(size_t)c * N + x];
     s *= inv_rows;
     S[(size_t)b * N + x] = s;
     ls += s;

@@ -153,10 +153,10 @@ def test_merge_duplicate_rows_tie_to_lower_index():
 
 
 # ------------------------------------------------------------------ the named workloads
-def test_cfg1_single_f32():
+@pytest.mark.parametrize("lam,norm", [(0.5, "none"), (0.5, "sum1"), (0.0, "none"), (1.0, "none")])
+def test_cfg1_single_f32(lam, norm):
     cfg = inputs.CONFIGS["cfg1_single_f32"]
-    check_config(cfg, [0])
-    check_config(cfg, [0], score_norm="sum1")
+    check_config(cfg, [0], lam=lam, score_norm=norm)
 
 
 @pytest.mark.parametrize("lam,norm", [(0.5, "none"), (0.5, "sum1"), (0.0, "none"), (1.0, "none")])
@@ -212,6 +212,8 @@ def test_cfg5_bench_point_sampled_images():
     cfg = inputs.CONFIGS["cfg5_sweep_f16"]
     flips = check_config(cfg, [0, 31, 63])
     assert flips["flips_sets"] <= 2 and flips["flips_merge"] <= 2, flips
+    flips = check_config(cfg, [17, 50], score_norm="sum1")
+    assert flips["flips_sets"] <= 2 and flips["flips_merge"] <= 2, flips
 
 
 def test_cfg5_bench_point_in_the_bench_launch_mode():
@@ -264,9 +266,10 @@ def test_cfg5_sweep_corners(T, keep):
     check_config(cfg, [0, 7])
 
 
-def test_cfg4_anyres():
+@pytest.mark.parametrize("norm,image", [("none", 2), ("sum1", 1)])
+def test_cfg4_anyres(norm, image):
     cfg = inputs.CONFIGS["cfg4_anyres_f16"]
-    check_config(cfg, [2])
+    check_config(cfg, [image], score_norm=norm)
 
 
 # ------------------------------------------------------------------ launch modes
