@@ -283,8 +283,8 @@ def run_ours(args):
         "eig": cfg.batch * (14.0 / 3.0) * k ** 3,
         "chol_inv": cfg.batch * (2.0 / 3.0) * k ** 3,
         "gemm_f32_GQ": cfg.batch * 2.0 * N * N * k,
-        "gemm_f32_YtY": cfg.batch * 2.0 * N * k * k,
-        "gemm_f32_YRinv": cfg.batch * 2.0 * N * k * k,
+        "gemm_f32_YtY": cfg.batch * 1.0 * N * k * (k + 1),  # symmetric: upper triangle only
+        "gemm_f32_YRinv": cfg.batch * 2.0 * N * k * k * 11.0 / 15.0,
     }
     if top_name in flops_per_launch:
         roof = {"kernel": top_name, "bound": "alu", "achieved": flops_per_launch[top_name] / per_launch_s / 1e12,
@@ -357,8 +357,10 @@ def kernel_fractions(cfg, P, k, prof, steps, pk):
         "compact": (B * (P + cfg.keep) * (d + 2 * H * dh) * e, pk["hbm_gbs"] * 1e9, "hbm"),
         "gram": (B * 2.0 * N * N * d, pk["bf16_tflops_sustained"] * 1e12, "tensor"),
         "gemm_f32_GQ": (B * 2.0 * N * N * k, alu_peak, "alu"),
-        "gemm_f32_YtY": (B * 2.0 * N * k * k, alu_peak, "alu"),
-        "gemm_f32_YRinv": (B * 2.0 * N * k * k, alu_peak, "alu"),
+        "gemm_f32_YtY": (B * 1.0 * N * k * (k + 1), alu_peak, "alu"),  # symmetric: upper triangle only
+        # five launches per step: four Y R^-1 that skip the zero part of R^-1 (2/3 of the work
+        # with three 48-column tiles) and one Z Q1^T: 11/15 of a full product on average
+        "gemm_f32_YRinv": (B * 2.0 * N * k * k * 11.0 / 15.0, alu_peak, "alu"),
         "chol_inv": (B * (2.0 / 3.0) * k ** 3, alu_peak, "alu"),
         "eig": (B * (14.0 / 3.0) * k ** 3, alu_peak, "alu"),
     }
