@@ -95,9 +95,11 @@ tc_status make_dims(const tc_params* p, Dims* out) {
   D.lambda = p->lambda;
   D.rank_tol = p->rank_tol;
   D.score_norm = p->score_norm;
-  // row chunks of the attention reduction: enough blocks to fill the GPU, at least 32 rows each
+  // row chunks of the attention reduction: sixteen blocks per SM when the rows allow it (the
+  // blocks are not all the same length, so many short ones balance better than a few long
+  // ones), at least 32 rows each
   const int R = D.H * D.T;
-  int chunks = (4 * 148 + D.B - 1) / D.B;
+  int chunks = (16 * 148 + D.B - 1) / D.B;
   if (chunks > R / 32) chunks = R / 32;
   if (chunks > 64) chunks = 64;
   if (chunks < 1) chunks = 1;

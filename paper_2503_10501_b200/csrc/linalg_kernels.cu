@@ -700,12 +700,12 @@ __global__ void sketch_vec_kernel(const T* __restrict__ O, float* __restrict__ Y
 #pragma unroll
   for (int i = 0; i < L; ++i) acc[i] = 0.f;
   int g = tx;
-  for (; g + 3 * kg < ng; g += 4 * kg) {
-    uint4 v[4];
+  for (; g + 7 * kg < ng; g += 8 * kg) {  // eight 16-byte loads in flight per thread
+    uint4 v[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = __ldg(row + g + u * kg);
+    for (int u = 0; u < 8; ++u) v[u] = __ldg(row + g + u * kg);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < 8; ++u) {
       const T* e = reinterpret_cast<const T*>(&v[u]);
       const float* sg = sgn + (size_t)(g + u * kg) * L;
 #pragma unroll
@@ -1149,59 +1149,83 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
   __syncthreads();
 
   // ---------------- phase 1: Cholesky, R^T R = S + shift I ----------------
+  // One warp factors and inverts a diagonal block; so that the others need not wait for it, the
+  // trailing update of a block column first brings the rows of the next diagonal block up to
+  // date, and that block is then factored while the rest of the update runs.
+  auto diag = [&](int jb) {
+    const int j0 = jb * CNB;
+    float* Dj = Dinv + jb * CNB * CNB;
+    // lane c (< 16) keeps column c of the diagonal block
+    float col[CNB], rd[CNB];
+    const int gc = j0 + (lane & 15);
+#pragma unroll
+    for (int r = 0; r < CNB; ++r) col[r] = (r <= (lane & 15)) ? A[(j0 + r) * ld + gc] : 0.f;
+#pragma unroll
+    for (int i = 0; i < CNB; ++i) {
+      float piv = __shfl_sync(0xffffffffu, col[i], i);
+      if (!(piv > 0.f)) {
+        piv = tiny;
+        if (lane == 0) s_bad = 1;
+      }
+      const float rinv = rsqrtf(piv);
+      rd[i] = rinv;  // 1 / R_ii, the same in every lane
+      if ((lane & 15) == i) col[i] = piv * rinv;
+      else if ((lane & 15) > i) col[i] = col[i] * rinv;
+      if (lane < CNB) s_row[i & 1][lane] = col[i];
+      __syncwarp();
+#pragma unroll
+      for (int r = i + 1; r < CNB; ++r) {
+        const float v = s_row[i & 1][r];
+        if ((lane & 15) >= r) col[r] = fmaf(-v, col[i], col[r]);
+      }
+    }
+    if (lane < CNB) {
+#pragma unroll
+      for (int r = 0; r < CNB; ++r)
+        if (r <= lane) A[(j0 + r) * ld + gc] = col[r];
+    }
+    __syncwarp();
+    // lane c solves R_JJ x = e_c by back substitution: x_c = 1/R_cc,
+    // x_i = -(1/R_ii) sum_{i < mm <= c} R[i][mm] x_mm.  Row entries are broadcast reads.
+    float x[CNB];
+#pragma unroll
+    for (int i = 0; i < CNB; ++i) x[i] = 0.f;
+    const int c = lane & 15;
+#pragma unroll
+    for (int i = CNB - 1; i >= 0; --i) {
+      float sacc = 0.f;
+#pragma unroll
+      for (int mm = i + 1; mm < CNB; ++mm) sacc = fmaf(A[(j0 + i) * ld + j0 + mm], x[mm], sacc);
+      x[i] = (i == c) ? rd[i] : ((i < c) ? -rd[i] * sacc : 0.f);
+    }
+    if (lane < CNB) {
+#pragma unroll
+      for (int i = 0; i < CNB; ++i) Dj[i * CNB + c] = x[i];
+    }
+  };
+  // one 4-row x 32-column unit of the trailing update of block column jb (P = its block row)
+  auto trail_unit = [&](int j1, int m, int r0, int u) {
+    const int cl = u * 32 + lane;
+    const bool on = cl < m;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < CNB; ++i) {
+      const float4 a4 = *reinterpret_cast<const float4*>(P + i * PW + r0);
+      const float bv = on ? P[i * PW + cl] : 0.f;
+      acc[0] = fmaf(a4.x, bv, acc[0]);
+      acc[1] = fmaf(a4.y, bv, acc[1]);
+      acc[2] = fmaf(a4.z, bv, acc[2]);
+      acc[3] = fmaf(a4.w, bv, acc[3]);
+    }
+#pragma unroll
+    for (int xx = 0; xx < 4; ++xx)
+      if (on && r0 + xx < m && cl >= r0 + xx) A[(j1 + r0 + xx) * ld + j1 + cl] -= acc[xx];
+  };
+  if (warp == 0) diag(0);
+  __syncthreads();
   for (int jb = 0; jb < nblk; ++jb) {
     const int j0 = jb * CNB, j1 = j0 + CNB, m = k - j1;
     float* Dj = Dinv + jb * CNB * CNB;
-    if (warp == 0) {
-      // lane c (< 16) keeps column c of the diagonal block
-      float col[CNB], rd[CNB];
-      const int gc = j0 + (lane & 15);
-#pragma unroll
-      for (int r = 0; r < CNB; ++r) col[r] = (r <= (lane & 15)) ? A[(j0 + r) * ld + gc] : 0.f;
-#pragma unroll
-      for (int i = 0; i < CNB; ++i) {
-        float piv = __shfl_sync(0xffffffffu, col[i], i);
-        if (!(piv > 0.f)) {
-          piv = tiny;
-          if (lane == 0) s_bad = 1;
-        }
-        const float rinv = rsqrtf(piv);
-        rd[i] = rinv;  // 1 / R_ii, the same in every lane
-        if ((lane & 15) == i) col[i] = piv * rinv;
-        else if ((lane & 15) > i) col[i] = col[i] * rinv;
-        if (lane < CNB) s_row[i & 1][lane] = col[i];
-        __syncwarp();
-#pragma unroll
-        for (int r = i + 1; r < CNB; ++r) {
-          const float v = s_row[i & 1][r];
-          if ((lane & 15) >= r) col[r] = fmaf(-v, col[i], col[r]);
-        }
-      }
-      if (lane < CNB) {
-#pragma unroll
-        for (int r = 0; r < CNB; ++r)
-          if (r <= lane) A[(j0 + r) * ld + gc] = col[r];
-      }
-      __syncwarp();
-      // lane c solves R_JJ x = e_c by back substitution: x_c = 1/R_cc,
-      // x_i = -(1/R_ii) sum_{i < mm <= c} R[i][mm] x_mm.  Row entries are broadcast reads.
-      float x[CNB];
-#pragma unroll
-      for (int i = 0; i < CNB; ++i) x[i] = 0.f;
-      const int c = lane & 15;
-#pragma unroll
-      for (int i = CNB - 1; i >= 0; --i) {
-        float sacc = 0.f;
-#pragma unroll
-        for (int mm = i + 1; mm < CNB; ++mm) sacc = fmaf(A[(j0 + i) * ld + j0 + mm], x[mm], sacc);
-        x[i] = (i == c) ? rd[i] : ((i < c) ? -rd[i] * sacc : 0.f);
-      }
-      if (lane < CNB) {
-#pragma unroll
-        for (int i = 0; i < CNB; ++i) Dj[i * CNB + c] = x[i];
-      }
-    }
-    __syncthreads();
     // block row: R[j0 + i][c] = sum_{mm <= i} D[mm][i] S[j0 + mm][c] for c >= j1.
     // thread = (column, group ig of four outputs i = 4 ig ..); 128 columns per pass.
     for (int cb = 0; cb < m; cb += 128) {
@@ -1233,26 +1257,21 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
       }
     }
     __syncthreads();
-    // trailing update of the upper triangle
-    for (int s4 = warp; s4 * 4 < m; s4 += 16) {
-      const int r0 = 4 * s4;  // rows j1 + r0 .. + 3
-      for (int u = r0 >> 5; u * 32 < m; ++u) {
-        const int cl = u * 32 + lane;
-        const bool on = cl < m;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int i = 0; i < CNB; ++i) {
-          const float4 a4 = *reinterpret_cast<const float4*>(P + i * PW + r0);
-          const float bv = on ? P[i * PW + cl] : 0.f;
-          acc[0] = fmaf(a4.x, bv, acc[0]);
-          acc[1] = fmaf(a4.y, bv, acc[1]);
-          acc[2] = fmaf(a4.z, bv, acc[2]);
-          acc[3] = fmaf(a4.w, bv, acc[3]);
-        }
-#pragma unroll
-        for (int xx = 0; xx < 4; ++xx)
-          if (on && r0 + xx < m && cl >= r0 + xx) A[(j1 + r0 + xx) * ld + j1 + cl] -= acc[xx];
+    // trailing update, first the rows of the next diagonal block (four strips of four rows)
+    {
+      const int nu = (m + 31) >> 5;
+      const int n_first = min(4, m >> 2) * nu;
+      for (int id = warp; id < n_first; id += 16) {
+        const int s4 = id / nu, u = id - s4 * nu;
+        if (u >= ((4 * s4) >> 5)) trail_unit(j1, m, 4 * s4, u);
       }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      if (jb + 1 < nblk) diag(jb + 1);
+    } else {
+      for (int s4 = 4 + (warp - 1); s4 * 4 < m; s4 += 15)
+        for (int u = (4 * s4) >> 5; u * 32 < m; ++u) trail_unit(j1, m, 4 * s4, u);
     }
     __syncthreads();
   }

@@ -60,6 +60,15 @@ extern "C" tc_status tc_attn_score_noalloc(const tc_params* p, const void* A, fl
   tc_status s = make_dims(p, &D);
   if (s != TC_OK) return s;
   if (A == nullptr || S == nullptr || ((uintptr_t)A & 15u) != 0) return TC_ERR_INVALID_ARG;
+  // this entry point keeps its own, smaller chunk count: its scratch is fixed in size
+  {
+    const int R = D.H * D.T;
+    int chunks = (4 * 148 + D.B - 1) / D.B;
+    if (chunks > R / 32) chunks = R / 32;
+    if (chunks > 64) chunks = 64;
+    if (chunks < 1) chunks = 1;
+    D.chunks = chunks;
+  }
   const size_t need = (size_t)D.B * D.chunks * D.N;
   if (need > kScratchFloats) return TC_ERR_SCRATCH_LIMIT;
   float* scratch = nullptr;
