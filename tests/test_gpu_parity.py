@@ -116,6 +116,15 @@ def test_medium_ragged(rank_cap):
     check_config(cfg, range(5), rank_cap=rank_cap)
 
 
+def test_maximum_token_count():
+    # N = 4096 is the most the selection kernels take (16 tokens per thread); a subspace size
+    # that none of the kernels is specialised for, and fewer attention rows than one chunk
+    cfg = inputs.tiny_config(n_tokens=4096, d_model=256, n_heads=2, head_dim=64, n_query=8,
+                             keep=512, rank=48, dtype="f16", batch=1, seed=31, noise=0.01, tau=2.0,
+                             rank_tol=2e-3)
+    check_config(cfg, [0], rank_cap=64)
+
+
 # ------------------------------------------------------------------ selection kernels alone
 def test_prune_exact_with_ties():
     rng = np.random.default_rng(3)

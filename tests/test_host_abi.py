@@ -44,10 +44,17 @@ def test_bad_arguments_are_rejected_on_the_host():
     for kw, code in [(dict(keep=0), 1), (dict(keep=577), 1), (dict(lam=1.5), 1), (dict(rho=-0.1), 1),
                      (dict(n_tokens=5000, keep=10), 2), (dict(d_model=4100, dtype="f16"), 2),
                      (dict(rank_cap=-1), 1), (dict(rank_cap=4), 1), (dict(n_tokens=2880, keep=640), 2),
-                     (dict(batch=0), 1)]:
+                     (dict(batch=0), 1),
+                     # one past the largest token count and the largest subspace
+                     (dict(n_tokens=4097, keep=10, rank_cap=64), 2),
+                     (dict(n_tokens=4096, keep=10, rank_cap=1025), 2)]:
         with pytest.raises(tcb.TokenCarveError) as e:
             tcb.tc_workspace_bytes(_params(**kw))
         assert e.value.status == code, kw
+
+
+def test_largest_supported_shape_is_accepted():
+    assert tcb.tc_workspace_bytes(_params(n_tokens=4096, keep=10, rank_cap=1024)) > 0
 
 
 def test_workspace_grows_with_batch_and_host_variant_adds_staging():
