@@ -10,7 +10,11 @@ the paper itself names (an SVD, a matrix product, a sort); there is no blocking,
 fusion or reordering.  A LAPACK-free one-sided Jacobi SVD (`svd_jacobi`) is kept
 beside the LAPACK call so each can check the other.
 
-Paper passages followed (TokenCarve, Sec. 3.3):
+Paper passages followed (TokenCarve, Sec. 3.3; Sec. 3.2 for `token_information`):
+  Sec. 3.2    the information quantity of the visual tokens is measured by the
+              matrix rank of their rows of the attention-output matrix, followed
+              as tokens are removed (Visual Token Information curve; appendix
+              "Attention Output Matrix Rank").
   Sec. 3.3.1  Z = U Sigma V^T; row expansion Eq. 3-5; information contribution
               score Eq. 3-6; attention score Eq. 3-7; combined score Eq. 3-8;
               Stage I keeps L_vc (1 + rho) tokens.
@@ -147,6 +151,17 @@ def numerical_rank(sigma: np.ndarray, rank_tol: float) -> int:
     if sigma.size == 0 or sigma[0] <= 0.0:
         return 0
     return int(np.sum(sigma > F64(np.float32(rank_tol)) * sigma[0]))
+
+
+def token_information(O: np.ndarray, idx: Optional[Sequence[int]], rank_tol: float,
+                      method: str = "lapack") -> Tuple[np.ndarray, int]:
+    """Information quantity of a set of visual tokens (Sec. 3.2, "Visual Token Information";
+    appendix "Attention Output Matrix Rank"): the matrix rank of the rows of the attention
+    output that belong to the tokens `idx` (all rows when idx is None), taken as the numerical
+    rank #{sigma_i > rank_tol * sigma_1}.  Returns (sigma descending [min(n, d)], rank)."""
+    rows = np.asarray(O, F64) if idx is None else np.asarray(O, F64)[np.asarray(list(idx), int)]
+    _, sigma = svd_lapack(rows) if method == "lapack" else svd_jacobi(rows)
+    return sigma, numerical_rank(sigma, rank_tol)
 
 
 # --------------------------------------------------------------------------

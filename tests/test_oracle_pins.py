@@ -424,3 +424,38 @@ def test_carve_tiny_against_independent_brute_force():
         for j, a in enumerate(kept):
             grp = [a] + [b for b in chosen if best[b][1] == a]
             np.testing.assert_allclose(res["Xo"][j], X[grp].sum(0) / len(grp), atol=1e-13)
+
+
+# ------------------------------------------------------------------ Sec. 3.2: rank of a token set
+def test_token_information_closed_forms():
+    rng = np.random.default_rng(5)
+    # mutually orthogonal rows: every subset of n rows has rank n and its sigma are the row norms
+    Q, _ = np.linalg.qr(rng.standard_normal((12, 12)))
+    norms = np.arange(1.0, 13.0)
+    O = Q * norms[:, None]
+    for idx in ([0, 3, 7], [11, 2], list(range(12))):
+        sig, r = orc.token_information(O, idx, 1e-6)
+        assert r == len(idx)
+        assert np.allclose(sig[:len(idx)], sorted(norms[idx], reverse=True), rtol=1e-12)
+    # both SVD routes
+    assert np.allclose(orc.token_information(O, [1, 4, 9], 0.0, "jacobi")[0],
+                       orc.token_information(O, [1, 4, 9], 0.0, "lapack")[0], rtol=1e-10)
+    # a copy of a row adds no rank; a row outside the span adds one
+    L = rng.standard_normal((9, 4)) @ rng.standard_normal((4, 30))      # rank 4
+    assert orc.token_information(L, None, 1e-9)[1] == 4
+    assert orc.token_information(np.vstack([L, L[2:3]]), None, 1e-9)[1] == 4
+    assert orc.token_information(np.vstack([L, rng.standard_normal((1, 30))]), None, 1e-9)[1] == 5
+    # fewer rows than the rank: the rank is the row count; removing rows never raises it
+    assert orc.token_information(L, [0, 5, 8], 1e-9)[1] == 3
+    ranks = [orc.token_information(L, list(range(n)), 1e-9)[1] for n in range(9, 0, -1)]
+    assert all(a >= b for a, b in zip(ranks, ranks[1:])) and ranks[-1] == 1
+    # order of the token list and scaling of O do not matter; rank_tol cuts relative to sigma_1
+    s1, r1 = orc.token_information(L, [1, 6, 3, 8], 1e-9)
+    s2, r2 = orc.token_information(7.0 * L, [8, 3, 6, 1], 1e-9)
+    assert r1 == r2 and np.allclose(7.0 * s1, s2, rtol=1e-12)
+    D = np.diag([10.0, 1.0, 0.1, 0.01])
+    assert [orc.token_information(D, None, t)[1] for t in (0.5, 0.05, 0.005, 0.0)] == [1, 2, 3, 4]
+    # sum of squares of sigma = squared Frobenius norm of the chosen rows
+    sig, _ = orc.token_information(L, [0, 2, 4, 6], 0.0)
+    assert np.isclose(np.sum(sig ** 2), np.sum(L[[0, 2, 4, 6]] ** 2), rtol=1e-12)
+
