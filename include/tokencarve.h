@@ -192,6 +192,31 @@ tc_status tc_attn_score_noalloc(const tc_params* p, const void* A, float* S, voi
 tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream);
 
 /*
+ * Sec. 3.2 ("Visual Token Information") and the appendix "Attention Output Matrix Rank": the
+ * information quantity of a set of visual tokens is the matrix rank of their rows of the
+ * attention-output matrix, followed as tokens are removed.  For every image b, the singular
+ * values of the n_sub x d matrix made of the rows idx[b][0..n_sub) of O and its numerical rank
+ * #{sigma_i > rank_tol * sigma_1}, from the same Gram and eigen kernels as tc_score (rank_cap
+ * applies as there: 0 = full solve, otherwise a bound on the rank, checked on the device).
+ *   p        describes O ([batch, n_tokens, d_model], dtype) and rank_tol, rank_cap, max_sweeps;
+ *            keep, n_merge, rho, lambda, score_norm are not used
+ *   O        device, [B, N, d]
+ *   idx      device, [B, n_sub] int32, distinct token numbers in [0, N) in any order (the
+ *            result does not depend on the order); NULL = all rows, n_sub must then be N.  A
+ *            number outside [0, N) gives TC_ERR_INVALID_ARG in that image's status, never a fault
+ *   sigma    device, [B, min(n_sub, d)] float32 out, descending; may be NULL
+ *   rank     device, [B] int32 out
+ *   img_status  device, [B] int32 out, as in tc_score
+ *   ws       device scratch of tc_rank_workspace_bytes(p, n_sub) bytes, 16-byte aligned, owned by
+ *            the caller; nothing is allocated.  Asynchronous on `stream`.
+ * Returns TC_ERR_INVALID_ARG / TC_ERR_UNSUPPORTED / TC_ERR_WORKSPACE with nothing enqueued.
+ */
+tc_status tc_rank_workspace_bytes(const tc_params* p, int32_t n_sub, size_t* bytes);
+tc_status tc_rank(const tc_params* p, const void* O, const int32_t* idx, int32_t n_sub,
+                  float* sigma, int32_t* rank, int32_t* img_status, void* ws, size_t ws_bytes,
+                  void* stream);
+
+/*
  * Number of image groups tc_score / tc_carve run side by side (1..8, default 4; the paper has no
  * counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
  * chains are enqueued on internal streams forked from `stream` and joined back into it before

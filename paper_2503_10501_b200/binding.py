@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "TC_OK", 1: "TC_ERR_INVALID_ARG", 2: "TC_ERR_UNSUPPORTED", 3:
 EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge", "tc_compact",
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
-           "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups")
+           "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
+           "tc_rank_workspace_bytes")
 
 
 class TcParams(C.Structure):
@@ -70,6 +71,8 @@ def lib() -> C.CDLL:
         L.tc_compact.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
         L.tc_carve.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_carve_host.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
+        L.tc_rank_workspace_bytes.argtypes = [pp, C.c_int32, C.POINTER(sz)]
+        L.tc_rank.argtypes = [pp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         L.tc_gram.argtypes = [pp, vp, vp, vp]
         L.tc_set_groups.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
@@ -191,6 +194,29 @@ def tc_score(p: Params, O, A, ws=None) -> Dict[str, torch.Tensor]:
     _check("tc_score", lib().tc_score(C.byref(cp), _ptr(O), _ptr(A), _ptr(out["E"]), _ptr(out["C"]),
                                       _ptr(out["S"]), _ptr(out["sigma"]), _ptr(out["rank"]),
                                       _ptr(out["img_status"]), _ptr(ws), ws.numel(), _stream()))
+    return out
+
+
+def tc_rank_workspace_bytes(p: Params, n_sub: int) -> int:
+    n = C.c_size_t()
+    cp = p.c()
+    _check("tc_rank_workspace_bytes", lib().tc_rank_workspace_bytes(C.byref(cp), n_sub, C.byref(n)))
+    return n.value
+
+
+def tc_rank(p: Params, O, idx=None, ws=None) -> Dict[str, torch.Tensor]:
+    """sigma [B, min(n_sub, d)], rank [B], img_status [B] of the rows idx [B, n_sub] of O."""
+    dev = O.device
+    n_sub = p.n_tokens if idx is None else int(idx.shape[1])
+    if ws is None:
+        ws = torch.empty(tc_rank_workspace_bytes(p, n_sub), dtype=torch.uint8, device=dev)
+    out = {"sigma": torch.empty(p.batch, min(n_sub, p.d_model), dtype=torch.float32, device=dev),
+           "rank": torch.empty(p.batch, dtype=torch.int32, device=dev),
+           "img_status": torch.empty(p.batch, dtype=torch.int32, device=dev)}
+    cp = p.c()
+    _check("tc_rank", lib().tc_rank(C.byref(cp), _ptr(O), _ptr(idx), n_sub, _ptr(out["sigma"]),
+                                    _ptr(out["rank"]), _ptr(out["img_status"]), _ptr(ws), ws.numel(),
+                                    _stream()))
     return out
 
 

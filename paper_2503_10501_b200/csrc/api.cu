@@ -530,6 +530,64 @@ tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream) {
   return check_launch();
 }
 
+// ---- Sec. 3.2: information quantity (numerical rank) of a set of tokens -----------------------
+// The score path's own Gram and eigen kernels on the gathered rows.
+// beyond the score path's own plan: the gathered rows, and four n x n arrays per image for the
+// tridiagonal solver when the full problem is small enough for it
+static size_t rank_rows_bytes(const Dims& D) { return align_up((size_t)D.B * D.N * D.d * D.esz, 256); }
+static bool rank_small_full(const Dims& D) { return D.full && D.N <= 224; }
+static size_t rank_extra_bytes(const Dims& D) {
+  return rank_rows_bytes(D) + (rank_small_full(D) ? 4 * (size_t)D.B * D.N * D.N * sizeof(float) : 0);
+}
+
+static tc_status rank_dims(const tc_params* p, int32_t n_sub, Dims* full, Dims* sub) {
+  if (p == nullptr) return TC_ERR_INVALID_ARG;
+  tc_params pf = *p;  // the carve counts play no part here
+  pf.keep = 1;
+  pf.n_merge = 0;
+  tc_status s = make_dims(&pf, full);
+  if (s != TC_OK) return s;
+  if (n_sub < 1 || n_sub > full->N) return TC_ERR_INVALID_ARG;
+  pf.n_tokens = n_sub;
+  return make_dims(&pf, sub);
+}
+
+tc_status tc_rank_workspace_bytes(const tc_params* p, int32_t n_sub, size_t* bytes) {
+  Dims F, D;
+  tc_status s = rank_dims(p, n_sub, &F, &D);
+  if (s != TC_OK) return s;
+  if (bytes == nullptr) return TC_ERR_INVALID_ARG;
+  const Plan P = make_plan(D);
+  *bytes = align_up(P.total, 256) + rank_extra_bytes(D);
+  return TC_OK;
+}
+
+tc_status tc_rank(const tc_params* p, const void* O, const int32_t* idx, int32_t n_sub,
+                  float* sigma, int32_t* rank, int32_t* img_status, void* ws, size_t ws_bytes,
+                  void* stream) {
+  Dims F, D;
+  tc_status s = rank_dims(p, n_sub, &F, &D);
+  if (s != TC_OK) return s;
+  if (!O || !rank || !img_status || !ws || misaligned(O) || misaligned(ws)) return TC_ERR_INVALID_ARG;
+  if (idx == nullptr && n_sub != F.N) return TC_ERR_INVALID_ARG;
+  const Plan P = make_plan(D);
+  const size_t rows_off = align_up(P.total, 256);
+  if (ws_bytes < rows_off + rank_extra_bytes(D)) return TC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w = (char*)ws;
+  fill_i32(img_status, D.B, 0, st);
+  const void* rows = O;
+  if (idx != nullptr) {
+    launch_gather_rows(F, n_sub, O, idx, w + rows_off, img_status, st);
+    rows = w + rows_off;
+  }
+  s = launch_gram(D, rows, (float*)(w + P.G), img_status, st);
+  if (s != TC_OK) return s;
+  launch_ics(D, P, w, 0, rows, (float*)(w + P.C), sigma, rank, img_status, st,
+             rank_small_full(D) ? (float*)(w + rows_off + rank_rows_bytes(D)) : nullptr);
+  return check_launch();
+}
+
 const char* tc_status_string(int32_t status) {
   switch (status) {
     case TC_OK: return "ok";

@@ -2376,7 +2376,8 @@ void fill_i32(int32_t* p, int n, int v, cudaStream_t st) {
 // The whole of Eq. 3-5 / 3-6 for a batch, given G in the workspace.
 // ==========================================================================================
 void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
-                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st) {
+                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
+                float* full_scratch) {
   // D.B images starting at image b0 of the workspace arrays; O and the outputs already point at
   // image b0.
   const int B = D.B, N = D.N, k = D.k;
@@ -2388,7 +2389,13 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   float* theta = (float*)(ws + P.sigma) + (size_t)b0 * k;
 
   if (D.full) {
-    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, nullptr, nullptr, nullptr, nullptr, 0, img_status, st);
+    // with scratch for it (four N x N arrays per image) the tridiagonal solver takes the full
+    // problem when it fits in shared memory: it has no sweeps that a spectrum without a gap at
+    // the rounding level could keep alive
+    float* fs = full_scratch;
+    launch_jacobi(G, W, ZT, theta, N, B, D.max_sweeps, D.rank_tol, fs, fs ? fs + (size_t)B * sG : nullptr,
+                  fs ? fs + 2 * (size_t)B * sG : nullptr, fs ? fs + 3 * (size_t)B * sG : nullptr, sG,
+                  img_status, st);
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)N * sizeof(float), st>>>(
           theta, ZT, C_out, sigma_out, rank_out, img_status, N, N, q, D.rank_tol, 1); note_launch(); }

@@ -299,4 +299,32 @@ void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
                                                     D.H, D.dh, D.keep, D.M); note_launch(); }
 }
 
+// ------------------------------------------------------------------------------------------
+// Rows idx[b][0..n_sub) of O [B, N, d] copied to Os [B, n_sub, d] (Sec. 3.2: the rows of the
+// attention output that belong to a set of tokens).  grid (n_sub, B); 16-byte vectors.  An
+// index outside [0, N) gives a zero row and TC_ERR_INVALID_ARG in the image's status.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) gather_rows_kernel(const uint4* __restrict__ O,
+                                                         const int32_t* __restrict__ idx,
+                                                         uint4* __restrict__ Os, int N, int n_sub,
+                                                         int vec_per_row,
+                                                         int32_t* __restrict__ status) {
+  const int b = blockIdx.y, j = blockIdx.x;
+  const int t = idx[(size_t)b * n_sub + j];
+  const bool ok = t >= 0 && t < N;
+  if (!ok && threadIdx.x == 0) atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+  const uint4* src = O + ((size_t)b * N + (ok ? t : 0)) * vec_per_row;
+  uint4* dst = Os + ((size_t)b * n_sub + j) * vec_per_row;
+  for (int v = threadIdx.x; v < vec_per_row; v += 128)
+    dst[v] = ok ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
+}
+
+void launch_gather_rows(const Dims& D, int n_sub, const void* O, const int32_t* idx, void* Os,
+                        int32_t* status, cudaStream_t st) {
+  Scope scope_(KC_COMPACT, st);
+  dim3 grid(n_sub, D.B);
+  { gather_rows_kernel<<<grid, 128, 0, st>>>((const uint4*)O, idx, (uint4*)Os, D.N, n_sub,
+                                            D.d * D.esz / 16, status); note_launch(); }
+}
+
 }  // namespace tc

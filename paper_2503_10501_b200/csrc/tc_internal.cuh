@@ -87,11 +87,19 @@ void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
                     const int32_t* kept, const int32_t* msrc, const int32_t* mdst, void* Xo,
                     void* Ko, void* Vo, cudaStream_t st);
 
+// Sec. 3.2: rows idx[b][0..n_sub) of O gathered into Os [B, n_sub, d] (D describes O).
+void launch_gather_rows(const Dims& D, int n_sub, const void* O, const int32_t* idx, void* Os,
+                        int32_t* status, cudaStream_t st);
+void fill_i32(int32_t* p, int n, int v, cudaStream_t st);
+
 // G = O O^T (float32 out).
 tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 
 // Eigen-decomposition of G and Eq. 3-6:  C, theta (unsorted), then sorted sigma / rank.
+// full_scratch: optional 4 * B * N * N floats; with it a full solve (rank_cap = 0) of a matrix
+// that fits in shared memory goes through the tridiagonal solver instead of Jacobi sweeps.
 void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
-                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st);
+                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
+                float* full_scratch = nullptr);
 
 }  // namespace tc

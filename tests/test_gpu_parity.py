@@ -281,6 +281,53 @@ def test_cfg4_anyres(norm, image):
     check_config(cfg, [image], score_norm=norm)
 
 
+# ------------------------------------------------------------------ Sec. 3.2: rank of a token set
+def test_token_information_against_oracle():
+    # the rank curve of Sec. 3.2 on one workload: all tokens, the tokens a carve keeps, a random
+    # half, a handful (fewer rows than the rank), in shuffled order
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=3)
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    O = dev(batch["O"])
+    kept = host(tcb.tc_carve(p, O, dev(batch["A"]), dev(batch["X"]), dev(batch["K"]), dev(batch["V"]))[3])
+    rng = np.random.default_rng(3)
+    sets = {"all": None, "kept": kept,
+            "half": np.stack([rng.permutation(cfg.n_tokens)[:288] for _ in range(3)]).astype(np.int32),
+            "few": np.stack([rng.permutation(cfg.n_tokens)[:40] for _ in range(3)]).astype(np.int32)}
+    # A token set's spectrum has no gap where rank_tol cuts, unlike the carve workloads', so the
+    # comparison is the one float32 eigenvalues of a Gram matrix allow: sigma^2 within 4e-6 of
+    # sigma_1^2 (the Gram entries carry ~2e-6 relative error), and the rank anywhere between the
+    # counts that this band leaves open at the cut.
+    pr = params_of(cfg, rank_tol=1e-2)
+    for name, idx in sets.items():
+        g = tcb.tc_rank(pr, O, None if idx is None else dev(idx))
+        torch.cuda.synchronize()
+        assert not host(g["img_status"]).any(), (name, host(g["img_status"]))
+        for b in range(3):
+            sig, r = orc.token_information(batch["O"][b].astype(np.float64),
+                                           None if idx is None else idx[b], pr.rank_tol)
+            gs = host(g["sigma"])[b].astype(np.float64)
+            band = 4e-6 * sig[0] ** 2
+            assert np.max(np.abs(gs[:len(sig)] ** 2 - sig ** 2)) <= band, (name, b)
+            cut2 = (float(np.float32(pr.rank_tol)) * sig[0]) ** 2
+            r_lo, r_hi = int(np.sum(sig ** 2 > cut2 + band)), int(np.sum(sig ** 2 > cut2 - band))
+            assert r_lo <= int(host(g["rank"])[b]) <= r_hi, (name, b, int(host(g["rank"])[b]), r)
+            # well above the cut the singular values themselves agree to the usual 1e-3
+            big = sig > 0.05 * sig[0]
+            assert pu.rel_err(gs[:len(sig)][big], sig[big]) <= pu.REL_SCORE, (name, b)
+    # the order of the token list does not matter; a bad token number is reported, not a fault
+    idx = sets["half"].copy()
+    a = tcb.tc_rank(pr, O, dev(idx))
+    b2 = tcb.tc_rank(pr, O, dev(np.ascontiguousarray(idx[:, ::-1])))
+    torch.cuda.synchronize()
+    assert np.array_equal(host(a["rank"]), host(b2["rank"]))
+    assert pu.rel_err(host(b2["sigma"])[:, :100], host(a["sigma"])[:, :100]) <= 1e-4
+    idx[1, 5] = cfg.n_tokens
+    bad = tcb.tc_rank(pr, O, dev(idx))
+    torch.cuda.synchronize()
+    assert host(bad["img_status"]).tolist() == [0, 1, 0]
+
+
 # ------------------------------------------------------------------ launch modes
 def test_image_groups_and_graph_replay_do_not_change_results():
     cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=6)
