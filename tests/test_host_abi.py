@@ -79,3 +79,23 @@ def test_null_pointers_and_short_workspace_return_status_without_a_gpu():
     assert lib.tc_prune(C.byref(cp), None, dummy, dummy, dummy, 1 << 40, None) == 1
     assert lib.tc_compact(C.byref(cp), dummy, dummy, None, dummy, dummy, dummy, dummy, None, None,
                           dummy, 1 << 40, None) == 1
+
+
+def test_tc_rank_arguments_are_checked_on_the_host():
+    lib = tcb.lib()
+    p = _params(batch=2, rank_cap=160)
+    full, half, few = (tcb.tc_rank_workspace_bytes(p, n) for n in (576, 288, 40))
+    assert full > half > few > 0
+    assert half >= 2 * 288 * 4096 * 2 + 2 * 288 * 288 * 4           # gathered rows + Gram
+    assert few >= 2 * 40 * 4096 * 2 + 4 * 2 * 40 * 40 * 4            # ... + tridiagonal scratch
+    for n_sub in (0, 577, -3):
+        with pytest.raises(tcb.TokenCarveError) as e:
+            tcb.tc_rank_workspace_bytes(p, n_sub)
+        assert e.value.status == 1
+    cp = p.c()
+    dummy = C.c_void_p(256)          # never dereferenced: the checks below fail first
+    # no token list means all rows
+    assert lib.tc_rank(C.byref(cp), dummy, None, 288, dummy, dummy, dummy, dummy, 1 << 40, None) == 1
+    # rank and status outputs are required, sigma is optional; a short workspace is refused
+    assert lib.tc_rank(C.byref(cp), dummy, dummy, 288, dummy, None, dummy, dummy, 1 << 40, None) == 1
+    assert lib.tc_rank(C.byref(cp), dummy, dummy, 288, None, dummy, dummy, dummy, 16, None) == 3
