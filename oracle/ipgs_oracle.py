@@ -164,6 +164,21 @@ def token_information(O: np.ndarray, idx: Optional[Sequence[int]], rank_tol: flo
     return sigma, numerical_rank(sigma, rank_tol)
 
 
+def reassemble(Hs: np.ndarray, n_sys: int, n_vis: int, Xo: np.ndarray, kept_idx: Sequence[int]
+               ) -> Tuple[np.ndarray, np.ndarray]:
+    """Sequence after the compression (Sec. 3.1: the input is [system, visual, prompt] tokens;
+    Sec. 3.2: the visual part is rows L_s .. L_s + L_v; Conclusion: the surviving tokens keep
+    their original position IDs).  Hs [L, d] holds all L = n_sys + n_vis + n_text hidden states
+    before it, Xo [keep, d] the compacted visual tokens in ascending original order, kept_idx
+    their original visual-token numbers.  Returns (rows [n_sys + keep + n_text, d] in Hs's dtype,
+    original position of every row)."""
+    kept = np.asarray(list(kept_idx), np.int64)
+    L = Hs.shape[0]
+    rows = np.concatenate([Hs[:n_sys], np.asarray(Xo, Hs.dtype), Hs[n_sys + n_vis:]], axis=0)
+    pos = np.concatenate([np.arange(n_sys), n_sys + kept, np.arange(n_sys + n_vis, L)])
+    return rows, pos.astype(np.int64)
+
+
 # --------------------------------------------------------------------------
 # scores (Sec. 3.3.1)
 # --------------------------------------------------------------------------

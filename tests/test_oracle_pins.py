@@ -459,3 +459,26 @@ def test_token_information_closed_forms():
     sig, _ = orc.token_information(L, [0, 2, 4, 6], 0.0)
     assert np.isclose(np.sum(sig ** 2), np.sum(L[[0, 2, 4, 6]] ** 2), rtol=1e-12)
 
+
+# ------------------------------------------------------------------ sequence after the compression
+def test_reassemble_closed_forms():
+    rng = np.random.default_rng(9)
+    n_sys, n_vis, n_text, d = 3, 7, 4, 5
+    Hs = rng.standard_normal((n_sys + n_vis + n_text, d)).astype(np.float32)
+    vis = Hs[n_sys:n_sys + n_vis]
+    # nothing removed: the sequence and its positions come back unchanged
+    rows, pos = orc.reassemble(Hs, n_sys, n_vis, vis, range(n_vis))
+    assert np.array_equal(rows, Hs) and pos.tolist() == list(range(len(Hs)))
+    # three visual tokens kept: system rows, those three, then the prompt rows, positions original
+    kept = [1, 4, 6]
+    Xo = 2.0 * vis[kept]
+    rows, pos = orc.reassemble(Hs, n_sys, n_vis, Xo, kept)
+    assert rows.shape == (n_sys + 3 + n_text, d) and rows.dtype == Hs.dtype
+    assert np.array_equal(rows[:3], Hs[:3]) and np.array_equal(rows[3:6], Xo)
+    assert np.array_equal(rows[6:], Hs[10:])
+    assert pos.tolist() == [0, 1, 2, 4, 7, 9, 10, 11, 12, 13]
+    assert np.all(np.diff(pos) > 0)
+    # no system or prompt tokens at all
+    rows, pos = orc.reassemble(vis, 0, n_vis, Xo, kept)
+    assert np.array_equal(rows, Xo) and pos.tolist() == kept
+
