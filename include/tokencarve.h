@@ -217,6 +217,27 @@ tc_status tc_rank(const tc_params* p, const void* O, const int32_t* idx, int32_t
                   void* stream);
 
 /*
+ * Sec. 3.1 (the LLM input is the sequence [system tokens, visual tokens, prompt tokens]) and
+ * the Conclusion (the surviving tokens keep their original positional relationships: rotary
+ * encodings of the later layers use the original position IDs): the hidden-state sequence the
+ * layers after the compression run on, and the original position of each of its rows.
+ *   p        batch, n_tokens (= the visual tokens before compression), d_model, dtype, keep
+ *   n_sys, n_text  numbers of system and prompt tokens (>= 0)
+ *   Hs       device, [B, n_sys + n_tokens + n_text, d] hidden states before the compression
+ *            (only its system and prompt rows are read; may be NULL when there are none)
+ *   Xo       device, [B, keep, d] compacted visual tokens (tc_compact / tc_carve output)
+ *   kept_idx device, [B, keep] int32 original visual-token numbers, ascending (same output)
+ *   Ho       device, [B, n_sys + keep + n_text, d] out
+ *   pos      device, [B, n_sys + keep + n_text] int32 out: 0 .. n_sys-1, n_sys + kept_idx,
+ *            n_sys + n_tokens .. (strictly ascending)
+ * Row lengths must be whole 16-byte vectors, pointers 16-byte aligned.  No workspace; asynchronous
+ * on `stream`.  kept_idx is trusted to lie in [0, n_tokens): it only enters `pos`.
+ */
+tc_status tc_reassemble(const tc_params* p, int32_t n_sys, int32_t n_text, const void* Hs,
+                        const void* Xo, const int32_t* kept_idx, void* Ho, int32_t* pos,
+                        void* stream);
+
+/*
  * Number of image groups tc_score / tc_carve run side by side (1..8, default 4; the paper has no
  * counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
  * chains are enqueued on internal streams forked from `stream` and joined back into it before

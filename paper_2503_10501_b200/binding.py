@@ -27,7 +27,7 @@ EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge"
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
            "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
-           "tc_rank_workspace_bytes")
+           "tc_rank_workspace_bytes", "tc_reassemble")
 
 
 class TcParams(C.Structure):
@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
         L.tc_carve_host.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_rank_workspace_bytes.argtypes = [pp, C.c_int32, C.POINTER(sz)]
         L.tc_rank.argtypes = [pp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
+        L.tc_reassemble.argtypes = [pp, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp]
         L.tc_gram.argtypes = [pp, vp, vp, vp]
         L.tc_set_groups.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
@@ -218,6 +219,18 @@ def tc_rank(p: Params, O, idx=None, ws=None) -> Dict[str, torch.Tensor]:
                                     _ptr(out["rank"]), _ptr(out["img_status"]), _ptr(ws), ws.numel(),
                                     _stream()))
     return out
+
+
+def tc_reassemble(p: Params, n_sys: int, n_text: int, Hs, Xo, kept_idx):
+    """(Ho [B, n_sys + keep + n_text, d], pos [B, n_sys + keep + n_text] int32)."""
+    dev = Xo.device
+    Lo = n_sys + p.keep + n_text
+    Ho = torch.empty(p.batch, Lo, p.d_model, dtype=Xo.dtype, device=dev)
+    pos = torch.empty(p.batch, Lo, dtype=torch.int32, device=dev)
+    cp = p.c()
+    _check("tc_reassemble", lib().tc_reassemble(C.byref(cp), n_sys, n_text, _ptr(Hs), _ptr(Xo),
+                                                _ptr(kept_idx), _ptr(Ho), _ptr(pos), _stream()))
+    return Ho, pos
 
 
 def tc_prune(p: Params, E, ws=None) -> Tuple[torch.Tensor, torch.Tensor]:

@@ -588,6 +588,19 @@ tc_status tc_rank(const tc_params* p, const void* O, const int32_t* idx, int32_t
   return check_launch();
 }
 
+tc_status tc_reassemble(const tc_params* p, int32_t n_sys, int32_t n_text, const void* Hs,
+                        const void* Xo, const int32_t* kept_idx, void* Ho, int32_t* pos,
+                        void* stream) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  if (n_sys < 0 || n_text < 0) return TC_ERR_INVALID_ARG;
+  if (!Xo || !kept_idx || !Ho || !pos || misaligned(Xo) || misaligned(Ho)) return TC_ERR_INVALID_ARG;
+  if ((n_sys > 0 || n_text > 0) && (!Hs || misaligned(Hs))) return TC_ERR_INVALID_ARG;
+  launch_reassemble(D, n_sys, n_text, Hs, Xo, kept_idx, Ho, pos, (cudaStream_t)stream);
+  return check_launch();
+}
+
 const char* tc_status_string(int32_t status) {
   switch (status) {
     case TC_OK: return "ok";

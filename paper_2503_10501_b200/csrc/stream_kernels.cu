@@ -327,4 +327,43 @@ void launch_gather_rows(const Dims& D, int n_sub, const void* O, const int32_t* 
                                             D.d * D.esz / 16, status); note_launch(); }
 }
 
+// ------------------------------------------------------------------------------------------
+// Sequence after the compression (Sec. 3.1: [system, visual, prompt]; Conclusion: original
+// position IDs are kept).  Output row j of image b: a system row, compacted visual row
+// j - n_sys, or a prompt row, with its original position.  grid (L_out, B); 16-byte vectors.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) reassemble_kernel(const uint4* __restrict__ Hs,
+                                                        const uint4* __restrict__ Xo,
+                                                        const int32_t* __restrict__ kept,
+                                                        uint4* __restrict__ Ho,
+                                                        int32_t* __restrict__ pos, int n_sys,
+                                                        int n_vis, int n_text, int keep,
+                                                        int vec_per_row) {
+  const int b = blockIdx.y, j = blockIdx.x;
+  const int L = n_sys + n_vis + n_text, Lo = n_sys + keep + n_text;
+  const uint4* src;
+  int p;
+  if (j < n_sys) {
+    p = j;
+    src = Hs + ((size_t)b * L + j) * vec_per_row;
+  } else if (j < n_sys + keep) {
+    p = n_sys + kept[(size_t)b * keep + j - n_sys];
+    src = Xo + ((size_t)b * keep + j - n_sys) * vec_per_row;
+  } else {
+    p = j - keep + n_vis;
+    src = Hs + ((size_t)b * L + p) * vec_per_row;
+  }
+  uint4* dst = Ho + ((size_t)b * Lo + j) * vec_per_row;
+  for (int v = threadIdx.x; v < vec_per_row; v += 128) dst[v] = __ldg(src + v);
+  if (threadIdx.x == 0) pos[(size_t)b * Lo + j] = p;
+}
+
+void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, const void* Xo,
+                       const int32_t* kept, void* Ho, int32_t* pos, cudaStream_t st) {
+  Scope scope_(KC_COMPACT, st);
+  dim3 grid(n_sys + D.keep + n_text, D.B);
+  { reassemble_kernel<<<grid, 128, 0, st>>>((const uint4*)Hs, (const uint4*)Xo, kept, (uint4*)Ho, pos,
+                                           n_sys, D.N, n_text, D.keep, D.d * D.esz / 16); note_launch(); }
+}
+
 }  // namespace tc

@@ -91,6 +91,9 @@ void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
 void launch_gather_rows(const Dims& D, int n_sub, const void* O, const int32_t* idx, void* Os,
                         int32_t* status, cudaStream_t st);
 void fill_i32(int32_t* p, int n, int v, cudaStream_t st);
+// Sec. 3.1 / Conclusion: [system, compacted visual, prompt] rows and their original positions.
+void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, const void* Xo,
+                       const int32_t* kept, void* Ho, int32_t* pos, cudaStream_t st);
 
 // G = O O^T (float32 out).
 tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);

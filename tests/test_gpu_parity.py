@@ -328,6 +328,24 @@ def test_token_information_against_oracle():
     assert host(bad["img_status"]).tolist() == [0, 1, 0]
 
 
+def test_reassembled_sequence_and_positions():
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=3)
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    out = tcb.tc_carve(p, dev(batch["O"]), dev(batch["A"]), dev(batch["X"]), dev(batch["K"]), dev(batch["V"]))
+    Xo, kept = out[0], out[3]
+    rng = np.random.default_rng(8)
+    for n_sys, n_text in ((35, 64), (0, 7), (5, 0), (0, 0)):
+        L = n_sys + cfg.n_tokens + n_text
+        Hs = rng.standard_normal((3, L, cfg.d_model)).astype(np.float16)
+        Hs[:, n_sys:n_sys + cfg.n_tokens] = batch["X"]
+        Ho, pos = tcb.tc_reassemble(p, n_sys, n_text, dev(Hs) if n_sys + n_text else None, Xo, kept)
+        torch.cuda.synchronize()
+        for b in range(3):
+            rows, want = orc.reassemble(Hs[b], n_sys, cfg.n_tokens, host(Xo)[b], host(kept)[b])
+            assert np.array_equal(host(Ho)[b], rows) and host(pos)[b].tolist() == want.tolist()
+
+
 # ------------------------------------------------------------------ launch modes
 def test_image_groups_and_graph_replay_do_not_change_results():
     cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=6)

@@ -99,3 +99,14 @@ def test_tc_rank_arguments_are_checked_on_the_host():
     # rank and status outputs are required, sigma is optional; a short workspace is refused
     assert lib.tc_rank(C.byref(cp), dummy, dummy, 288, dummy, None, dummy, dummy, 1 << 40, None) == 1
     assert lib.tc_rank(C.byref(cp), dummy, dummy, 288, None, dummy, dummy, dummy, 16, None) == 3
+
+
+def test_tc_reassemble_arguments_are_checked_on_the_host():
+    lib = tcb.lib()
+    cp = _params(batch=2, rank_cap=160).c()
+    dummy = C.c_void_p(256)          # never dereferenced: the checks below fail first
+    assert lib.tc_reassemble(C.byref(cp), -1, 4, dummy, dummy, dummy, dummy, dummy, None) == 1
+    assert lib.tc_reassemble(C.byref(cp), 3, 4, None, dummy, dummy, dummy, dummy, None) == 1
+    assert lib.tc_reassemble(C.byref(cp), 3, 4, dummy, None, dummy, dummy, dummy, None) == 1
+    assert lib.tc_reassemble(C.byref(cp), 0, 0, None, dummy, dummy, dummy, None, None) == 1
+    assert lib.tc_reassemble(C.byref(cp), 3, 4, C.c_void_p(8), dummy, dummy, dummy, dummy, None) == 1
