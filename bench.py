@@ -451,6 +451,67 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+# ----------------------------------------------------------------------------- the two side entries
+def run_extras(args):
+    """One JSON line each for tc_rank and tc_reassemble at the bench point (event-timed, inputs
+    resident): the information-quantity curve of Sec. 3.2 at three token counts, and the
+    re-assembled sequence of the layers after the compression."""
+    import torch
+    from paper_2503_10501_b200 import binding as tcb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the carve path")
+    torch.cuda.set_device(0)
+    tcb.lib()
+    pk = peaks()
+    cfg, name = workload(args)
+    p = tcb.Params(batch=cfg.batch, n_tokens=cfg.n_tokens, d_model=cfg.d_model, n_heads=cfg.n_heads,
+                   head_dim=cfg.head_dim, n_query=cfg.n_query, keep=cfg.keep, rho=cfg.rho,
+                   lam=cfg.lam, rank_tol=1e-2, dtype=cfg.dtype, rank_cap=cfg.rank_cap)
+    batch = inputs.make_batch(cfg)
+    dev = {k: torch.from_numpy(v).cuda() for k, v in batch.items()}
+    out = tcb.tc_carve(p, dev["O"], dev["A"], dev["X"], dev["K"], dev["V"])
+    Xo, kept = out[0], out[3]
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    e = 2 if cfg.dtype == "f16" else 4
+    g = torch.Generator().manual_seed(1)
+    for label, idx in (("all 576 tokens", None), ("the 128 kept tokens", kept),
+                       ("288 random tokens", torch.stack([torch.randperm(cfg.n_tokens, generator=g)[:288]
+                                                          for _ in range(cfg.batch)]).int().cuda())):
+        n_sub = cfg.n_tokens if idx is None else idx.shape[1]
+        ws = torch.empty(tcb.tc_rank_workspace_bytes(p, n_sub), dtype=torch.uint8, device="cuda")
+        res = tcb.tc_rank(p, dev["O"], idx, ws)
+        torch.cuda.synchronize()
+        ms = timed(lambda: tcb.tc_rank(p, dev["O"], idx, ws))
+        print(json.dumps({"entry": "tc_rank", "workload": name, "token_set": label,
+                          "ms_per_call": round(ms, 4), "images_per_s": round(cfg.batch / (ms * 1e-3), 1),
+                          "rank_of_image_0": int(res["rank"][0]), "status_any": bool(res["img_status"].any()),
+                          "bytes_read_per_call": cfg.batch * n_sub * cfg.d_model * e}), flush=True)
+    n_sys, n_text = 35, args.n_query
+    L = n_sys + cfg.n_tokens + n_text
+    Hs = torch.randn(cfg.batch, L, cfg.d_model, device="cuda").to(dev["X"].dtype)
+    ms = timed(lambda: tcb.tc_reassemble(p, n_sys, n_text, Hs, Xo, kept))
+    moved = 2 * cfg.batch * (n_sys + cfg.keep + n_text) * cfg.d_model * e
+    print(json.dumps({"entry": "tc_reassemble", "workload": name, "n_sys": n_sys, "n_text": n_text,
+                      "ms_per_call": round(ms, 4), "bytes_per_call": moved,
+                      "roofline": {"bound": "hbm", "achieved": round(moved / (ms * 1e-3) / 1e9, 1),
+                                   "peak": pk["hbm_gbs"], "unit": "GB/s",
+                                   "frac": round(moved / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], 4),
+                                   "note": "the call also allocates its two outputs"}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -469,8 +530,12 @@ def main():
                     help="images the CPU oracle is timed on (0 = skip)")
     ap.add_argument("--sweep", action="store_true",
                     help="one line per point of the T x keep sweep instead of the bench line")
+    ap.add_argument("--extras", action="store_true",
+                    help="time tc_rank and tc_reassemble at the bench point instead of the bench line")
     args = ap.parse_args()
-    if args.sweep:
+    if args.extras:
+        run_extras(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
