@@ -218,7 +218,7 @@ def run_ours(args):
 
     # The timed step replays a CUDA graph of one tc_carve call (same kernels, same streams: the
     # fork/join of the library's internal streams is captured as graph dependencies), which
-    # takes the ~25 dependent launches of a group's chain off the host: 1.85 ms against 1.91 ms
+    # takes the ~25 dependent launches of a group's chain off the host: 1.82 ms against 1.86 ms
     # per step for plain calls (--no-graph).
     eager_step = step
     graph = None

@@ -187,8 +187,9 @@ static tc_status open_ctx(const tc_params* p, void* ws, size_t ws_bytes, void* s
 constexpr int kMaxGroups = 8;
 struct GroupStreams {
   bool ready = false;
-  cudaStream_t s[kMaxGroups];
-  cudaEvent_t fork, join[kMaxGroups];
+  cudaStream_t s[kMaxGroups];    // a group's sketch -> Cholesky-QR -> eigen-solve chain
+  cudaStream_t s2[kMaxGroups];   // its Gram matrix, which the chain needs only from G Q on
+  cudaEvent_t fork, join[kMaxGroups], gram_done[kMaxGroups];
 };
 static std::mutex g_groups_mu;
 static GroupStreams g_groups[64];
@@ -201,7 +202,9 @@ static GroupStreams* group_streams() {
   if (!g.ready) {
     for (int i = 0; i < kMaxGroups; ++i) {
       if (cudaStreamCreateWithFlags(&g.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+      if (cudaStreamCreateWithFlags(&g.s2[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
       if (cudaEventCreateWithFlags(&g.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&g.gram_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     }
     if (cudaEventCreateWithFlags(&g.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     g.ready = true;
@@ -231,9 +234,19 @@ static void enqueue_score(const Ctx& c, const void* O, const void* A, float* E, 
     Dims Dg = D;
     Dg.B = nb;
     const char* Og = (const char*)O + (size_t)b0 * D.N * D.d * D.esz;
-    launch_gram(Dg, Og, (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N, img_status + b0, st);
+    // the sketch and its first Cholesky-QR pass do not read G: with groups, the Gram matrix is
+    // built beside them on a stream of its own and joined in front of the first product with G
+    cudaEvent_t gram_done = nullptr;
+    if (ng > 1 && !D.full) {
+      cudaStreamWaitEvent(gs->s2[g], gs->fork, 0);
+      launch_gram(Dg, Og, (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N, img_status + b0, gs->s2[g]);
+      cudaEventRecord(gs->gram_done[g], gs->s2[g]);
+      gram_done = gs->gram_done[g];
+    } else {
+      launch_gram(Dg, Og, (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N, img_status + b0, st);
+    }
     launch_ics(Dg, c.P, c.ws, b0, Og, C + (size_t)b0 * D.N, sigma ? sigma + (size_t)b0 * q : nullptr,
-               rank ? rank + b0 : nullptr, img_status + b0, st);
+               rank ? rank + b0 : nullptr, img_status + b0, st, nullptr, gram_done);
     if (ng > 1) {
       cudaEventRecord(gs->join[g], st);
       cudaStreamWaitEvent(c.st, gs->join[g], 0);

@@ -2377,7 +2377,7 @@ void fill_i32(int32_t* p, int n, int v, cudaStream_t st) {
 // ==========================================================================================
 void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
                 float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
-                float* full_scratch) {
+                float* full_scratch, cudaEvent_t g_ready) {
   // D.B images starting at image b0 of the workspace arrays; O and the outputs already point at
   // image b0.
   const int B = D.B, N = D.N, k = D.k;
@@ -2389,6 +2389,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   float* theta = (float*)(ws + P.sigma) + (size_t)b0 * k;
 
   if (D.full) {
+    if (g_ready) cudaStreamWaitEvent(st, g_ready, 0);
     // with scratch for it (four N x N arrays per image) the tridiagonal solver takes the full
     // problem when it fits in shared memory: it has no sweeps that a spectrum without a gap at
     // the rounding level could keep alive
@@ -2443,6 +2444,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   cholqr_pass(Y0, Y1, kShift);
   { float* t = Y0; Y0 = Y1; Y1 = t; }  // Q0 in Y0
   // 3. one multiplication by G sharpens the subspace:  Y1 = G Q0, then orthonormalise
+  if (g_ready) cudaStreamWaitEvent(st, g_ready, 0);
   gemm<float, float, false, false>(G, Y0, Y1, N, k, N, N, k, k, sG, sY, sY, B, st, KC_GEMM_GQ);
   cholqr_pass(Y1, Y2, kShift);
   cholqr_pass(Y2, Y1, kShift);

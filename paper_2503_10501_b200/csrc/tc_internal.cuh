@@ -99,10 +99,12 @@ void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, con
 tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 
 // Eigen-decomposition of G and Eq. 3-6:  C, theta (unsorted), then sorted sigma / rank.
+// g_ready: optional event after which G is complete when it is built on another stream (the
+// subspace solve waits for it in front of its first product with G).
 // full_scratch: optional 4 * B * N * N floats; with it a full solve (rank_cap = 0) of a matrix
 // that fits in shared memory goes through the tridiagonal solver instead of Jacobi sweeps.
 void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
                 float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
-                float* full_scratch = nullptr);
+                float* full_scratch = nullptr, cudaEvent_t g_ready = nullptr);
 
 }  // namespace tc
