@@ -242,7 +242,10 @@ tc_status tc_reassemble(const tc_params* p, int32_t n_sys, int32_t n_text, const
  * counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
  * chains are enqueued on internal streams forked from `stream` and joined back into it before
  * the call's remaining kernels, so that the one-block-per-image solver kernels of one group
- * overlap the GEMMs of another.  Results do not depend on the setting.  Process-wide.
+ * overlap the GEMMs of another.  Results do not depend on the setting.  Process-wide.  Each
+ * group costs the host a few dozen launches per call: more than four groups pay only when the
+ * call is replayed from a CUDA graph (measured at B = 64: 1.86 ms with 4 groups and 2.80 ms with
+ * 8 for plain calls, 1.82 ms with 8 under replay).
  */
 tc_status tc_set_groups(int32_t groups);
 

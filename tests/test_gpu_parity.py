@@ -307,6 +307,17 @@ def test_cfg5_bench_point_properties_of_every_image():
                     acc = acc + X[t].astype(np.float32)
                 want = (acc / np.float32(len(group) + 1)).astype(np.float16)
                 assert np.array_equal(Xo[j], want), (b, j)
+        if b in (0, 63):  # the same map on every head of K and V
+            for name in ("K", "V"):
+                T_, To = batch[name][b], res[name + "o"][b]        # [H, N, dh], [H, keep, dh]
+                for j, a in enumerate(kept):
+                    group = src[dst == a]
+                    acc = T_[:, a].astype(np.float32)
+                    for t in group:
+                        acc = acc + T_[:, t].astype(np.float32)
+                    want = T_[:, a] if len(group) == 0 else \
+                        (acc / np.float32(len(group) + 1)).astype(np.float16)
+                    assert np.array_equal(To[:, j], want), (name, b, j)
 
 
 @pytest.mark.parametrize("T,keep", [(32, 64), (512, 288)])
