@@ -91,6 +91,10 @@ tc_status make_dims(const tc_params* p, Dims* out) {
   D.k = D.full ? D.N : p->rank_cap;
   if (D.k > 1024) return TC_ERR_UNSUPPORTED;  // Jacobi keeps at most 32 elements per lane
   if (!D.full && D.k < 16) return TC_ERR_INVALID_ARG;
+  // the subspace solve runs its products on the tensor cores when the shapes fit its tiles
+  // (the sign sketch keeps one row of signs, d floats, in shared memory)
+  D.tcp = !D.full && (D.N & 3) == 0 && (size_t)D.d * sizeof(float) <= 48 * 1024 &&
+          gemm_split_supported(D.N, D.k, D.N) && gemm_split_supported(D.N, D.k, D.k);
   D.max_sweeps = p->max_sweeps > 0 ? p->max_sweeps : 30;
   D.lambda = p->lambda;
   D.rank_tol = p->rank_tol;
@@ -123,8 +127,18 @@ Plan make_plan(const Dims& D) {
   P.C = take(B * N * 4);
   P.E = take(B * N * 4);
   P.sigma = take(B * k * 4);
-  P.G = take(B * N * N * 4);
-  if (!D.full) {
+  P.G = take(B * N * N * 4 * (D.tcp ? 2 : 1));
+  if (D.tcp) {
+    P.panel_T_off = align_up(B * 2 * N * k * 4, 256);
+    P.PA = take(2 * P.panel_T_off);
+    P.PB = take(2 * P.panel_T_off);
+    P.Sk = take(B * k * k * 4);
+    P.Hk = take(B * k * k * 4);
+    P.RinvS = take(B * 2 * k * k * 4);
+    P.ZTs = take(B * 2 * k * k * 4);
+    P.Es = take(B * 5 * k * k * 4);
+    if (!D.f16) P.Gplain = take(B * N * N * 4);
+  } else if (!D.full) {
     P.Y0 = take(B * N * k * 4);
     P.Y1 = take(B * N * k * 4);
     P.Y2 = take(B * N * k * 4);
@@ -133,8 +147,10 @@ Plan make_plan(const Dims& D) {
     P.Rinv = take(B * k * k * 4);
     P.Hm = take(B * k * k * 4 * parts);
   }
-  P.W = take(B * k * k * 4);
-  P.ZT = take(B * k * k * 4);
+  if (!D.tcp) {
+    P.W = take(B * k * k * 4);
+    P.ZT = take(B * k * k * 4);
+  }
   P.setA = take(B * (size_t)(D.nA > 0 ? D.nA : 1) * 4);
   P.setB = take(B * (size_t)D.nB * 4);
   P.best_val = take(B * (size_t)D.nB * 4);
@@ -149,9 +165,17 @@ Plan make_plan(const Dims& D) {
 }
 
 // float16 inputs go to the tensor cores; float32 inputs keep full precision on the plain ALUs
-tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st) {
+// With Dims::tcp, G receives the two TF32 planes per image; float32 inputs first go to
+// `Gplain` [B][N][N] and are split from there.
+tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st,
+                      float* Gplain) {
   if (D.f16) return launch_gram_tc(D, O, G, status, st);
-  return launch_gram_simt(D, O, G, st);
+  if (!D.tcp) return launch_gram_simt(D, O, G, st);
+  if (Gplain == nullptr) return TC_ERR_INVALID_ARG;
+  tc_status s = launch_gram_simt(D, O, Gplain, st);
+  if (s != TC_OK) return s;
+  launch_split_panel(Gplain, D.N, D.N, D.B, G, nullptr, st, KC_GRAM);
+  return TC_OK;
 }
 
 static tc_status check_launch() {
@@ -213,8 +237,11 @@ static GroupStreams* group_streams() {
 }
 
 // score: S partial sums || (Gram -> eigen-solve -> C per image group) -> E
-static void enqueue_score(const Ctx& c, const void* O, const void* A, float* E, float* C, float* S,
-                          float* sigma, int32_t* rank, int32_t* img_status) {
+// A launcher that refuses (tensor map, function attribute) stops the enqueue: the group streams
+// forked so far are joined back, the status words of the images not reached are set, and the
+// caller gets the status.
+static tc_status enqueue_score(const Ctx& c, const void* O, const void* A, float* E, float* C, float* S,
+                               float* sigma, int32_t* rank, int32_t* img_status) {
   const Dims& D = c.D;
   const int q = D.N < D.d ? D.N : D.d;
   fill_i32(img_status, D.B, 0, c.st);
@@ -227,7 +254,8 @@ static void enqueue_score(const Ctx& c, const void* O, const void* A, float* E, 
   launch_attn_colsum(D, A, (float*)(c.ws + c.P.s_part), c.st);
   const int base = D.B / ng, extra = D.B % ng;
   int b0 = 0;
-  for (int g = 0; g < ng; ++g) {
+  tc_status err = TC_OK;
+  for (int g = 0; g < ng && err == TC_OK; ++g) {
     const int nb = base + (g < extra ? 1 : 0);
     cudaStream_t st = ng > 1 ? gs->s[g] : c.st;
     if (ng > 1) cudaStreamWaitEvent(st, gs->fork, 0);
@@ -237,23 +265,31 @@ static void enqueue_score(const Ctx& c, const void* O, const void* A, float* E, 
     // the sketch and its first Cholesky-QR pass do not read G: with groups, the Gram matrix is
     // built beside them on a stream of its own and joined in front of the first product with G
     cudaEvent_t gram_done = nullptr;
+    float* Gg = (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N * (D.tcp ? 2 : 1);
+    float* Gp = (D.tcp && !D.f16) ? (float*)(c.ws + c.P.Gplain) + (size_t)b0 * D.N * D.N : nullptr;
     if (ng > 1 && !D.full) {
       cudaStreamWaitEvent(gs->s2[g], gs->fork, 0);
-      launch_gram(Dg, Og, (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N, img_status + b0, gs->s2[g]);
+      err = launch_gram(Dg, Og, Gg, img_status + b0, gs->s2[g], Gp);
       cudaEventRecord(gs->gram_done[g], gs->s2[g]);
       gram_done = gs->gram_done[g];
     } else {
-      launch_gram(Dg, Og, (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N, img_status + b0, st);
+      err = launch_gram(Dg, Og, Gg, img_status + b0, st, Gp);
     }
-    launch_ics(Dg, c.P, c.ws, b0, Og, C + (size_t)b0 * D.N, sigma ? sigma + (size_t)b0 * q : nullptr,
-               rank ? rank + b0 : nullptr, img_status + b0, st, nullptr, gram_done);
+    if (err == TC_OK)
+      err = launch_ics(Dg, c.P, c.ws, b0, Og, C + (size_t)b0 * D.N, sigma ? sigma + (size_t)b0 * q : nullptr,
+                       rank ? rank + b0 : nullptr, img_status + b0, st, nullptr, gram_done);
+    else if (gram_done)
+      cudaStreamWaitEvent(st, gram_done, 0);  // the side stream still joins the group's stream
     if (ng > 1) {
       cudaEventRecord(gs->join[g], st);
       cudaStreamWaitEvent(c.st, gs->join[g], 0);
     }
+    if (err != TC_OK) fill_i32(img_status + b0, D.B - b0, (int)err, c.st);
     b0 += nb;
   }
+  if (err != TC_OK) return err;
   launch_combine(D, (const float*)(c.ws + c.P.s_part), C, S, E, c.st);
+  return TC_OK;
 }
 
 }  // namespace tc
@@ -291,7 +327,8 @@ tc_status tc_score(const tc_params* p, const void* O, const void* A, float* E, f
   if (!O || !A || !E || !img_status || misaligned(O) || misaligned(A)) return TC_ERR_INVALID_ARG;
   float* Cw = C ? C : (float*)(c.ws + c.P.C);
   float* Sw = S ? S : (float*)(c.ws + c.P.S);
-  enqueue_score(c, O, A, E, Cw, Sw, sigma, rank, img_status);
+  s = enqueue_score(c, O, A, E, Cw, Sw, sigma, rank, img_status);
+  if (s != TC_OK) return s;
   return check_launch();
 }
 
@@ -359,7 +396,8 @@ tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void*
   int32_t* bd = (int32_t*)(c.ws + c.P.best_dst);
   int32_t* msrc = (int32_t*)(c.ws + c.P.msrc);
   int32_t* mdst = (int32_t*)(c.ws + c.P.mdst);
-  enqueue_score(c, O, A, E, C, S, nullptr, nullptr, img_status);
+  s = enqueue_score(c, O, A, E, C, S, nullptr, nullptr, img_status);
+  if (s != TC_OK) return s;
   launch_prune(D, E, setA, setB, c.st);
   if (D.M > 0) launch_match_gram(D, (const float*)(c.ws + c.P.G), setA, setB, bv, bd, c.st);
   launch_merge_select(D, setA, setB, bv, bd, msrc, mdst, kept_idx, c.st);
@@ -538,7 +576,32 @@ tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream) {
   tc_status s = make_dims(p, &D);
   if (s != TC_OK) return s;
   if (!O || !G || misaligned(O) || misaligned(G)) return TC_ERR_INVALID_ARG;
-  s = launch_gram(D, O, G, nullptr, (cudaStream_t)stream);
+  D.tcp = false;  // plain float32 out, whatever rank_cap says
+  s = launch_gram(D, O, G, nullptr, (cudaStream_t)stream, nullptr);
+  if (s != TC_OK) return s;
+  return check_launch();
+}
+
+size_t tc_matmul_f32x3_workspace_bytes(int32_t batch, int32_t M, int32_t NN, int32_t K) {
+  if (batch < 1 || M < 1 || NN < 1 || K < 1) return 0;
+  return align_up((size_t)batch * 2 * M * K * 4, 256) + align_up((size_t)batch * 2 * NN * K * 4, 256);
+}
+
+tc_status tc_matmul_f32x3(const float* A, const float* B, float* C, float* CT, int32_t batch,
+                          int32_t M, int32_t NN, int32_t K, int32_t* img_status, void* ws,
+                          size_t ws_bytes, void* stream) {
+  if (!A || !B || !C || !ws || batch < 1 || M < 1 || NN < 1 || K < 1) return TC_ERR_INVALID_ARG;
+  if (misaligned(A) || misaligned(B) || misaligned(C) || misaligned(ws) || (CT && misaligned(CT)))
+    return TC_ERR_INVALID_ARG;
+  if (!gemm_split_supported(M, NN, K)) return TC_ERR_UNSUPPORTED;
+  if (ws_bytes < tc_matmul_f32x3_workspace_bytes(batch, M, NN, K)) return TC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* As = (float*)ws;
+  float* Bs = (float*)((char*)ws + align_up((size_t)batch * 2 * M * K * 4, 256));
+  if (img_status) fill_i32(img_status, batch, 0, st);
+  launch_split_panel(A, M, K, batch, As, nullptr, st, KC_GEMM);
+  launch_split_panel(B, NN, K, batch, Bs, nullptr, st, KC_GEMM);
+  tc_status s = launch_gemm_split(As, Bs, M, NN, K, batch, C, CT, nullptr, nullptr, img_status, st, KC_GEMM);
   if (s != TC_OK) return s;
   return check_launch();
 }
@@ -594,10 +657,12 @@ tc_status tc_rank(const tc_params* p, const void* O, const int32_t* idx, int32_t
     launch_gather_rows(F, n_sub, O, idx, w + rows_off, img_status, st);
     rows = w + rows_off;
   }
-  s = launch_gram(D, rows, (float*)(w + P.G), img_status, st);
+  s = launch_gram(D, rows, (float*)(w + P.G), img_status, st,
+                  (D.tcp && !D.f16) ? (float*)(w + P.Gplain) : nullptr);
   if (s != TC_OK) return s;
-  launch_ics(D, P, w, 0, rows, (float*)(w + P.C), sigma, rank, img_status, st,
-             rank_small_full(D) ? (float*)(w + rows_off + rank_rows_bytes(D)) : nullptr);
+  s = launch_ics(D, P, w, 0, rows, (float*)(w + P.C), sigma, rank, img_status, st,
+                 rank_small_full(D) ? (float*)(w + rows_off + rank_rows_bytes(D)) : nullptr);
+  if (s != TC_OK) return s;
   return check_launch();
 }
 

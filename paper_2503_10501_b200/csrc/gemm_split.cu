@@ -1,0 +1,314 @@
+// Batched float32-accurate products  C = A B^T  on the 5th-generation tensor cores (tcgen05,
+// kind::tf32): the dense products of the subspace solve behind Eq. 3-5 / 3-6 (Sec. 3.3.1).
+//
+// A float32 value x is carried as two TF32 numbers, x ~ hi + lo (both rounded to nearest, so the
+// pair is good to 2^-22 |x| and unbiased); a product is the three tensor-core products
+// hi hi + hi lo + lo hi, accumulated in float32.  Operands therefore live in memory as "split
+// panels": [image][2][rows][K] float32, plane 0 = hi, plane 1 = lo, the contraction index K
+// contiguous (both operands K-major).  Whoever writes an operand writes it in this form.
+//
+// One CTA produces a 128 x NN tile of C for one image (NN = the whole width of C, a multiple of
+// 16; 128, 144, 160 and 192 are built):
+//   - warp 8 (one lane) streams 32-wide K slabs of the four operand planes into a ring of
+//     shared-memory stages with TMA (128-byte swizzle, out-of-range rows / K read as zero);
+//   - warp 9 (one lane) issues the twelve tcgen05.mma (M = 128, N = NN, K = 8) of a slab into one
+//     of two TMEM accumulators, the small cross terms first, and frees the stage with
+//     tcgen05.commit;
+//   - warps 0-7 read a finished accumulator back with tcgen05.ld and add it to a float32
+//     register tile: the tensor core adds into its accumulator with truncation, so a fresh
+//     accumulator per slab and round-to-nearest adds in registers keep the bias out.
+// The epilogue writes C as plain float32 and / or as split panels, row-major and / or
+// transposed, as the consumer needs.  Every mbarrier wait is bounded; a wait that runs out
+// records an error for the image and the CTA winds down (TMEM is still freed).
+#include "tc_internal.cuh"
+#include "tcgen05_util.cuh"
+
+namespace tc {
+
+namespace {
+
+using namespace t5;
+
+constexpr int BM = 128;   // rows of C per CTA
+constexpr int BK = 32;    // floats of K per stage = one 128-byte swizzle row
+constexpr int UK = 8;     // K of one tcgen05.mma kind::tf32
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = (EPI_WARPS + 2) * 32;
+constexpr uint32_t TMEM_COLS = 512;   // two accumulators of up to 256 columns
+constexpr uint32_t ACC_STRIDE = 256;
+
+__host__ __device__ constexpr uint32_t a_plane_bytes() { return BM * BK * 4; }
+__host__ __device__ constexpr uint32_t b_plane_bytes(int nn) { return (uint32_t)nn * BK * 4; }
+__host__ __device__ constexpr uint32_t stage_bytes(int nn) { return 2 * a_plane_bytes() + 2 * b_plane_bytes(nn); }
+__host__ __device__ constexpr int stages_for(int nn) {
+  return (int)((226u * 1024u - 2048u) / stage_bytes(nn)) > 4 ? 4
+                                                              : (int)((226u * 1024u - 2048u) / stage_bytes(nn));
+}
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc,
+                                          uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accum)
+      : "memory");
+}
+
+struct Out {
+  float* plain;    // [batch][M][NN]
+  float* plainT;   // [batch][NN][M]
+  float* split;    // [batch][2][M][NN]
+  float* splitT;   // [batch][2][NN][M]
+};
+
+// NN: width of C (compile time: it sizes the register tile).  NCH = 16-column chunks per thread.
+template <int NN>
+__global__ void __launch_bounds__(THREADS) gemm_split_kernel(const __grid_constant__ CUtensorMap mapA,
+                                                           const __grid_constant__ CUtensorMap mapB,
+                                                           Out out, int M, int K, int m_tiles,
+                                                           int32_t* __restrict__ status) {
+  constexpr int STAGES = stages_for(NN);
+  constexpr int NCHUNK = NN / 16;            // 16-column chunks of the accumulator
+  constexpr int NCH = (NCHUNK + 1) / 2;      // chunks per thread (two column halves)
+  constexpr uint32_t A_PL = a_plane_bytes(), B_PL = b_plane_bytes(NN), STG = stage_bytes(NN);
+  // D float32, A and B TF32, both K-major, M = 128, N = NN
+  constexpr uint32_t IDESC = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(NN >> 3) << 17) |
+                             ((uint32_t)(BM >> 4) << 24);
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[STAGES];
+  __shared__ __align__(8) uint64_t bar_empty[STAGES];
+  __shared__ __align__(8) uint64_t bar_acc_full[2];
+  __shared__ __align__(8) uint64_t bar_acc_empty[2];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x / m_tiles, mt = blockIdx.x % m_tiles;
+  const int slabs = (K + BK - 1) / BK;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  auto st_a = [&](int s, int plane) { return smem_base + (uint32_t)s * STG + (uint32_t)plane * A_PL; };
+  auto st_b = [&](int s, int plane) { return smem_base + (uint32_t)s * STG + 2u * A_PL + (uint32_t)plane * B_PL; };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bar_acc_full[i]), 1);
+      mbar_init(smem_u32(&bar_acc_empty[i]), EPI_WARPS);
+    }
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == EPI_WARPS + 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&s_tmem)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = s_tmem;
+
+  if (warp == EPI_WARPS) {
+    // ---- TMA producer ----
+    if (lane == 0) {
+      for (int kb = 0; kb < slabs; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t round = (uint32_t)(kb / STAGES);
+        if (!mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u)) {
+          s_fail = 1;
+          break;
+        }
+        const uint32_t full = smem_u32(&bar_full[s]);
+        mbar_expect_tx(full, STG);
+        tma_load_3d(st_a(s, 0), &mapA, kb * BK, mt * BM, 2 * b, full);
+        tma_load_3d(st_a(s, 1), &mapA, kb * BK, mt * BM, 2 * b + 1, full);
+        tma_load_3d(st_b(s, 0), &mapB, kb * BK, 0, 2 * b, full);
+        tma_load_3d(st_b(s, 1), &mapB, kb * BK, 0, 2 * b + 1, full);
+      }
+    }
+  } else if (warp == EPI_WARPS + 1) {
+    // ---- MMA issuer ----
+    if (lane == 0) {
+      for (int kb = 0; kb < slabs; ++kb) {
+        const int buf = kb & 1;
+        if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), (((uint32_t)kb >> 1) & 1u) ^ 1u)) {
+          s_fail = 1;
+          break;
+        }
+        const int s = kb % STAGES;
+        const uint32_t round = (uint32_t)(kb / STAGES);
+        if (!mbar_wait(smem_u32(&bar_full[s]), round & 1u)) {
+          s_fail = 1;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t tmem_d = tmem_base + (uint32_t)buf * ACC_STRIDE;
+        const uint64_t ah = umma_desc(st_a(s, 0)), al = umma_desc(st_a(s, 1));
+        const uint64_t bh = umma_desc(st_b(s, 0)), bl = umma_desc(st_b(s, 1));
+        // 8 floats = 32 bytes further along K inside the swizzled row: +2 in 16-byte units.
+        // The cross terms go first: what the accumulator truncates while they are added is
+        // relative to their own small size.
+#pragma unroll
+        for (int k = 0; k < BK / UK; ++k)
+          umma_tf32(tmem_d, al + (uint64_t)(2 * k), bh + (uint64_t)(2 * k), IDESC, k > 0 ? 1u : 0u);
+#pragma unroll
+        for (int k = 0; k < BK / UK; ++k)
+          umma_tf32(tmem_d, ah + (uint64_t)(2 * k), bl + (uint64_t)(2 * k), IDESC, 1u);
+#pragma unroll
+        for (int k = 0; k < BK / UK; ++k)
+          umma_tf32(tmem_d, ah + (uint64_t)(2 * k), bh + (uint64_t)(2 * k), IDESC, 1u);
+        umma_commit(smem_u32(&bar_empty[s]));
+        umma_commit(smem_u32(&bar_acc_full[buf]));
+      }
+    }
+  } else {
+    // ---- epilogue: warp w owns TMEM lanes 32 (w % 4) .. + 31 (rows of the tile) and the
+    //      16-column chunks  half, half + 2, ...  with half = w / 4 ----
+    const int quad = warp & 3, half = warp >> 2;
+    float acc[NCH][16];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c)
+#pragma unroll
+      for (int j = 0; j < 16; ++j) acc[c][j] = 0.f;
+    bool ok = true;
+    for (int kb = 0; kb < slabs; ++kb) {
+      const int buf = kb & 1;
+      if (!mbar_wait(smem_u32(&bar_acc_full[buf]), ((uint32_t)kb >> 1) & 1u)) {
+        ok = false;
+        break;
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * ACC_STRIDE;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        const int chunk = 2 * c + half;
+        if (chunk < NCHUNK) {
+          float v[16];
+          tmem_ld16(taddr + (uint32_t)(chunk * 16), v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) acc[c][j] += v[j];
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_acc_empty[buf]))
+                     : "memory");
+    }
+    if (ok && s_fail == 0) {
+      const int row = mt * BM + quad * 32 + lane;
+      if (row < M) {
+        const size_t MN = (size_t)M * NN;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const int chunk = 2 * c + half;
+          if (chunk >= NCHUNK) continue;
+          const int col0 = chunk * 16;
+          float hi[16], lo[16];
+          if (out.split != nullptr || out.splitT != nullptr) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) tf32_split(acc[c][j], hi[j], lo[j]);
+          }
+          if (out.plain != nullptr) {
+            float4* dst = reinterpret_cast<float4*>(out.plain + (size_t)b * MN + (size_t)row * NN + col0);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              dst[j] = make_float4(acc[c][4 * j], acc[c][4 * j + 1], acc[c][4 * j + 2], acc[c][4 * j + 3]);
+          }
+          if (out.split != nullptr) {
+            float4* dh = reinterpret_cast<float4*>(out.split + (size_t)b * 2 * MN + (size_t)row * NN + col0);
+            float4* dl = reinterpret_cast<float4*>(out.split + (size_t)b * 2 * MN + MN + (size_t)row * NN + col0);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              dh[j] = make_float4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
+              dl[j] = make_float4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
+            }
+          }
+          if (out.plainT != nullptr) {
+            float* dst = out.plainT + (size_t)b * MN + (size_t)col0 * M + row;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) dst[(size_t)j * M] = acc[c][j];
+          }
+          if (out.splitT != nullptr) {
+            float* dh = out.splitT + (size_t)b * 2 * MN + (size_t)col0 * M + row;
+            float* dl = dh + MN;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              dh[(size_t)j * M] = hi[j];
+              dl[(size_t)j * M] = lo[j];
+            }
+          }
+        }
+      }
+    } else if (status != nullptr && threadIdx.x == 0) {
+      atomicMax(&status[b], (int)TC_ERR_CUDA);
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == EPI_WARPS + 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// [K, rows, 2 * batch] float32, box 32 x box_rows x 1, 128-byte swizzle, zero fill
+bool encode_panel(CUtensorMap* map, const float* base, int rows, int K, int batch, int box_rows) {
+  encode_fn enc = get_encode();
+  if (enc == nullptr) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)(2 * batch)};
+  const cuuint64_t strides[2] = {(cuuint64_t)K * 4, (cuuint64_t)rows * K * 4};
+  const cuuint32_t box[3] = {BK, (cuuint32_t)box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NN>
+tc_status launch_nn(const CUtensorMap& mapA, const CUtensorMap& mapB, const Out& out, int M, int K,
+                    int batch, int32_t* status, cudaStream_t st) {
+  constexpr uint32_t smem = (uint32_t)stages_for(NN) * stage_bytes(NN) + 1024;
+  if (cudaFuncSetAttribute((const void*)gemm_split_kernel<NN>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return TC_ERR_CUDA;
+  const int m_tiles = (M + BM - 1) / BM;
+  gemm_split_kernel<NN><<<batch * m_tiles, THREADS, smem, st>>>(mapA, mapB, out, M, K, m_tiles, status);
+  note_launch();
+  return TC_OK;
+}
+
+}  // namespace
+
+bool gemm_split_supported(int M, int NN, int K) {
+  if (M < 1 || K < 4 || (K & 3) != 0) return false;  // TMA rows are whole 16-byte vectors
+  return NN == 128 || NN == 144 || NN == 160 || NN == 192;
+}
+
+// C [batch][M][NN] = A B^T with A split [batch][2][M][K], B split [batch][2][NN][K].
+tc_status launch_gemm_split(const float* A, const float* B, int M, int NN, int K, int batch,
+                            float* C_plain, float* C_plainT, float* C_split, float* C_splitT,
+                            int32_t* status, cudaStream_t st, int cls) {
+  if (!gemm_split_supported(M, NN, K)) return TC_ERR_UNSUPPORTED;
+  CUtensorMap mapA, mapB;
+  if (!encode_panel(&mapA, A, M, K, batch, BM) || !encode_panel(&mapB, B, NN, K, batch, NN))
+    return TC_ERR_CUDA;
+  Out out{C_plain, C_plainT, C_split, C_splitT};
+  Scope scope_(cls, st);
+  switch (NN) {
+    case 128: return launch_nn<128>(mapA, mapB, out, M, K, batch, status, st);
+    case 144: return launch_nn<144>(mapA, mapB, out, M, K, batch, status, st);
+    case 160: return launch_nn<160>(mapA, mapB, out, M, K, batch, status, st);
+    case 192: return launch_nn<192>(mapA, mapB, out, M, K, batch, status, st);
+    default: return TC_ERR_UNSUPPORTED;
+  }
+}
+
+}  // namespace tc

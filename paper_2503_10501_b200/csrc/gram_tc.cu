@@ -17,13 +17,14 @@
 // round-to-nearest, while the tensor core already works on the other accumulator.
 // Only tiles on or below the diagonal are computed.  Every mbarrier wait is bounded: a wait
 // that runs out records an error for the image and the CTA winds down (TMEM is still freed).
-#include <cuda.h>
-
 #include "tc_internal.cuh"
+#include "tcgen05_util.cuh"
 
 namespace tc {
 
 namespace {
+
+using namespace t5;
 
 constexpr int TILE = 128;         // rows of O per operand tile = tile edge of G
 constexpr int BK = 64;            // K elements per stage: 64 halves = one 128-byte swizzle row
@@ -33,56 +34,6 @@ constexpr uint32_t TILE_BYTES = TILE * BK * 2;  // 16 KB
 constexpr uint32_t SMEM_BYTES = STAGES * 2 * TILE_BYTES + 1024;  // + alignment slack
 constexpr uint32_t TMEM_COLS = 256;  // two 128-column accumulators
 constexpr int DRAIN_KB = 2;          // stages per accumulation chunk (128 elements of K)
-constexpr uint32_t WAIT_LIMIT = 1u << 20;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-
-// Bounded wait: false when the phase did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y,
-                                            int z, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
-      : "memory");
-}
-
-// Shared-memory matrix descriptor: K-major tile, rows of 128 bytes, 128-byte swizzle; groups of
-// eight rows are 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address
-  d |= (uint64_t)(1024u >> 4) << 32;             // stride between 8-row groups
-  d |= (uint64_t)1 << 46;                        // descriptor version
-  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
-  return d;
-}
 
 // Instruction descriptor: D float32, A and B float16, both K-major, M = 128, N = 128.
 constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
@@ -96,32 +47,12 @@ __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t 
       : "memory");
 }
 
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
-        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-__global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CUtensorMap map,
+// lo_off = 0: G [image][N][N] plain float32 (img_stride = N N).  lo_off > 0: every entry goes
+// out as its two TF32 parts, the high one at G[...] and the low one lo_off floats further on.
+__global__ void __launch_bounds__(192, 2) gram_tc_kernel(const __grid_constant__ CUtensorMap map,
                                                      float* __restrict__ G, int N, int d,
-                                                     int tiles_per_image,
+                                                     int tiles_per_image, size_t img_stride,
+                                                     size_t lo_off,
                                                      int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[STAGES];
@@ -249,12 +180,41 @@ __global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CU
                      : "memory");
     }
     if (ok && s_fail == 0) {
-      float* Gb = G + (size_t)b * N * N;
+      float* Gb = G + (size_t)b * img_stride;
       const int row = ti * TILE + warp * 32 + lane;
       if (row < N) {
 #pragma unroll
         for (int q = 0; q < TILE / 32; ++q) {
           const int col0 = tj * TILE + q * 32;
+          if (lo_off != 0) {
+            // the two TF32 planes the tensor-core products of the subspace solve read: the low
+            // parts go out here, four at a time, and the high parts take the place of the values
+            const bool vec = col0 + 32 <= N && (N & 3) == 0;
+#pragma unroll
+            for (int j4 = 0; j4 < 8; ++j4) {
+              float lo[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const float v = acc[q * 32 + 4 * j4 + u];
+                const float hi = tf32_round(v);
+                lo[u] = tf32_round(v - hi);
+                acc[q * 32 + 4 * j4 + u] = hi;
+              }
+              if (vec) {
+                *reinterpret_cast<float4*>(Gb + lo_off + (size_t)row * N + col0 + 4 * j4) =
+                    make_float4(lo[0], lo[1], lo[2], lo[3]);
+              } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                  if (col0 + 4 * j4 + u < N) Gb[lo_off + (size_t)row * N + col0 + 4 * j4 + u] = lo[u];
+              }
+              if (!diag) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                  if (col0 + 4 * j4 + u < N) Gb[lo_off + (size_t)(col0 + 4 * j4 + u) * N + row] = lo[u];
+              }
+            }
+          }
           if (col0 + 32 <= N && (N & 3) == 0) {
             float4* dst = reinterpret_cast<float4*>(Gb + (size_t)row * N + col0);
 #pragma unroll
@@ -273,8 +233,14 @@ __global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CU
           }
         }
       }
-    } else if (status != nullptr && threadIdx.x == 0) {
-      atomicMax(&status[b], (int)TC_ERR_CUDA);
+    } else if (status != nullptr) {
+      if (threadIdx.x == 0) atomicMax(&status[b], (int)TC_ERR_CUDA);
+    } else {
+      // no status word to report to: the tile is marked with NaN instead of being left unwritten
+      const int row = ti * TILE + warp * 32 + lane;
+      if (row < N)
+        for (int j = 0; j < TILE; ++j)
+          if (tj * TILE + j < N) G[(size_t)b * img_stride + (size_t)row * N + tj * TILE + j] = __int_as_float(0x7fc00000);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -284,25 +250,6 @@ __global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CU
                  "r"(TMEM_COLS)
                  : "memory");
   }
-}
-
-typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                              CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                              CUtensorMapFloatOOBfill);
-
-encode_fn get_encode() {
-  static encode_fn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (encode_fn)p;
-  }
-  return fn;
 }
 
 }  // namespace
@@ -327,7 +274,9 @@ tc_status launch_gram_tc(const Dims& D, const void* O, float* G, int32_t* status
   const int nt = (D.N + TILE - 1) / TILE;
   const int tiles = nt * (nt + 1) / 2;
   Scope scope_(KC_GRAM, st);
-  gram_tc_kernel<<<D.B * tiles, 192, SMEM_BYTES, st>>>(map, G, D.N, D.d, tiles, status);
+  const size_t NN = (size_t)D.N * D.N;
+  gram_tc_kernel<<<D.B * tiles, 192, SMEM_BYTES, st>>>(map, G, D.N, D.d, tiles, D.tcp ? 2 * NN : NN,
+                                                       D.tcp ? NN : 0, status);
   note_launch();
   return TC_OK;
 }

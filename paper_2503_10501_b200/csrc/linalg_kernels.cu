@@ -1076,7 +1076,7 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
                                                            float* __restrict__ RinvT, int k_rt,
                                                            float shift_rel,
                                                            int32_t* __restrict__ status,
-                                                           int nparts) {
+                                                           int nparts, int split_out) {
   const int k = KT ? KT : k_rt;
   extern __shared__ __align__(16) float fsm[];
   __shared__ float s_red[16];
@@ -1347,7 +1347,19 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
     }
     __syncthreads();
   }
-  // RinvT[c][m] = X[m][c] for m <= c, zero otherwise
+  // RinvT[c][m] = X[m][c] for m <= c, zero otherwise; with split_out as the two TF32 planes
+  // [2][k][k] the tensor-core products read
+  if (split_out) {
+    float* out = RinvT + b * 2 * kk;
+    for (int e = tid; e < (int)kk; e += 512) {
+      const int c = e / k, mrow = e - c * k;
+      const float v = (mrow <= c) ? A[mrow * ld + c] : 0.f;
+      const float hi = tf32_round(v);
+      out[e] = hi;
+      out[kk + e] = tf32_round(v - hi);
+    }
+    return;
+  }
   float* out = RinvT + b * kk;
   for (int e = tid; e < (int)kk; e += 512) {
     const int c = e / k, mrow = e - c * k;
@@ -1540,7 +1552,8 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ u0g, float* __restrict__ u1g,
                                                          float* __restrict__ u2g, float* yg, float* __restrict__ mlg,
                                                          size_t ml_stride,
-                                                         int32_t* __restrict__ status, int nparts) {
+                                                         int32_t* __restrict__ status, int nparts,
+                                                         int split_out) {
   const int n = NT ? NT : n_rt;
   extern __shared__ __align__(16) float sm[];
   const int ld = n | 1;
@@ -2138,7 +2151,8 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     // ---------------- Z = Q Y:  ZT[p][i] = sum_j Q[i][j] Y[j][p] ----------------
     // thread = (four eigenvectors p, twelve rows i): per j one 16-byte load of Y (coalesced over
     // p) and twelve broadcast reads of Q from shared memory feed 48 multiply-adds
-    float* out = ZTg + img;
+    // with split_out ZT goes out as the two TF32 planes [2][n][n] the tensor-core product reads
+    float* out = ZTg + (split_out ? 2 * img : img);
     const bool vec = (n & 3) == 0;
     const int npg = (n + 3) >> 2, nrg = (n + 11) / 12;
     for (int w = tid; w < npg * nrg; w += 512) {
@@ -2177,7 +2191,15 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       for (int v = 0; v < 4; ++v) {
         if (p0 + v >= n) continue;
         float* orow = out + (size_t)(p0 + v) * n + i0;
-        if (vec && i0 + 12 <= n) {
+        if (split_out) {
+#pragma unroll
+          for (int u = 0; u < 12; ++u)
+            if (i0 + u < n) {
+              const float hi = tf32_round(acc[u][v]);
+              orow[u] = hi;
+              orow[(size_t)n * n + u] = tf32_round(acc[u][v] - hi);
+            }
+        } else if (vec && i0 + 12 <= n) {
 #pragma unroll
           for (int u = 0; u < 12; u += 4)
             *reinterpret_cast<float4*>(orow + u) =
@@ -2217,14 +2239,14 @@ constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared 
 static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
                           int max_sweeps, float rank_tol, float* scr1, float* scr2, float* scr3,
                           float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st,
-                          int nparts = 1) {
+                          int nparts = 1, int split_out = 0) {
   Scope scope_(KC_JACOBI, st);
   {
     const size_t tri = ((size_t)n * (n | 1) + 27 * (size_t)((n + 3) & ~3)) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       auto go = [&](auto kernel) {
         cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
-        { kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts); note_launch(); }
+        { kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts, split_out); note_launch(); }
       };
       switch (n) {
         case 128: go(tridiag_eig_kernel<128>); break;
@@ -2253,13 +2275,14 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
 }
 
 static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
-                            float shift_rel, int32_t* status, cudaStream_t st, int nparts) {
+                            float shift_rel, int32_t* status, cudaStream_t st, int nparts,
+                            int split_out = 0) {
   Scope scope_(KC_CHOL, st);
   const size_t fast = ((size_t)k * (k | 1) + (size_t)CNB * k + (size_t)(k / CNB) * CNB * CNB) * sizeof(float);
   if (k % CNB == 0 && k >= CNB && fast <= SMEM_LIMIT) {
     auto go = [&](auto kernel) {
       cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast);
-      { kernel<<<batch, 512, fast, st>>>(S, RinvT, k, shift_rel, status, nparts); note_launch(); }
+      { kernel<<<batch, 512, fast, st>>>(S, RinvT, k, shift_rel, status, nparts, split_out); note_launch(); }
     };
     switch (k) {
       case 128: go(chol_inv_fast_kernel<128>); break;
@@ -2284,6 +2307,55 @@ static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, i
   if (use_smem)
     cudaFuncSetAttribute((const void*)chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   { chol_inv_kernel<<<batch, 512, smem, st>>>(S, RinvT, Rwork, k, shift_rel, use_smem, status); note_launch(); }
+}
+
+// ==========================================================================================
+// A float32 matrix as the two TF32 planes the tensor-core products read, row-major and / or
+// transposed:  in [R][C]  ->  split [2][R][C], splitT [2][C][R]  (per image).
+// 32 x 32 tiles through shared memory so that both forms are written along their rows.
+// grid (C tiles, R tiles, batch), block (32, 8).
+// ==========================================================================================
+__global__ void __launch_bounds__(256) split_panel_kernel(const float* __restrict__ in, int R, int C,
+                                                         float* __restrict__ split,
+                                                         float* __restrict__ splitT) {
+  __shared__ float th[32][33], tl[32][33];
+  const int b = blockIdx.z, r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const size_t RC = (size_t)R * C;
+  const float* src = in + (size_t)b * RC;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = r0 + ty + 8 * i, c = c0 + tx;
+    float hi = 0.f, lo = 0.f;
+    if (r < R && c < C) {
+      const float v = src[(size_t)r * C + c];
+      hi = tf32_round(v);
+      lo = tf32_round(v - hi);
+      if (split != nullptr) {
+        split[(size_t)b * 2 * RC + (size_t)r * C + c] = hi;
+        split[(size_t)b * 2 * RC + RC + (size_t)r * C + c] = lo;
+      }
+    }
+    th[ty + 8 * i][tx] = hi;
+    tl[ty + 8 * i][tx] = lo;
+  }
+  if (splitT == nullptr) return;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int c = c0 + ty + 8 * i, r = r0 + tx;
+    if (r < R && c < C) {
+      splitT[(size_t)b * 2 * RC + (size_t)c * R + r] = th[tx][ty + 8 * i];
+      splitT[(size_t)b * 2 * RC + RC + (size_t)c * R + r] = tl[tx][ty + 8 * i];
+    }
+  }
+}
+
+void launch_split_panel(const float* in, int R, int C, int batch, float* split, float* splitT,
+                        cudaStream_t st, int cls) {
+  Scope scope_(cls, st);
+  dim3 grid((C + 31) / 32, (R + 31) / 32, batch), block(32, 8);
+  { split_panel_kernel<<<grid, block, 0, st>>>(in, R, C, split, splitT); note_launch(); }
 }
 
 // ==========================================================================================
@@ -2375,9 +2447,9 @@ void fill_i32(int32_t* p, int n, int v, cudaStream_t st) {
 // ==========================================================================================
 // The whole of Eq. 3-5 / 3-6 for a batch, given G in the workspace.
 // ==========================================================================================
-void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
-                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
-                float* full_scratch, cudaEvent_t g_ready) {
+tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
+                     float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
+                     float* full_scratch, cudaEvent_t g_ready) {
   // D.B images starting at image b0 of the workspace arrays; O and the outputs already point at
   // image b0.
   const int B = D.B, N = D.N, k = D.k;
@@ -2400,18 +2472,9 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)N * sizeof(float), st>>>(
           theta, ZT, C_out, sigma_out, rank_out, img_status, N, N, q, D.rank_tol, 1); note_launch(); }
-    return;
+    return TC_OK;
   }
-  float* Y0 = (float*)(ws + P.Y0) + b0 * sY;
-  float* Y1 = (float*)(ws + P.Y1) + b0 * sY;
-  float* Y2 = (float*)(ws + P.Y2) + b0 * sY;
-  const int parts = tn_parts(k);  // the k x k products come in this many parts per image
-  float* Sm = (float*)(ws + P.Sm) + b0 * sK * parts;
-  float* Rinv = (float*)(ws + P.Rinv) + b0 * sK;
-  float* Hm = (float*)(ws + P.Hm) + b0 * sK * parts;
-
-  // 1. sketch of the column space of O
-  {
+  auto sketch_into = [&](float* Y0) {
     Scope scope_(KC_SKETCH, st);
     const int L = D.f16 ? 8 : 4;
     if (k % L == 0 && k / L <= 256 && (size_t)D.d * sizeof(float) <= 48 * 1024) {
@@ -2431,7 +2494,70 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
       else
         { sketch_kernel<float><<<grid, threads, 0, st>>>((const float*)O, Y0, N, D.d, k); note_launch(); }
     }
+  };
+  if (D.tcp) {
+    // ---- the products on the tensor cores, operands as split TF32 panels (gemm_split.cu) ----
+    // Two sets of panels, each held row-major [B][2][N][k] and transposed [B][2][k][N].
+    float* PAr = (float*)(ws + P.PA) + b0 * 2 * sY;
+    float* PAt = (float*)(ws + P.PA) + (size_t)P.panel_T_off / sizeof(float) + b0 * 2 * sY;
+    float* PBr = (float*)(ws + P.PB) + b0 * 2 * sY;
+    float* PBt = (float*)(ws + P.PB) + (size_t)P.panel_T_off / sizeof(float) + b0 * 2 * sY;
+    float* Sk = (float*)(ws + P.Sk) + b0 * sK;
+    float* Hk = (float*)(ws + P.Hk) + b0 * sK;
+    float* RinvS = (float*)(ws + P.RinvS) + b0 * 2 * sK;
+    float* ZTs = (float*)(ws + P.ZTs) + b0 * 2 * sK;
+    float* Es = (float*)(ws + P.Es) + b0 * 5 * sK;
+    const float* Gs = (const float*)(ws + P.G) + b0 * 2 * sG;
+    int32_t* stp = img_status;
+    // 1. sketch (plain, in the room of set B, which is free until the first pass writes it)
+    sketch_into(PBr);
+    launch_split_panel(PBr, N, k, B, PAr, PAt, st, KC_SKETCH);
+    // one Cholesky-QR pass  dst = src R^{-1}  with  R^T R = src^T src + shift
+    tc_status err = TC_OK;
+    auto mm = [&](const float* A_, const float* B_, int M_, int K_, float* c0, float* c1, float* c2,
+                  float* c3, int cls) {
+      if (err == TC_OK) err = launch_gemm_split(A_, B_, M_, k, K_, B, c0, c1, c2, c3, stp, st, cls);
+    };
+    auto pass = [&](const float* srcR, const float* srcT, float* dstR, float* dstT, float shift_rel) {
+      mm(srcT, srcT, k, N, Sk, nullptr, nullptr, nullptr, KC_GEMM_TN);
+      if (err != TC_OK) return;
+      launch_chol_inv(Sk, RinvS, nullptr, k, B, shift_rel, stp, st, 1, 1);
+      mm(srcR, RinvS, N, k, nullptr, nullptr, dstR, dstT, KC_GEMM);
+    };
+    // 2. a well-conditioned basis Q0 of the sketch
+    pass(PAr, PAt, nullptr, PBt, 1e-6f);
+    // 3. Y1 = G Q0, then two passes: the first (shifted) brings the condition number from ~1e7
+    //    down to ~1e3, the second leaves a basis whose departure from orthonormality lies in the
+    //    directions under the rank cut-off; the Ritz values above it are unaffected
+    if (g_ready) cudaStreamWaitEvent(st, g_ready, 0);
+    mm(Gs, PBt, N, N, nullptr, nullptr, PAr, PAt, KC_GEMM_GQ);
+    pass(PAr, PAt, PBr, PBt, 1e-6f);
+    pass(PBr, PBt, PAr, PAt, 1e-7f);  // Q1 in set A
+    // 4. Rayleigh-Ritz:  T = G Q1 (kept transposed),  H = Q1^T T
+    mm(Gs, PAt, N, N, nullptr, nullptr, nullptr, PBt, KC_GEMM_GQ);
+    mm(PAt, PBt, k, N, Hk, nullptr, nullptr, nullptr, KC_GEMM_TN);
+    if (err != TC_OK) return err;
+    launch_jacobi(Hk, Es, ZTs, theta, k, B, D.max_sweeps, D.rank_tol, Es + (size_t)B * sK,
+                  Es + 2 * (size_t)B * sK, Es + 3 * (size_t)B * sK, Es + 4 * (size_t)B * sK, sK, stp, st, 1, 1);
+    // 5. PT[p][x] = sum_i ZT[p][i] Q1[x][i]: the product Q1 ZT^T written transposed
+    float* PT = PBr;
+    mm(PAr, ZTs, N, k, nullptr, PT, nullptr, nullptr, KC_GEMM);
+    if (err != TC_OK) return err;
+    Scope scope_(KC_ICS, st);
+    { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
+          theta, PT, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0); note_launch(); }
+    return TC_OK;
   }
+  float* Y0 = (float*)(ws + P.Y0) + b0 * sY;
+  float* Y1 = (float*)(ws + P.Y1) + b0 * sY;
+  float* Y2 = (float*)(ws + P.Y2) + b0 * sY;
+  const int parts = tn_parts(k);  // the k x k products come in this many parts per image
+  float* Sm = (float*)(ws + P.Sm) + b0 * sK * parts;
+  float* Rinv = (float*)(ws + P.Rinv) + b0 * sK;
+  float* Hm = (float*)(ws + P.Hm) + b0 * sK * parts;
+
+  // 1. sketch of the column space of O
+  sketch_into(Y0);
   // one Cholesky-QR pass: dst = src R^{-1},  R^T R = src^T src (+ shift)
   auto cholqr_pass = [&](const float* src, float* dst, float shift_rel) {
     gemm_tn_sym(src, src, Sm, k, N, sY, sY, B, st, KC_GEMM_TN);
@@ -2459,6 +2585,7 @@ void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, f
   Scope scope_(KC_ICS, st);
   { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
         theta, Y0, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0); note_launch(); }
+  return TC_OK;
 }
 
 }  // namespace tc

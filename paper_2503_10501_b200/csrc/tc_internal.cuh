@@ -15,6 +15,7 @@ struct Dims {
   int keep, M, P, nA, nB;
   int k;          // dimension of the decomposed subspace: rank_cap, or N for the full solve
   bool full;      // rank_cap == 0
+  bool tcp;       // the subspace solve runs its products on the tensor cores (split panels)
   int esz;        // bytes per element of O, A, X, K, V
   bool f16;
   int chunks;     // row chunks of the attention column-mean
@@ -37,10 +38,25 @@ struct Plan {
   size_t setA, setB, best_val, best_dst, msrc, mdst, kept;  // int32 / f32 lists
   size_t rank;     // [B] int32
   size_t flags;    // [B] int32 device status scratch
+  // tensor-core subspace solve (Dims::tcp): G is then two TF32 planes [B][2][N][N], and
+  size_t PA, PB;   // two sets of split panels: [B][2][N][k] row-major, then, panel_T_off bytes
+                   // further on, [B][2][k][N] transposed
+  size_t panel_T_off;
+  size_t Gplain;   // [B][N][N] f32, only for float32 inputs (their Gram matrix is split afterwards)
+  size_t Sk, Hk;   // [B][k][k] f32: Y^T Y and the projected matrix
+  size_t RinvS, ZTs;  // [B][2][k][k] split: R^{-T} and the eigenvectors of the projection
+  size_t Es;       // [B][5][k][k] f32 scratch of the tridiagonal solver
   size_t total;
 };
 
 Plan make_plan(const Dims& D);
+
+// value rounded to the nearest TF32 (low 13 mantissa bits zero)
+__device__ __forceinline__ float tf32_round(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return __uint_as_float(r);
+}
 
 // Number of parts per image in which the k x k products of the subspace solve are stored
 // (partial sums over chunks of the long dimension, added up by the kernel that reads them).
@@ -74,6 +90,7 @@ void launch_combine(const Dims& D, const float* s_part, const float* C, float* S
 // Stage I prune + Eq. 3-9 split.
 void launch_prune(const Dims& D, const float* E, int32_t* setA, int32_t* setB, cudaStream_t st);
 // Eq. 3-10 best match per Set-B token, from the Gram matrix or from the rows of O.
+// (with Dims::tcp, G is the pair of TF32 planes and an entry is the sum of its two parts)
 void launch_match_gram(const Dims& D, const float* G, const int32_t* setA, const int32_t* setB,
                        float* best_val, int32_t* best_dst, cudaStream_t st);
 void launch_match_rows(const Dims& D, const void* O, const int32_t* setA, const int32_t* setB,
@@ -95,16 +112,27 @@ void fill_i32(int32_t* p, int n, int v, cudaStream_t st);
 void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, const void* Xo,
                        const int32_t* kept, void* Ho, int32_t* pos, cudaStream_t st);
 
-// G = O O^T (float32 out).
-tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
+// G = O O^T (float32 out; with Dims::tcp as two TF32 planes [B][2][N][N]).
+tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st,
+                      float* Gplain);
+
+// C = A B^T on the tensor cores from split panels (A [batch][2][M][K], B [batch][2][NN][K]);
+// any of the four output forms may be null.
+bool gemm_split_supported(int M, int NN, int K);
+tc_status launch_gemm_split(const float* A, const float* B, int M, int NN, int K, int batch,
+                            float* C_plain, float* C_plainT, float* C_split, float* C_splitT,
+                            int32_t* status, cudaStream_t st, int cls);
+// in [batch][R][C] float32 -> split [batch][2][R][C] and / or splitT [batch][2][C][R]
+void launch_split_panel(const float* in, int R, int C, int batch, float* split, float* splitT,
+                        cudaStream_t st, int cls);
 
 // Eigen-decomposition of G and Eq. 3-6:  C, theta (unsorted), then sorted sigma / rank.
 // g_ready: optional event after which G is complete when it is built on another stream (the
 // subspace solve waits for it in front of its first product with G).
 // full_scratch: optional 4 * B * N * N floats; with it a full solve (rank_cap = 0) of a matrix
 // that fits in shared memory goes through the tridiagonal solver instead of Jacobi sweeps.
-void launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
-                float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
-                float* full_scratch = nullptr, cudaEvent_t g_ready = nullptr);
+tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void* O, float* C_out,
+                     float* sigma_out, int32_t* rank_out, int32_t* img_status, cudaStream_t st,
+                     float* full_scratch = nullptr, cudaEvent_t g_ready = nullptr);
 
 }  // namespace tc

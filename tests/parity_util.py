@@ -44,6 +44,74 @@ def check_scores(g: Dict[str, np.ndarray], o: Dict[str, np.ndarray], rank_tol: f
     assert rel_err(g["E"], o["E"]) <= REL_SCORE, ("E", rel_err(g["E"], o["E"]))
 
 
+def band_population(E_or: np.ndarray, P: int, nA: int) -> int:
+    """How many tokens sit inside the 1e-3 band around the two cuts (Stage-I cut and A/B cut):
+    the tokens for which "exact outside the band" says nothing."""
+    N = len(E_or)
+    E32 = np.asarray(E_or, np.float64).astype(np.float32).astype(np.float64)
+    order = orc.descending_order(E_or)
+    inside = np.zeros(N, bool)
+    for c in (nA, P):
+        if 0 < c < N:
+            v = 0.5 * (E32[order[c - 1]] + E32[order[c]])
+            inside |= np.abs(E32 - v) <= REL_SCORE * abs(v)
+    return int(inside.sum())
+
+
+def cut_gaps(E_or: np.ndarray, P: int, nA: int):
+    """Relative gap of the float32-rounded oracle scores across the A/B cut and the Stage-I cut."""
+    N = len(E_or)
+    E32 = np.asarray(E_or, np.float64).astype(np.float32).astype(np.float64)
+    order = orc.descending_order(E_or)
+    gaps = []
+    for c in (nA, P):
+        if 0 < c < N:
+            hi, lo = E32[order[c - 1]], E32[order[c]]
+            gaps.append((hi - lo) / max(abs(hi), 1e-300))
+    return gaps
+
+
+def open_score_gaps(O: np.ndarray, A: np.ndarray, cfgp: dict, min_gap: float = 3e-3,
+                    near: float = 2.5e-3, step: float = 4e-3, max_pass: int = 6) -> np.ndarray:
+    """Test-side conditioning of one image's O (storage dtype in, storage dtype out): rows whose
+    oracle score lies within `near` (relative) of the Stage-I cut or of the A/B cut (Sec. 3.3.1
+    last paragraph, Eq. 3-9) are scaled by (1 + step) when they are above the cut and by
+    (1 - step) when below, bit-identical rows together so that twins stay twins, then rounded
+    to the storage type again; repeated until both gaps exceed `min_gap`.  Scaling a row of O
+    scales its information contribution (Eq. 3-6) by nearly the same factor.  Returns the new O;
+    raises if the gaps cannot be opened."""
+    O = np.array(O, copy=True)
+    N = O.shape[0]
+    M, P, nA, nB = orc.resolve_counts(N, cfgp["keep"], cfgp["rho"], cfgp.get("n_merge", -1))
+    # groups of bit-identical rows
+    keys = {}
+    for x in range(N):
+        keys.setdefault(O[x].tobytes(), []).append(x)
+    group_of = {x: g for g in keys.values() for x in g}
+    for _ in range(max_pass):
+        o = oracle_scores(cfgp, O, A)
+        if min(cut_gaps(o["E"], P, nA), default=1.0) >= min_gap:
+            return O
+        E32 = np.asarray(o["E"], np.float64).astype(np.float32).astype(np.float64)
+        order = orc.descending_order(o["E"])
+        pos = np.empty(N, int)
+        pos[order] = np.arange(N)
+        done = set()
+        for c in (nA, P):
+            if not 0 < c < N:
+                continue
+            v = 0.5 * (E32[order[c - 1]] + E32[order[c]])
+            for x in np.nonzero(np.abs(E32 - v) <= near * abs(v))[0]:
+                if int(x) in done:
+                    continue
+                up = pos[x] < c
+                f = (1.0 + step) if up else (1.0 - step)
+                for y in group_of[int(x)]:
+                    O[y] = (O[y].astype(np.float64) * f).astype(O.dtype)
+                    done.add(y)
+    raise AssertionError("score gaps could not be opened")
+
+
 def check_sets(E_or: np.ndarray, setA_g, setB_g, P: int, nA: int) -> int:
     """Exact agreement outside the unresolvable band; returns the number of in-band flips."""
     N = len(E_or)
@@ -155,4 +223,5 @@ def check_image(cfgp: dict, im: Dict[str, np.ndarray], g: Dict[str, np.ndarray],
                               g["dst"], g["kept"], cfgp["keep"])
     check_compact(im["X"], im.get("K"), im.get("V"), g["kept"], g["src"], g["dst"], g["Xo"],
                   g.get("Ko"), g.get("Vo"))
-    return {"flips_sets": flips_sets, "flips_merge": flips_merge}
+    return {"flips_sets": flips_sets, "flips_merge": flips_merge,
+            "in_band": band_population(o["E"], P, nA)}

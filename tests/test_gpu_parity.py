@@ -59,7 +59,11 @@ def cfgp_of(p):
                 score_norm=p.score_norm)
 
 
-def check_config(cfg, images, with_kv=True, **over):
+def check_config(cfg, images, with_kv=True, max_flips=0, **over):
+    """Staged and fused calls on the configuration, sampled images against the oracle.
+    max_flips: how many tokens in all may sit on the other side of a cut than in the oracle
+    (always inside the band the float32 scores cannot resolve, see parity_util); the count of
+    tokens inside the band is printed so that the weight of "exact outside the band" shows."""
     p = params_of(cfg, **over)
     batch = inputs.make_batch(cfg)
     res = run_staged(p, batch, with_kv)
@@ -70,14 +74,17 @@ def check_config(cfg, images, with_kv=True, **over):
     assert np.array_equal(res["cX"], res["Xo"])
     if with_kv:
         assert np.array_equal(res["cK"], res["Ko"]) and np.array_equal(res["cV"], res["Vo"])
-    flips = {"flips_sets": 0, "flips_merge": 0}
+    flips = {"flips_sets": 0, "flips_merge": 0, "in_band": 0}
     for b in images:
         im = {k: batch[k][b] for k in batch}
         if not with_kv:
             im.pop("K"), im.pop("V")
         f = pu.check_image(cfgp_of(p), im, image_slice(res, b, with_kv))
+        print(f"{cfg.name} image {b}: tokens inside the score band {f['in_band']}, "
+              f"flips at the score cuts {f['flips_sets']}, in the matching {f['flips_merge']}")
         for k in f:
             flips[k] += f[k]
+    assert flips["flips_sets"] + flips["flips_merge"] <= max_flips, flips
     return flips
 
 
@@ -113,7 +120,7 @@ def test_medium_ragged(rank_cap):
     cfg = inputs.tiny_config(n_tokens=200, d_model=264, n_heads=3, head_dim=24, n_query=37, keep=61,
                              rank=40, dtype="f16", batch=5, seed=23, noise=0.01, tau=2.0,
                              rank_tol=2e-3, dup_frac=0.05)
-    check_config(cfg, range(5), rank_cap=rank_cap)
+    check_config(cfg, range(5), rank_cap=rank_cap, max_flips=2)
 
 
 def test_maximum_token_count():
@@ -122,7 +129,7 @@ def test_maximum_token_count():
     cfg = inputs.tiny_config(n_tokens=4096, d_model=256, n_heads=2, head_dim=64, n_query=8,
                              keep=512, rank=48, dtype="f16", batch=1, seed=31, noise=0.01, tau=2.0,
                              rank_tol=2e-3)
-    check_config(cfg, [0], rank_cap=64)
+    check_config(cfg, [0], rank_cap=64, max_flips=4)
 
 
 # ------------------------------------------------------------------ selection kernels alone
@@ -165,24 +172,24 @@ def test_merge_duplicate_rows_tie_to_lower_index():
 @pytest.mark.parametrize("lam,norm", [(0.5, "none"), (0.5, "sum1"), (0.0, "none"), (1.0, "none")])
 def test_cfg1_single_f32(lam, norm):
     cfg = inputs.CONFIGS["cfg1_single_f32"]
-    check_config(cfg, [0], lam=lam, score_norm=norm)
+    check_config(cfg, [0], lam=lam, score_norm=norm, max_flips=1)
 
 
 @pytest.mark.parametrize("lam,norm", [(0.5, "none"), (0.5, "sum1"), (0.0, "none"), (1.0, "none")])
 def test_cfg2_llava7b(lam, norm):
     cfg = inputs.CONFIGS["cfg2_llava7b_f16"]
-    check_config(cfg, [0, 7, 15], lam=lam, score_norm=norm)
+    check_config(cfg, [0, 7, 15], lam=lam, score_norm=norm, max_flips=2)
 
 
 @pytest.mark.parametrize("norm", ["none", "sum1"])
 def test_cfg3_llava13b(norm):
     cfg = inputs.CONFIGS["cfg3_llava13b_f16"]
-    check_config(cfg, [1, 14], score_norm=norm)
+    check_config(cfg, [1, 14], score_norm=norm, max_flips=2)
 
 
 def test_cfg2_full_solve_agrees():
     cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=2)
-    check_config(cfg, [0, 1], rank_cap=0)
+    check_config(cfg, [0, 1], rank_cap=0, max_flips=2)
 
 
 def test_rank_cap_too_small_is_reported():
@@ -219,10 +226,8 @@ def test_gram_f16_against_float64(B, N, d):
 def test_cfg5_bench_point_sampled_images():
     # the launch configuration bench.py times: 64 images, T = 128, keep = 128
     cfg = inputs.CONFIGS["cfg5_sweep_f16"]
-    flips = check_config(cfg, [0, 31, 63])
-    assert flips["flips_sets"] <= 2 and flips["flips_merge"] <= 2, flips
-    flips = check_config(cfg, [17, 50], score_norm="sum1")
-    assert flips["flips_sets"] <= 2 and flips["flips_merge"] <= 2, flips
+    check_config(cfg, [0, 31, 63], max_flips=2)
+    check_config(cfg, [17, 50], score_norm="sum1", max_flips=2)
 
 
 def test_cfg5_bench_point_in_the_bench_launch_mode():
@@ -261,12 +266,20 @@ def test_cfg5_bench_point_in_the_bench_launch_mode():
     for a, b in zip(plain, replay):
         assert np.array_equal(a, b)
     assert not replay[4].any()
-    # kept indices and merged rows of sampled images against the oracle's compaction
+    # sampled images of the replay against the oracle, stage by stage: the lists the staged
+    # entry points give on the same inputs (bit-identical kept_idx was asserted above) and the
+    # replay's own X', K', V'
+    sc = tcb.tc_score(p, d["O"], d["A"], ws)
+    setA, setB = tcb.tc_prune(p, sc["E"], ws)
+    src, dst, kept = tcb.tc_merge(p, d["O"], setA, setB, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(host(kept), replay[3])
     for b in (5, 40):
-        o = pu.oracle_scores(cfgp_of(p), batch["O"][b], batch["A"][b])
-        M, P, nA, nB = orc.resolve_counts(cfg.n_tokens, cfg.keep, cfg.rho, -1)
-        order = orc.descending_order(o["E"])
-        assert len(set(replay[3][b].tolist()) - set(int(t) for t in order[:P + 4])) <= 2
+        g = {k: host(sc[k])[b] for k in ("E", "C", "S", "sigma", "rank")}
+        g.update(setA=host(setA)[b], setB=host(setB)[b], src=host(src)[b], dst=host(dst)[b],
+                 kept=replay[3][b], Xo=replay[0][b], Ko=replay[1][b], Vo=replay[2][b])
+        f = pu.check_image(cfgp_of(p), {k: batch[k][b] for k in batch}, g)
+        assert f["flips_sets"] + f["flips_merge"] <= 2, f
 
 
 def test_cfg5_bench_point_properties_of_every_image():
@@ -323,13 +336,58 @@ def test_cfg5_bench_point_properties_of_every_image():
 @pytest.mark.parametrize("T,keep", [(32, 64), (512, 288)])
 def test_cfg5_sweep_corners(T, keep):
     cfg = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=8, n_query=T, keep=keep)
-    check_config(cfg, [0, 7])
+    check_config(cfg, [0, 7], max_flips=2)
 
 
 @pytest.mark.parametrize("norm,image", [("none", 2), ("sum1", 1)])
 def test_cfg4_anyres(norm, image):
     cfg = inputs.CONFIGS["cfg4_anyres_f16"]
-    check_config(cfg, [image], score_norm=norm)
+    check_config(cfg, [image], score_norm=norm, max_flips=4)
+
+
+# ------------------------------------------------------------------ inputs with a gap at the cuts
+@pytest.mark.parametrize("name,nb", [("cfg2_llava7b_f16", 4), ("cfg5_sweep_f16", 6)])
+def test_gapped_scores_give_the_oracle_lists_bit_for_bit(name, nb):
+    # The scores of the synthetic images are dense around the cuts (several tokens within 1e-3 of
+    # the Stage-I cut and of the A/B cut of Eq. 3-9), where float32 cannot be asked to agree with
+    # float64.  Here the rows next to a cut are rescaled by the test (oracle side only, see
+    # parity_util.open_score_gaps) until both cuts have a gap of 3e-3: then Set A, Set B must be
+    # the oracle's exactly, and so must merge_src, merge_dst and kept_idx unless two
+    # similarities of Eq. 3-10 that decide a choice are closer than 1e-4 and not identical.
+    cfg = inputs.CONFIGS[name].with_(batch=nb)
+    p = params_of(cfg)
+    cfgp = cfgp_of(p)
+    batch = inputs.make_batch(cfg)
+    for b in range(nb):
+        batch["O"][b] = pu.open_score_gaps(batch["O"][b], batch["A"][b], cfgp)
+    res = run_staged(p, batch)
+    assert not res["img_status"].any() and not res["cstatus"].any()
+    assert np.array_equal(res["ckept"], res["kept"])
+    M, P, nA, nB = tcb.tc_counts(p)
+    exact_images = 0
+    for b in range(nb):
+        im = {k: batch[k][b] for k in batch}
+        f = pu.check_image(cfgp, im, image_slice(res, b))
+        assert f["in_band"] == 0 and f["flips_sets"] == 0, f
+        o = orc.carve(im["O"].astype(np.float64), im["A"].astype(np.float64), im["X"], im["K"],
+                      im["V"], cfg.keep, cfg.rho, cfg.lam, cfg.rank_tol, "none")
+        assert res["setA"][b].tolist() == sorted(o["setA"].tolist())
+        assert res["setB"][b].tolist() == sorted(o["setB"].tolist())
+        # similarities that decide something: the merge cut and each merged token's best two
+        sim = orc.similarity(im["O"].astype(np.float64), sorted(o["setA"].tolist()), sorted(o["setB"].tolist()))
+        best = np.sort(sim.max(axis=1))[::-1]
+        tight = M < nB and best[M - 1] - best[M] <= pu.SIM_BAND
+        top2 = np.sort(sim, axis=1)[:, -2:]
+        rows_tight = (top2[:, 1] - top2[:, 0] <= pu.SIM_BAND) & (top2[:, 1] != top2[:, 0])
+        if not tight and not rows_tight.any():
+            order = np.argsort(o["merge_src"])
+            assert res["src"][b].tolist() == o["merge_src"][order].tolist()
+            assert res["dst"][b].tolist() == o["merge_dst"][order].tolist()
+            assert res["kept"][b].tolist() == o["kept_idx"].tolist()
+            assert f["flips_merge"] == 0
+            exact_images += 1
+    print(f"{name}: {exact_images} of {nb} images compared bit for bit with the unconditioned oracle")
+    assert exact_images >= 1
 
 
 # ------------------------------------------------------------------ Sec. 3.2: rank of a token set

@@ -21,7 +21,7 @@ def _params(**kw):
 def test_library_exports_every_declared_symbol():
     lib = tcb.lib()
     header = open(os.path.join(ROOT, "include", "tokencarve.h")).read()
-    declared = set(re.findall(r"\b(tc_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(tc_[a-z0-9_]+)\s*\(", header))
     assert declared == set(tcb.EXPORTS)
     for name in declared:
         assert getattr(lib, name) is not None

@@ -1,4 +1,4 @@
-"""tc_attn_score_noalloc against tc_score's S.
+"""tc_attn_score_noalloc against tc_score's S and against the oracle's Eq. 3-7.
 
 The entry point exists for callers that cannot allocate device memory where they need the
 attention scores (a plug-in inside someone else's forward pass, a latency-bound serving loop, a
@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import ipgs_oracle as orc
 from paper_2503_10501_b200 import binding as tcb
 from paper_2503_10501_b200 import inputs
 
@@ -52,6 +53,9 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
         got = S.cpu().numpy()
         assert np.all(np.isfinite(got))
         np.testing.assert_allclose(got, want, rtol=1e-3, atol=0)
+        for b in range(p.batch):                  # and Eq. 3-7 itself, in float64
+            ref = orc.attention_score(batch["A"][b].astype(np.float64))
+            np.testing.assert_allclose(got[b], ref, rtol=1e-3, atol=0)
     # and once more for the first problem, after the array has held the second one's sums
     p, batch, A, S = runs[0]
     S.fill_(float("nan"))
