@@ -194,17 +194,15 @@ tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream);
 /*
  * The product kernel of the subspace solve behind Eq. 3-5 / 3-6 (Sec. 3.3.1), exposed for
  * inspection: C [batch][M][NN] = A B^T for float32 A [batch][M][K] and B [batch][NN][K] (device,
- * row-major, 16-byte aligned), computed on the tensor cores with every operand carried as two
+ * row-major, 16-byte aligned), computed on the tensor cores with every operand value used as two
  * TF32 numbers (three products per term, float32 accumulation), so that the result is as good
- * as a float32 product.  CT, when not NULL, also receives the transposed result
- * [batch][NN][M].  NN is 128, 144, 160 or 192 and K a multiple of 4, else TC_ERR_UNSUPPORTED.
- * ws: device scratch of at least tc_matmul_f32x3_workspace_bytes(batch, M, NN, K) bytes.
- * img_status [batch] (may be NULL) receives TC_ERR_CUDA for an image whose tile pipeline gave up.
+ * as a float32 product.  C and / or CT (the transposed result [batch][NN][M]) are written;
+ * either may be NULL, not both.  NN is 128, 144, 160 or 192 and K a multiple of 4, else
+ * TC_ERR_UNSUPPORTED.  img_status [batch] (may be NULL) receives TC_ERR_CUDA for an image whose
+ * tile pipeline gave up.  Allocates nothing, only enqueues.
  */
-size_t tc_matmul_f32x3_workspace_bytes(int32_t batch, int32_t M, int32_t NN, int32_t K);
 tc_status tc_matmul_f32x3(const float* A, const float* B, float* C, float* CT, int32_t batch,
-                          int32_t M, int32_t NN, int32_t K, int32_t* img_status, void* ws,
-                          size_t ws_bytes, void* stream);
+                          int32_t M, int32_t NN, int32_t K, int32_t* img_status, void* stream);
 
 /*
  * Sec. 3.2 ("Visual Token Information") and the appendix "Attention Output Matrix Rank": the

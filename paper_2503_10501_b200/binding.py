@@ -27,8 +27,7 @@ EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge"
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
            "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
-           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3",
-           "tc_matmul_f32x3_workspace_bytes")
+           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3")
 
 
 class TcParams(C.Structure):
@@ -76,8 +75,7 @@ def lib() -> C.CDLL:
         L.tc_rank.argtypes = [pp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         L.tc_reassemble.argtypes = [pp, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp]
         L.tc_gram.argtypes = [pp, vp, vp, vp]
-        L.tc_matmul_f32x3_workspace_bytes.argtypes = [C.c_int32] * 4
-        L.tc_matmul_f32x3.argtypes = [vp, vp, vp, vp] + [C.c_int32] * 4 + [vp, vp, sz, vp]
+        L.tc_matmul_f32x3.argtypes = [vp, vp, vp, vp] + [C.c_int32] * 4 + [vp, vp]
         L.tc_set_groups.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
         L.tc_status_string.argtypes = [C.c_int32]
@@ -86,11 +84,9 @@ def lib() -> C.CDLL:
         L.tc_kernel_class_name.restype = C.c_char_p
         L.tc_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int32]
         for name in EXPORTS:
-            if name not in ("tc_status_string", "tc_kernel_class_name", "tc_attn_score_noalloc",
-                            "tc_set_groups", "tc_matmul_f32x3_workspace_bytes"):
+            if name not in ("tc_status_string", "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups"):
                 getattr(L, name).restype = C.c_int32
         L.tc_launch_count.restype = C.c_int64
-        L.tc_matmul_f32x3_workspace_bytes.restype = sz
         _lib = L
     return _lib
 
@@ -176,21 +172,19 @@ def tc_gram(p: Params, O: torch.Tensor) -> torch.Tensor:
 
 
 def tc_matmul_f32x3(A: torch.Tensor, B: torch.Tensor, transposed: bool = False):
-    """C = A B^T per image for float32 A [batch, M, K], B [batch, NN, K] through the split-TF32
-    tensor-core kernel; returns (C, CT or None, img_status)."""
+    """C = A B^T per image for float32 A [batch, M, K], B [batch, NN, K] through the three-product
+    TF32 tensor-core kernel; returns (C, CT or None, img_status)."""
     assert A.dtype == torch.float32 and B.dtype == torch.float32 and A.is_contiguous() and B.is_contiguous()
     batch, M, K = A.shape
     NN = B.shape[1]
     assert B.shape[0] == batch and B.shape[2] == K
     L = lib()
-    n = L.tc_matmul_f32x3_workspace_bytes(batch, M, NN, K)
-    ws = torch.empty(max(int(n), 256), dtype=torch.uint8, device=A.device)
     Cm = torch.empty(batch, M, NN, dtype=torch.float32, device=A.device)
     CT = torch.empty(batch, NN, M, dtype=torch.float32, device=A.device) if transposed else None
     st = torch.empty(batch, dtype=torch.int32, device=A.device)
     _check("tc_matmul_f32x3",
            L.tc_matmul_f32x3(_ptr(A), _ptr(B), _ptr(Cm), _ptr(CT) if CT is not None else None,
-                             batch, M, NN, K, _ptr(st), _ptr(ws), ws.numel(), _stream()))
+                             batch, M, NN, K, _ptr(st), _stream()))
     return Cm, CT, st
 
 

@@ -94,7 +94,7 @@ tc_status make_dims(const tc_params* p, Dims* out) {
   // the subspace solve runs its products on the tensor cores when the shapes fit its tiles
   // (the sign sketch keeps one row of signs, d floats, in shared memory)
   D.tcp = !D.full && (D.N & 3) == 0 && (size_t)D.d * sizeof(float) <= 48 * 1024 &&
-          gemm_split_supported(D.N, D.k, D.N) && gemm_split_supported(D.N, D.k, D.k);
+          gemm_f32x3_supported(D.N, D.k, D.N) && gemm_f32x3_supported(D.N, D.k, D.k);
   D.max_sweeps = p->max_sweeps > 0 ? p->max_sweeps : 30;
   D.lambda = p->lambda;
   D.rank_tol = p->rank_tol;
@@ -127,17 +127,15 @@ Plan make_plan(const Dims& D) {
   P.C = take(B * N * 4);
   P.E = take(B * N * 4);
   P.sigma = take(B * k * 4);
-  P.G = take(B * N * N * 4 * (D.tcp ? 2 : 1));
+  P.G = take(B * N * N * 4);
   if (D.tcp) {
-    P.panel_T_off = align_up(B * 2 * N * k * 4, 256);
+    P.panel_T_off = align_up(B * N * k * 4, 256);
     P.PA = take(2 * P.panel_T_off);
     P.PB = take(2 * P.panel_T_off);
     P.Sk = take(B * k * k * 4);
     P.Hk = take(B * k * k * 4);
-    P.RinvS = take(B * 2 * k * k * 4);
-    P.ZTs = take(B * 2 * k * k * 4);
-    P.Es = take(B * 5 * k * k * 4);
-    if (!D.f16) P.Gplain = take(B * N * N * 4);
+    P.Rinv = take(B * k * k * 4);
+    P.Es = take(B * 4 * k * k * 4);
   } else if (!D.full) {
     P.Y0 = take(B * N * k * 4);
     P.Y1 = take(B * N * k * 4);
@@ -165,17 +163,9 @@ Plan make_plan(const Dims& D) {
 }
 
 // float16 inputs go to the tensor cores; float32 inputs keep full precision on the plain ALUs
-// With Dims::tcp, G receives the two TF32 planes per image; float32 inputs first go to
-// `Gplain` [B][N][N] and are split from there.
-tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st,
-                      float* Gplain) {
+tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st) {
   if (D.f16) return launch_gram_tc(D, O, G, status, st);
-  if (!D.tcp) return launch_gram_simt(D, O, G, st);
-  if (Gplain == nullptr) return TC_ERR_INVALID_ARG;
-  tc_status s = launch_gram_simt(D, O, Gplain, st);
-  if (s != TC_OK) return s;
-  launch_split_panel(Gplain, D.N, D.N, D.B, G, nullptr, st, KC_GRAM);
-  return TC_OK;
+  return launch_gram_simt(D, O, G, st);
 }
 
 static tc_status check_launch() {
@@ -265,15 +255,14 @@ static tc_status enqueue_score(const Ctx& c, const void* O, const void* A, float
     // the sketch and its first Cholesky-QR pass do not read G: with groups, the Gram matrix is
     // built beside them on a stream of its own and joined in front of the first product with G
     cudaEvent_t gram_done = nullptr;
-    float* Gg = (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N * (D.tcp ? 2 : 1);
-    float* Gp = (D.tcp && !D.f16) ? (float*)(c.ws + c.P.Gplain) + (size_t)b0 * D.N * D.N : nullptr;
+    float* Gg = (float*)(c.ws + c.P.G) + (size_t)b0 * D.N * D.N;
     if (ng > 1 && !D.full) {
       cudaStreamWaitEvent(gs->s2[g], gs->fork, 0);
-      err = launch_gram(Dg, Og, Gg, img_status + b0, gs->s2[g], Gp);
+      err = launch_gram(Dg, Og, Gg, img_status + b0, gs->s2[g]);
       cudaEventRecord(gs->gram_done[g], gs->s2[g]);
       gram_done = gs->gram_done[g];
     } else {
-      err = launch_gram(Dg, Og, Gg, img_status + b0, st, Gp);
+      err = launch_gram(Dg, Og, Gg, img_status + b0, st);
     }
     if (err == TC_OK)
       err = launch_ics(Dg, c.P, c.ws, b0, Og, C + (size_t)b0 * D.N, sigma ? sigma + (size_t)b0 * q : nullptr,
@@ -576,32 +565,20 @@ tc_status tc_gram(const tc_params* p, const void* O, float* G, void* stream) {
   tc_status s = make_dims(p, &D);
   if (s != TC_OK) return s;
   if (!O || !G || misaligned(O) || misaligned(G)) return TC_ERR_INVALID_ARG;
-  D.tcp = false;  // plain float32 out, whatever rank_cap says
-  s = launch_gram(D, O, G, nullptr, (cudaStream_t)stream, nullptr);
+  s = launch_gram(D, O, G, nullptr, (cudaStream_t)stream);
   if (s != TC_OK) return s;
   return check_launch();
 }
 
-size_t tc_matmul_f32x3_workspace_bytes(int32_t batch, int32_t M, int32_t NN, int32_t K) {
-  if (batch < 1 || M < 1 || NN < 1 || K < 1) return 0;
-  return align_up((size_t)batch * 2 * M * K * 4, 256) + align_up((size_t)batch * 2 * NN * K * 4, 256);
-}
-
 tc_status tc_matmul_f32x3(const float* A, const float* B, float* C, float* CT, int32_t batch,
-                          int32_t M, int32_t NN, int32_t K, int32_t* img_status, void* ws,
-                          size_t ws_bytes, void* stream) {
-  if (!A || !B || !C || !ws || batch < 1 || M < 1 || NN < 1 || K < 1) return TC_ERR_INVALID_ARG;
-  if (misaligned(A) || misaligned(B) || misaligned(C) || misaligned(ws) || (CT && misaligned(CT)))
+                          int32_t M, int32_t NN, int32_t K, int32_t* img_status, void* stream) {
+  if (!A || !B || (!C && !CT) || batch < 1 || M < 1 || NN < 1 || K < 1) return TC_ERR_INVALID_ARG;
+  if (misaligned(A) || misaligned(B) || (C && misaligned(C)) || (CT && misaligned(CT)))
     return TC_ERR_INVALID_ARG;
-  if (!gemm_split_supported(M, NN, K)) return TC_ERR_UNSUPPORTED;
-  if (ws_bytes < tc_matmul_f32x3_workspace_bytes(batch, M, NN, K)) return TC_ERR_WORKSPACE;
+  if (!gemm_f32x3_supported(M, NN, K)) return TC_ERR_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
-  float* As = (float*)ws;
-  float* Bs = (float*)((char*)ws + align_up((size_t)batch * 2 * M * K * 4, 256));
   if (img_status) fill_i32(img_status, batch, 0, st);
-  launch_split_panel(A, M, K, batch, As, nullptr, st, KC_GEMM);
-  launch_split_panel(B, NN, K, batch, Bs, nullptr, st, KC_GEMM);
-  tc_status s = launch_gemm_split(As, Bs, M, NN, K, batch, C, CT, nullptr, nullptr, img_status, st, KC_GEMM);
+  tc_status s = launch_gemm_f32x3(A, B, M, NN, K, batch, C, CT, img_status, st, KC_GEMM);
   if (s != TC_OK) return s;
   return check_launch();
 }
@@ -657,8 +634,7 @@ tc_status tc_rank(const tc_params* p, const void* O, const int32_t* idx, int32_t
     launch_gather_rows(F, n_sub, O, idx, w + rows_off, img_status, st);
     rows = w + rows_off;
   }
-  s = launch_gram(D, rows, (float*)(w + P.G), img_status, st,
-                  (D.tcp && !D.f16) ? (float*)(w + P.Gplain) : nullptr);
+  s = launch_gram(D, rows, (float*)(w + P.G), img_status, st);
   if (s != TC_OK) return s;
   s = launch_ics(D, P, w, 0, rows, (float*)(w + P.C), sigma, rank, img_status, st,
                  rank_small_full(D) ? (float*)(w + rows_off + rank_rows_bytes(D)) : nullptr);

@@ -47,12 +47,9 @@ __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t 
       : "memory");
 }
 
-// lo_off = 0: G [image][N][N] plain float32 (img_stride = N N).  lo_off > 0: every entry goes
-// out as its two TF32 parts, the high one at G[...] and the low one lo_off floats further on.
-__global__ void __launch_bounds__(192, 2) gram_tc_kernel(const __grid_constant__ CUtensorMap map,
+__global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CUtensorMap map,
                                                      float* __restrict__ G, int N, int d,
-                                                     int tiles_per_image, size_t img_stride,
-                                                     size_t lo_off,
+                                                     int tiles_per_image,
                                                      int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[STAGES];
@@ -180,41 +177,12 @@ __global__ void __launch_bounds__(192, 2) gram_tc_kernel(const __grid_constant__
                      : "memory");
     }
     if (ok && s_fail == 0) {
-      float* Gb = G + (size_t)b * img_stride;
+      float* Gb = G + (size_t)b * N * N;
       const int row = ti * TILE + warp * 32 + lane;
       if (row < N) {
 #pragma unroll
         for (int q = 0; q < TILE / 32; ++q) {
           const int col0 = tj * TILE + q * 32;
-          if (lo_off != 0) {
-            // the two TF32 planes the tensor-core products of the subspace solve read: the low
-            // parts go out here, four at a time, and the high parts take the place of the values
-            const bool vec = col0 + 32 <= N && (N & 3) == 0;
-#pragma unroll
-            for (int j4 = 0; j4 < 8; ++j4) {
-              float lo[4];
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const float v = acc[q * 32 + 4 * j4 + u];
-                const float hi = tf32_round(v);
-                lo[u] = tf32_round(v - hi);
-                acc[q * 32 + 4 * j4 + u] = hi;
-              }
-              if (vec) {
-                *reinterpret_cast<float4*>(Gb + lo_off + (size_t)row * N + col0 + 4 * j4) =
-                    make_float4(lo[0], lo[1], lo[2], lo[3]);
-              } else {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                  if (col0 + 4 * j4 + u < N) Gb[lo_off + (size_t)row * N + col0 + 4 * j4 + u] = lo[u];
-              }
-              if (!diag) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                  if (col0 + 4 * j4 + u < N) Gb[lo_off + (size_t)(col0 + 4 * j4 + u) * N + row] = lo[u];
-              }
-            }
-          }
           if (col0 + 32 <= N && (N & 3) == 0) {
             float4* dst = reinterpret_cast<float4*>(Gb + (size_t)row * N + col0);
 #pragma unroll
@@ -240,7 +208,7 @@ __global__ void __launch_bounds__(192, 2) gram_tc_kernel(const __grid_constant__
       const int row = ti * TILE + warp * 32 + lane;
       if (row < N)
         for (int j = 0; j < TILE; ++j)
-          if (tj * TILE + j < N) G[(size_t)b * img_stride + (size_t)row * N + tj * TILE + j] = __int_as_float(0x7fc00000);
+          if (tj * TILE + j < N) G[((size_t)b * N + row) * N + tj * TILE + j] = __int_as_float(0x7fc00000);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -274,9 +242,7 @@ tc_status launch_gram_tc(const Dims& D, const void* O, float* G, int32_t* status
   const int nt = (D.N + TILE - 1) / TILE;
   const int tiles = nt * (nt + 1) / 2;
   Scope scope_(KC_GRAM, st);
-  const size_t NN = (size_t)D.N * D.N;
-  gram_tc_kernel<<<D.B * tiles, 192, SMEM_BYTES, st>>>(map, G, D.N, D.d, tiles, D.tcp ? 2 * NN : NN,
-                                                       D.tcp ? NN : 0, status);
+  gram_tc_kernel<<<D.B * tiles, 192, SMEM_BYTES, st>>>(map, G, D.N, D.d, tiles, status);
   note_launch();
   return TC_OK;
 }

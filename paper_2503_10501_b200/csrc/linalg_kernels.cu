@@ -1076,7 +1076,7 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
                                                            float* __restrict__ RinvT, int k_rt,
                                                            float shift_rel,
                                                            int32_t* __restrict__ status,
-                                                           int nparts, int split_out) {
+                                                           int nparts) {
   const int k = KT ? KT : k_rt;
   extern __shared__ __align__(16) float fsm[];
   __shared__ float s_red[16];
@@ -1347,19 +1347,7 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
     }
     __syncthreads();
   }
-  // RinvT[c][m] = X[m][c] for m <= c, zero otherwise; with split_out as the two TF32 planes
-  // [2][k][k] the tensor-core products read
-  if (split_out) {
-    float* out = RinvT + b * 2 * kk;
-    for (int e = tid; e < (int)kk; e += 512) {
-      const int c = e / k, mrow = e - c * k;
-      const float v = (mrow <= c) ? A[mrow * ld + c] : 0.f;
-      const float hi = tf32_round(v);
-      out[e] = hi;
-      out[kk + e] = tf32_round(v - hi);
-    }
-    return;
-  }
+  // RinvT[c][m] = X[m][c] for m <= c, zero otherwise
   float* out = RinvT + b * kk;
   for (int e = tid; e < (int)kk; e += 512) {
     const int c = e / k, mrow = e - c * k;
@@ -1552,8 +1540,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ u0g, float* __restrict__ u1g,
                                                          float* __restrict__ u2g, float* yg, float* __restrict__ mlg,
                                                          size_t ml_stride,
-                                                         int32_t* __restrict__ status, int nparts,
-                                                         int split_out) {
+                                                         int32_t* __restrict__ status, int nparts) {
   const int n = NT ? NT : n_rt;
   extern __shared__ __align__(16) float sm[];
   const int ld = n | 1;
@@ -1602,6 +1589,26 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         dst[1] = (q[0].y + q[1].y) + (q[2].y + q[3].y);
         dst[2] = (q[0].z + q[1].z) + (q[2].z + q[3].z);
         dst[3] = (q[0].w + q[1].w) + (q[2].w + q[3].w);
+      }
+    }
+  } else if (nparts == 1 && (n & 3) == 0) {
+    // one part that need not be symmetric to the last bit (a product Q^T (G Q)): 16-byte loads,
+    // then the two triangles are averaged in shared memory
+    const float4* H4 = reinterpret_cast<const float4*>(Hb);
+    const int kv = n >> 2, nv = (n * n) >> 2;
+    for (int e = tid; e < nv; e += 512) {
+      const float4 p = __ldg(H4 + e);
+      const int r = e / kv, c = (e - r * kv) * 4;
+      float* dst = A + r * ld + c;
+      dst[0] = p.x; dst[1] = p.y; dst[2] = p.z; dst[3] = p.w;
+    }
+    __syncthreads();
+    for (int e = tid; e < n * n; e += 512) {
+      const int r = e / n, c = e - r * n;
+      if (c > r) {
+        const float m = 0.5f * (A[r * ld + c] + A[c * ld + r]);
+        A[r * ld + c] = m;
+        A[c * ld + r] = m;
       }
     }
   } else {
@@ -2151,8 +2158,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     // ---------------- Z = Q Y:  ZT[p][i] = sum_j Q[i][j] Y[j][p] ----------------
     // thread = (four eigenvectors p, twelve rows i): per j one 16-byte load of Y (coalesced over
     // p) and twelve broadcast reads of Q from shared memory feed 48 multiply-adds
-    // with split_out ZT goes out as the two TF32 planes [2][n][n] the tensor-core product reads
-    float* out = ZTg + (split_out ? 2 * img : img);
+    float* out = ZTg + img;
     const bool vec = (n & 3) == 0;
     const int npg = (n + 3) >> 2, nrg = (n + 11) / 12;
     for (int w = tid; w < npg * nrg; w += 512) {
@@ -2191,15 +2197,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       for (int v = 0; v < 4; ++v) {
         if (p0 + v >= n) continue;
         float* orow = out + (size_t)(p0 + v) * n + i0;
-        if (split_out) {
-#pragma unroll
-          for (int u = 0; u < 12; ++u)
-            if (i0 + u < n) {
-              const float hi = tf32_round(acc[u][v]);
-              orow[u] = hi;
-              orow[(size_t)n * n + u] = tf32_round(acc[u][v] - hi);
-            }
-        } else if (vec && i0 + 12 <= n) {
+        if (vec && i0 + 12 <= n) {
 #pragma unroll
           for (int u = 0; u < 12; u += 4)
             *reinterpret_cast<float4*>(orow + u) =
@@ -2239,14 +2237,14 @@ constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared 
 static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
                           int max_sweeps, float rank_tol, float* scr1, float* scr2, float* scr3,
                           float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st,
-                          int nparts = 1, int split_out = 0) {
+                          int nparts = 1) {
   Scope scope_(KC_JACOBI, st);
   {
     const size_t tri = ((size_t)n * (n | 1) + 27 * (size_t)((n + 3) & ~3)) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       auto go = [&](auto kernel) {
         cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
-        { kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts, split_out); note_launch(); }
+        { kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts); note_launch(); }
       };
       switch (n) {
         case 128: go(tridiag_eig_kernel<128>); break;
@@ -2275,14 +2273,13 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
 }
 
 static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
-                            float shift_rel, int32_t* status, cudaStream_t st, int nparts,
-                            int split_out = 0) {
+                            float shift_rel, int32_t* status, cudaStream_t st, int nparts) {
   Scope scope_(KC_CHOL, st);
   const size_t fast = ((size_t)k * (k | 1) + (size_t)CNB * k + (size_t)(k / CNB) * CNB * CNB) * sizeof(float);
   if (k % CNB == 0 && k >= CNB && fast <= SMEM_LIMIT) {
     auto go = [&](auto kernel) {
       cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast);
-      { kernel<<<batch, 512, fast, st>>>(S, RinvT, k, shift_rel, status, nparts, split_out); note_launch(); }
+      { kernel<<<batch, 512, fast, st>>>(S, RinvT, k, shift_rel, status, nparts); note_launch(); }
     };
     switch (k) {
       case 128: go(chol_inv_fast_kernel<128>); break;
@@ -2310,52 +2307,32 @@ static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, i
 }
 
 // ==========================================================================================
-// A float32 matrix as the two TF32 planes the tensor-core products read, row-major and / or
-// transposed:  in [R][C]  ->  split [2][R][C], splitT [2][C][R]  (per image).
-// 32 x 32 tiles through shared memory so that both forms are written along their rows.
+// out [C][R] = in [R][C]^T per image, 32 x 32 tiles through shared memory.
 // grid (C tiles, R tiles, batch), block (32, 8).
 // ==========================================================================================
-__global__ void __launch_bounds__(256) split_panel_kernel(const float* __restrict__ in, int R, int C,
-                                                         float* __restrict__ split,
-                                                         float* __restrict__ splitT) {
-  __shared__ float th[32][33], tl[32][33];
+__global__ void __launch_bounds__(256) transpose_kernel(const float* __restrict__ in, int R, int C,
+                                                       float* __restrict__ out) {
+  __shared__ float t[32][33];
   const int b = blockIdx.z, r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
   const size_t RC = (size_t)R * C;
-  const float* src = in + (size_t)b * RC;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int r = r0 + ty + 8 * i, c = c0 + tx;
-    float hi = 0.f, lo = 0.f;
-    if (r < R && c < C) {
-      const float v = src[(size_t)r * C + c];
-      hi = tf32_round(v);
-      lo = tf32_round(v - hi);
-      if (split != nullptr) {
-        split[(size_t)b * 2 * RC + (size_t)r * C + c] = hi;
-        split[(size_t)b * 2 * RC + RC + (size_t)r * C + c] = lo;
-      }
-    }
-    th[ty + 8 * i][tx] = hi;
-    tl[ty + 8 * i][tx] = lo;
+    t[ty + 8 * i][tx] = (r < R && c < C) ? in[(size_t)b * RC + (size_t)r * C + c] : 0.f;
   }
-  if (splitT == nullptr) return;
   __syncthreads();
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int c = c0 + ty + 8 * i, r = r0 + tx;
-    if (r < R && c < C) {
-      splitT[(size_t)b * 2 * RC + (size_t)c * R + r] = th[tx][ty + 8 * i];
-      splitT[(size_t)b * 2 * RC + RC + (size_t)c * R + r] = tl[tx][ty + 8 * i];
-    }
+    if (r < R && c < C) out[(size_t)b * RC + (size_t)c * R + r] = t[tx][ty + 8 * i];
   }
 }
 
-void launch_split_panel(const float* in, int R, int C, int batch, float* split, float* splitT,
-                        cudaStream_t st, int cls) {
+static void launch_transpose(const float* in, int R, int C, int batch, float* out, cudaStream_t st, int cls) {
   Scope scope_(cls, st);
   dim3 grid((C + 31) / 32, (R + 31) / 32, batch), block(32, 8);
-  { split_panel_kernel<<<grid, block, 0, st>>>(in, R, C, split, splitT); note_launch(); }
+  { transpose_kernel<<<grid, block, 0, st>>>(in, R, C, out); note_launch(); }
 }
 
 // ==========================================================================================
@@ -2496,52 +2473,51 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
     }
   };
   if (D.tcp) {
-    // ---- the products on the tensor cores, operands as split TF32 panels (gemm_split.cu) ----
-    // Two sets of panels, each held row-major [B][2][N][k] and transposed [B][2][k][N].
-    float* PAr = (float*)(ws + P.PA) + b0 * 2 * sY;
-    float* PAt = (float*)(ws + P.PA) + (size_t)P.panel_T_off / sizeof(float) + b0 * 2 * sY;
-    float* PBr = (float*)(ws + P.PB) + b0 * 2 * sY;
-    float* PBt = (float*)(ws + P.PB) + (size_t)P.panel_T_off / sizeof(float) + b0 * 2 * sY;
+    // ---- the products on the tensor cores (gemm_f32x3.cu: C = A B^T, both operands with the
+    //      contraction index contiguous).  Every tall panel is therefore kept twice, row-major
+    //      [N][k] and transposed [k][N]; a product writes whichever forms its consumers read.
+    float* Ar = (float*)(ws + P.PA) + b0 * sY;
+    float* At = (float*)(ws + P.PA) + (size_t)P.panel_T_off / sizeof(float) + b0 * sY;
+    float* Br = (float*)(ws + P.PB) + b0 * sY;
+    float* Bt = (float*)(ws + P.PB) + (size_t)P.panel_T_off / sizeof(float) + b0 * sY;
     float* Sk = (float*)(ws + P.Sk) + b0 * sK;
     float* Hk = (float*)(ws + P.Hk) + b0 * sK;
-    float* RinvS = (float*)(ws + P.RinvS) + b0 * 2 * sK;
-    float* ZTs = (float*)(ws + P.ZTs) + b0 * 2 * sK;
-    float* Es = (float*)(ws + P.Es) + b0 * 5 * sK;
-    const float* Gs = (const float*)(ws + P.G) + b0 * 2 * sG;
+    float* Rinv = (float*)(ws + P.Rinv) + b0 * sK;
+    float* Es = (float*)(ws + P.Es) + b0 * 4 * sK;
     int32_t* stp = img_status;
-    // 1. sketch (plain, in the room of set B, which is free until the first pass writes it)
-    sketch_into(PBr);
-    launch_split_panel(PBr, N, k, B, PAr, PAt, st, KC_SKETCH);
-    // one Cholesky-QR pass  dst = src R^{-1}  with  R^T R = src^T src + shift
     tc_status err = TC_OK;
-    auto mm = [&](const float* A_, const float* B_, int M_, int K_, float* c0, float* c1, float* c2,
-                  float* c3, int cls) {
-      if (err == TC_OK) err = launch_gemm_split(A_, B_, M_, k, K_, B, c0, c1, c2, c3, stp, st, cls);
+    auto mm = [&](const float* A_, const float* B_, int M_, int K_, float* c, float* ct, int cls) {
+      if (err == TC_OK) err = launch_gemm_f32x3(A_, B_, M_, k, K_, B, c, ct, stp, st, cls);
     };
+    // one Cholesky-QR pass  dst = src R^{-1}  with  R^T R = src^T src + shift
     auto pass = [&](const float* srcR, const float* srcT, float* dstR, float* dstT, float shift_rel) {
-      mm(srcT, srcT, k, N, Sk, nullptr, nullptr, nullptr, KC_GEMM_TN);
+      mm(srcT, srcT, k, N, Sk, nullptr, KC_GEMM_TN);
       if (err != TC_OK) return;
-      launch_chol_inv(Sk, RinvS, nullptr, k, B, shift_rel, stp, st, 1, 1);
-      mm(srcR, RinvS, N, k, nullptr, nullptr, dstR, dstT, KC_GEMM);
+      launch_chol_inv(Sk, Rinv, nullptr, k, B, shift_rel, stp, st, 1);
+      mm(srcR, Rinv, N, k, dstR, dstT, KC_GEMM);   // Rinv holds R^{-T}: (Y R^{-1})[x][c] = Y[x][:] . Rinv[c][:]
     };
-    // 2. a well-conditioned basis Q0 of the sketch
-    pass(PAr, PAt, nullptr, PBt, 1e-6f);
+    // 1. sketch of the column space of O, in both forms
+    sketch_into(Ar);
+    launch_transpose(Ar, N, k, B, At, st, KC_SKETCH);
+    // 2. a well-conditioned basis Q0 of the sketch (only its transposed form is read)
+    pass(Ar, At, nullptr, Bt, 1e-6f);
     // 3. Y1 = G Q0, then two passes: the first (shifted) brings the condition number from ~1e7
     //    down to ~1e3, the second leaves a basis whose departure from orthonormality lies in the
     //    directions under the rank cut-off; the Ritz values above it are unaffected
     if (g_ready) cudaStreamWaitEvent(st, g_ready, 0);
-    mm(Gs, PBt, N, N, nullptr, nullptr, PAr, PAt, KC_GEMM_GQ);
-    pass(PAr, PAt, PBr, PBt, 1e-6f);
-    pass(PBr, PBt, PAr, PAt, 1e-7f);  // Q1 in set A
+    mm(G, Bt, N, N, Ar, At, KC_GEMM_GQ);
+    pass(Ar, At, Br, Bt, 1e-6f);
+    pass(Br, Bt, Ar, At, 1e-7f);  // Q1 in set A
     // 4. Rayleigh-Ritz:  T = G Q1 (kept transposed),  H = Q1^T T
-    mm(Gs, PAt, N, N, nullptr, nullptr, nullptr, PBt, KC_GEMM_GQ);
-    mm(PAt, PBt, k, N, Hk, nullptr, nullptr, nullptr, KC_GEMM_TN);
+    mm(G, At, N, N, nullptr, Bt, KC_GEMM_GQ);
+    mm(At, Bt, k, N, Hk, nullptr, KC_GEMM_TN);
     if (err != TC_OK) return err;
-    launch_jacobi(Hk, Es, ZTs, theta, k, B, D.max_sweeps, D.rank_tol, Es + (size_t)B * sK,
-                  Es + 2 * (size_t)B * sK, Es + 3 * (size_t)B * sK, Es + 4 * (size_t)B * sK, sK, stp, st, 1, 1);
+    float* ZTk = Sk;  // the k x k matrices of the passes are free now
+    launch_jacobi(Hk, Es, ZTk, theta, k, B, D.max_sweeps, D.rank_tol, Es + (size_t)B * sK,
+                  Es + 2 * (size_t)B * sK, Rinv, Es + 3 * (size_t)B * sK, sK, stp, st, 1);
     // 5. PT[p][x] = sum_i ZT[p][i] Q1[x][i]: the product Q1 ZT^T written transposed
-    float* PT = PBr;
-    mm(PAr, ZTs, N, k, nullptr, PT, nullptr, nullptr, KC_GEMM);
+    float* PT = Br;
+    mm(Ar, ZTk, N, k, nullptr, PT, KC_GEMM);
     if (err != TC_OK) return err;
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(

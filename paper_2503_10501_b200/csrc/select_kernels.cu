@@ -156,23 +156,20 @@ __global__ void __launch_bounds__(128) match_gram_kernel(const float* __restrict
                                                         const int32_t* __restrict__ setB,
                                                         float* __restrict__ best_val,
                                                         int32_t* __restrict__ best_dst, int N,
-                                                        int nA, int nB, int split) {
+                                                        int nA, int nB) {
   const int b = blockIdx.y;
   const int jb = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (jb >= nB) return;
-  // split: G is kept as two TF32 planes [2][N][N] per image and an entry is their sum
-  const size_t NN = (size_t)N * N;
-  const float* Gb = G + (size_t)b * (split ? 2 * NN : NN);
-  auto g_at = [&](size_t i) { return split ? Gb[i] + Gb[NN + i] : Gb[i]; };
+  const float* Gb = G + (size_t)b * N * N;
   const int tb = setB[(size_t)b * nB + jb];
-  const float inv_b = inv_norm_from_sq(g_at((size_t)tb * N + tb));
+  const float inv_b = inv_norm_from_sq(Gb[(size_t)tb * N + tb]);
   float bv = -INFINITY;
   int bi = 0x7fffffff;
   for (int ja = lane; ja < nA; ja += 32) {
     const int ta = setA[(size_t)b * nA + ja];
-    const float inv_a = inv_norm_from_sq(g_at((size_t)ta * N + ta));
-    const float c = g_at((size_t)tb * N + ta) * inv_b * inv_a;
+    const float inv_a = inv_norm_from_sq(Gb[(size_t)ta * N + ta]);
+    const float c = Gb[(size_t)tb * N + ta] * inv_b * inv_a;
     if (c > bv || (c == bv && ta < bi)) {
       bv = c;
       bi = ta;
@@ -190,7 +187,7 @@ void launch_match_gram(const Dims& D, const float* G, const int32_t* setA, const
   Scope scope_(KC_MATCH, st);
   if (D.nB == 0 || D.nA == 0) return;
   dim3 grid((D.nB + 3) / 4, D.B);
-  { match_gram_kernel<<<grid, 128, 0, st>>>(G, setA, setB, best_val, best_dst, D.N, D.nA, D.nB, D.tcp ? 1 : 0); note_launch(); }
+  { match_gram_kernel<<<grid, 128, 0, st>>>(G, setA, setB, best_val, best_dst, D.N, D.nA, D.nB); note_launch(); }
 }
 
 // ------------------------------------------------------------------------------------------

@@ -38,14 +38,12 @@ struct Plan {
   size_t setA, setB, best_val, best_dst, msrc, mdst, kept;  // int32 / f32 lists
   size_t rank;     // [B] int32
   size_t flags;    // [B] int32 device status scratch
-  // tensor-core subspace solve (Dims::tcp): G is then two TF32 planes [B][2][N][N], and
-  size_t PA, PB;   // two sets of split panels: [B][2][N][k] row-major, then, panel_T_off bytes
-                   // further on, [B][2][k][N] transposed
+  // tensor-core subspace solve (Dims::tcp)
+  size_t PA, PB;   // two sets of tall panels: [B][N][k] row-major and, panel_T_off bytes
+                   // further on, [B][k][N] transposed
   size_t panel_T_off;
-  size_t Gplain;   // [B][N][N] f32, only for float32 inputs (their Gram matrix is split afterwards)
-  size_t Sk, Hk;   // [B][k][k] f32: Y^T Y and the projected matrix
-  size_t RinvS, ZTs;  // [B][2][k][k] split: R^{-T} and the eigenvectors of the projection
-  size_t Es;       // [B][5][k][k] f32 scratch of the tridiagonal solver
+  size_t Sk, Hk;   // [B][k][k] f32: Y^T Y (later the eigenvectors) and the projected matrix
+  size_t Es;       // [B][4][k][k] f32 scratch of the tridiagonal solver
   size_t total;
 };
 
@@ -90,7 +88,6 @@ void launch_combine(const Dims& D, const float* s_part, const float* C, float* S
 // Stage I prune + Eq. 3-9 split.
 void launch_prune(const Dims& D, const float* E, int32_t* setA, int32_t* setB, cudaStream_t st);
 // Eq. 3-10 best match per Set-B token, from the Gram matrix or from the rows of O.
-// (with Dims::tcp, G is the pair of TF32 planes and an entry is the sum of its two parts)
 void launch_match_gram(const Dims& D, const float* G, const int32_t* setA, const int32_t* setB,
                        float* best_val, int32_t* best_dst, cudaStream_t st);
 void launch_match_rows(const Dims& D, const void* O, const int32_t* setA, const int32_t* setB,
@@ -112,19 +109,14 @@ void fill_i32(int32_t* p, int n, int v, cudaStream_t st);
 void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, const void* Xo,
                        const int32_t* kept, void* Ho, int32_t* pos, cudaStream_t st);
 
-// G = O O^T (float32 out; with Dims::tcp as two TF32 planes [B][2][N][N]).
-tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st,
-                      float* Gplain);
+// G = O O^T (float32 out).
+tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 
-// C = A B^T on the tensor cores from split panels (A [batch][2][M][K], B [batch][2][NN][K]);
-// any of the four output forms may be null.
-bool gemm_split_supported(int M, int NN, int K);
-tc_status launch_gemm_split(const float* A, const float* B, int M, int NN, int K, int batch,
-                            float* C_plain, float* C_plainT, float* C_split, float* C_splitT,
-                            int32_t* status, cudaStream_t st, int cls);
-// in [batch][R][C] float32 -> split [batch][2][R][C] and / or splitT [batch][2][C][R]
-void launch_split_panel(const float* in, int R, int C, int batch, float* split, float* splitT,
-                        cudaStream_t st, int cls);
+// C [batch][M][NN] = A B^T on the tensor cores, float32-accurate (A [batch][M][K],
+// B [batch][NN][K]); C and / or its transpose CT [batch][NN][M] are written (either may be null).
+bool gemm_f32x3_supported(int M, int NN, int K);
+tc_status launch_gemm_f32x3(const float* A, const float* B, int M, int NN, int K, int batch,
+                            float* C, float* CT, int32_t* status, cudaStream_t st, int cls);
 
 // Eigen-decomposition of G and Eq. 3-6:  C, theta (unsorted), then sorted sigma / rank.
 // g_ready: optional event after which G is complete when it is built on another stream (the

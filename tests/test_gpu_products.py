@@ -1,4 +1,4 @@
-"""The split-TF32 tensor-core product of the subspace solve (Sec. 3.3.1: the SVD behind Eq. 3-5
+"""The three-product TF32 tensor-core kernel of the subspace solve (Sec. 3.3.1: the SVD behind Eq. 3-5
 and 3-6 is taken through products with the Gram matrix) against float64, through the C ABI."""
 import numpy as np
 import pytest
