@@ -42,13 +42,36 @@ def peaks():
             "sm_max_mhz": 1965.0, "source": "fallback"}
 
 
+CONFIG_KEYS = {"cfg1": "cfg1_single_f32", "cfg2": "cfg2_llava7b_f16", "cfg3": "cfg3_llava13b_f16",
+               "cfg4": "cfg4_anyres_f16", "cfg5": "cfg5_sweep_f16"}
+
+
 def workload(args, rank=0):
-    cfg = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=args.batch, n_query=args.n_query,
-                                                 keep=args.keep)
-    if args.rank_cap:
-        cfg = cfg.with_(rank_cap=args.rank_cap)
-    name = f"cfg5_sweep_f16 B={cfg.batch} N={cfg.n_tokens} d={cfg.d_model} T={cfg.n_query} keep={cfg.keep}"
+    """The metric's workload (cfg5 at B=64, T=128, keep=128) unless --config names another of
+    the five; --batch / --n-query / --keep override the named configuration's own values."""
+    base = inputs.CONFIGS[CONFIG_KEYS[args.config]]
+    if args.config == "cfg5":
+        cfg = base.with_(batch=args.batch or 64, n_query=args.n_query or 128, keep=args.keep or 128)
+    else:
+        cfg = base.with_(batch=args.batch or base.batch, n_query=args.n_query or base.n_query,
+                         keep=args.keep or base.keep)
+    if args.rank_cap >= 0:
+        cfg = cfg.with_(rank_cap=args.rank_cap)   # 0 = the full solve (no rank hint)
+    name = (f"{cfg.name} B={cfg.batch} N={cfg.n_tokens} d={cfg.d_model} T={cfg.n_query} "
+            f"keep={cfg.keep} rank_cap={cfg.rank_cap}")
     return cfg, name
+
+
+def uses_tensor_products(cfg):
+    """Whether the subspace solve of this configuration runs its products on the tensor cores
+    (the library's own rule: a rank hint of 128, 144, 160 or 192 and N a multiple of 4)."""
+    return cfg.rank_cap in (128, 144, 160, 192) and cfg.n_tokens % 4 == 0 and cfg.d_model * 4 <= 48 * 1024
+
+
+def product_peak(pk):
+    """float32-equivalent peak of the three-product TF32 kernel: the measured sustained bf16
+    tensor throughput x 1/2 (nominal TF32 : bf16 ratio) / 3 (products per term)."""
+    return pk["bf16_tflops_sustained"] * 0.5 / 3.0
 
 
 def algorithmic_bytes_per_image(cfg, P):
@@ -60,20 +83,25 @@ def algorithmic_bytes_per_image(cfg, P):
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
-def time_oracle(cfg, n_images, first_image=0):
-    """Seconds per image of the float64 oracle as it stands, and the BLAS threads it may use."""
+def time_oracle(cfg, n_images, first_image=0, single_thread=False):
+    """Seconds per image of the float64 oracle as it stands, and the BLAS threads it used."""
     from oracle import ipgs_oracle as orc
+    import contextlib
+    limit = contextlib.nullcontext()
     try:
-        from threadpoolctl import threadpool_info
+        from threadpoolctl import threadpool_info, threadpool_limits
         threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        if single_thread:
+            limit, threads = threadpool_limits(limits=1), 1
     except Exception:
         threads = os.cpu_count() or 1
     ims = [inputs.make_image(cfg, first_image + b) for b in range(n_images)]
-    t0 = time.perf_counter()
-    for im in ims:
-        orc.carve(im["O"].astype(np.float64), im["A"].astype(np.float64), im["X"], im["K"], im["V"],
-                  cfg.keep, cfg.rho, cfg.lam, cfg.rank_tol, "none")
-    dt = time.perf_counter() - t0
+    with limit:
+        t0 = time.perf_counter()
+        for im in ims:
+            orc.carve(im["O"].astype(np.float64), im["A"].astype(np.float64), im["X"], im["K"], im["V"],
+                      cfg.keep, cfg.rho, cfg.lam, cfg.rank_tol, "none")
+        dt = time.perf_counter() - t0
     return dt / n_images, threads
 
 
@@ -264,47 +292,22 @@ def run_ours(args):
     nbytes = lambda ts: int(sum(t.numel() * t.element_size() for t in ts))
     pk = peaks()
 
-    # roofline of the kernel that takes the most device time per step (each profile class is one
-    # kernel; the float32 GEMM is three classes, one per kind of product)
-    top = max(prof.items(), key=lambda kv: kv[1][0])
-    top_name, (top_ms, top_launches) = top
-    per_launch_s = top_ms * 1e-3 / max(top_launches, 1)
+    # roofline of the kernel class that takes the most device time per step
     k = p.rank_cap if p.rank_cap else p.n_tokens
     N = cfg.n_tokens
     alg_bytes_img = algorithmic_bytes_per_image(cfg, P)
-    alu_peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
-    # DRAM bytes per image from the ncu capture of the current kernels at B=16
-    # (profiles/ncu_full_kernels_cfg5_B16.md); they grow in proportion to the batch
-    ncu_dram_per_image = {"eig": 5.377e6 / 16, "chol_inv": 5.369e6 / 16, "gram": (75.57e6 + 3.8e6) / 16,
-                          "attn_colsum": (75.52e6 + 1.7e6) / 16, "compact": (75.58e6 + 17.7e6) / 16,
-                          "sketch": (75.51e6 + 2.0e6) / 16}
-    flops_per_launch = {
-        # Householder tridiagonalisation 4/3 k^3, accumulation of Q 4/3 k^3, Z = Q Y 2 k^3
-        "eig": cfg.batch * (14.0 / 3.0) * k ** 3,
-        "chol_inv": cfg.batch * (2.0 / 3.0) * k ** 3,
-        "gemm_f32_GQ": cfg.batch * 2.0 * N * N * k,
-        "gemm_f32_YtY": cfg.batch * 1.0 * N * k * (k + 1),  # symmetric: upper triangle only
-        "gemm_f32_YRinv": cfg.batch * 2.0 * N * k * k * 11.0 / 15.0,
-    }
-    if top_name in flops_per_launch:
-        roof = {"kernel": top_name, "bound": "alu", "achieved": flops_per_launch[top_name] / per_launch_s / 1e12,
-                "peak": alu_peak, "unit": "TFLOP/s"}
-    elif top_name == "gram":
-        flops = cfg.batch * 2.0 * N ** 2 * cfg.d_model
-        roof = {"kernel": top_name, "bound": "tensor", "achieved": flops / per_launch_s / 1e12,
-                "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s"}
-    else:
-        e = 2
-        per = {"attn_colsum": cfg.n_heads * cfg.n_query * N * e,
-               "compact": (P + cfg.keep) * (cfg.d_model + 2 * cfg.n_heads * cfg.head_dim) * e,
-               "sketch": N * cfg.d_model * e}.get(top_name, alg_bytes_img)
-        roof = {"kernel": top_name, "bound": "hbm", "achieved": cfg.batch * per / per_launch_s / 1e9,
-                "peak": pk["hbm_gbs"], "unit": "GB/s"}
+    kfr = kernel_fractions(cfg, P, k, prof, args.steps, pk)
+    top_name = max((n for n in prof if prof[n][1] and n in kfr), key=lambda n: prof[n][0])
+    roof = {"kernel": top_name}
+    roof.update({f: kfr[top_name][f] for f in ("bound", "achieved", "peak", "unit", "frac", "peak_source")})
+    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of
+    # this kernel at B=16, scaled by the batch: the traffic of these kernels grows in proportion);
+    # null for a kernel that changed after its counters were taken
+    ncu_dram_per_image = {"gram": (75.57e6 + 3.8e6) / 16, "attn_colsum": (75.52e6 + 1.7e6) / 16,
+                          "compact": (75.58e6 + 17.7e6) / 16}
     same_shape = (cfg.n_tokens, cfg.d_model, cfg.n_query, cfg.keep, k) == (576, 4096, 128, 128, 144)
     roof["traffic"] = (ncu_dram_per_image[top_name] * cfg.batch
                        if same_shape and top_name in ncu_dram_per_image else None)
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["peak_source"] = pk["source"]
     # the whole path against the slower of its HBM bytes and its Gram flops
     t_hbm = alg_bytes_img / (pk["hbm_gbs"] * 1e9)
     t_tensor = 2.0 * cfg.n_tokens ** 2 * cfg.d_model / (pk["bf16_tflops_sustained"] * 1e12)
@@ -318,15 +321,24 @@ def run_ours(args):
         cpu = None
         if world == 1 and args.cpu_images > 0:
             sec, threads = time_oracle(cfg, args.cpu_images)
+            n1 = max(1, args.cpu_images // 4)
+            sec1, _ = time_oracle(cfg, n1, single_thread=True)
             cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
                    "sample": f"{args.cpu_images} images of the {cfg.batch}-image batch, "
-                             "float64 oracle (LAPACK SVD + loops)"}
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                             "float64 oracle (LAPACK SVD + loops)",
+                   "single_thread": {"value": 1.0 / sec1, "unit": UNIT, "cores": 1,
+                                     "sample": f"{n1} images, BLAS limited to one thread"}}
+        line = {"metric": METRIC if args.config == "cfg5" else "IPGS carve images/s", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": name, "images_per_gpu": cfg.batch, "rank_cap": p.rank_cap,
                            "rank_tol": p.rank_tol, "lambda": p.lam, "rho": p.rho,
-                           "l2": "inputs (1.5 GB per step) exceed the 126 MB L2",
+                           "l2": f"inputs ({nbytes(devin.values()) / 1e9:.2f} GB per step) "
+                                 + ("exceed the 126 MB L2" if nbytes(devin.values()) > 126e6
+                                    else "fit the 126 MB L2: cold-cache figures need a larger batch"),
+                           "solver": ("full Jacobi / tridiagonal solve" if not p.rank_cap else
+                                      "subspace solve, products on the tensor cores"
+                                      if uses_tensor_products(cfg) else "subspace solve, float32 ALU products"),
                            "image_groups": groups,
                            "launch": "CUDA graph replay of one tc_carve" if use_graph else "plain calls"},
                 "us_per_image": us_img,
@@ -337,7 +349,7 @@ def run_ours(args):
                 "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
                 "path_roofline": path,
                 "kernel_ms_per_step": {k_: round(v[0] / args.steps, 4) for k_, v in prof.items() if v[1]},
-                "kernel_roofline": kernel_fractions(cfg, P, k, prof, args.steps, pk),
+                "kernel_roofline": kfr,
                 "cpu_baseline": cpu}
         print(json.dumps(line))
     if world > 1:
@@ -347,33 +359,53 @@ def run_ours(args):
 # ----------------------------------------------------------------------------- sweep
 def kernel_fractions(cfg, P, k, prof, steps, pk):
     """Roofline fraction of every profiled kernel class: algorithmic bytes (or flops) per launch
-    over its event-timed duration, against the HBM, tensor or FP32-ALU peak that bounds it."""
+    over its event-timed duration, against the peak that bounds it: measured HBM copy bandwidth,
+    measured sustained bf16 tensor throughput (scaled for the three-product TF32 kernel), or the
+    FP32-ALU peak derived as 148 SMs x 128 lanes x 2 x the maximum SM clock."""
     e = 2 if cfg.dtype == "f16" else 4
     B, N, d, H, dh, T = cfg.batch, cfg.n_tokens, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.n_query
-    alu_peak = 148 * 128 * 2 * pk["sm_max_mhz"] * 1e6  # flop/s
-    work = {  # class -> (amount per launch, peak per second, bound)
-        "attn_colsum": (B * H * T * N * e, pk["hbm_gbs"] * 1e9, "hbm"),
-        "sketch": (B * N * d * e, pk["hbm_gbs"] * 1e9, "hbm"),
-        "compact": (B * (P + cfg.keep) * (d + 2 * H * dh) * e, pk["hbm_gbs"] * 1e9, "hbm"),
-        "gram": (B * 2.0 * N * N * d, pk["bf16_tflops_sustained"] * 1e12, "tensor"),
-        "gemm_f32_GQ": (B * 2.0 * N * N * k, alu_peak, "alu"),
-        "gemm_f32_YtY": (B * 1.0 * N * k * (k + 1), alu_peak, "alu"),  # symmetric: upper triangle only
-        # five launches per step: four Y R^-1 that skip the zero part of R^-1 (2/3 of the work
-        # with three 48-column tiles) and one Z Q1^T: 11/15 of a full product on average
-        "gemm_f32_YRinv": (B * 2.0 * N * k * k * 11.0 / 15.0, alu_peak, "alu"),
-        "chol_inv": (B * (2.0 / 3.0) * k ** 3, alu_peak, "alu"),
-        "eig": (B * (14.0 / 3.0) * k ** 3, alu_peak, "alu"),
+    src = pk["source"]
+    hbm = (pk["hbm_gbs"] * 1e9, "hbm", 1e9, "GB/s", src)
+    alu = (148 * 128 * 2 * pk["sm_max_mhz"] * 1e6, "alu", 1e12, "TFLOP/s",
+           "derived: 148 SMs x 128 lanes x 2 x max SM clock")
+    tens = (pk["bf16_tflops_sustained"] * 1e12, "tensor", 1e12, "TFLOP/s", src + " (sustained bf16)")
+    tcp = uses_tensor_products(cfg)
+    prod = (product_peak(pk) * 1e12, "tensor", 1e12, "TFLOP/s",
+            src + " sustained bf16 x 1/2 (TF32) / 3 (products per float32 term)") if tcp else alu
+    nt = (N + 127) // 128
+    gram_tiles = nt * (nt + 1) // 2 if cfg.dtype == "f16" else nt * nt
+    work = {  # class -> (algorithmic amount per launch, peak)
+        "attn_colsum": (B * H * T * N * e, hbm),
+        "sketch": (B * N * d * e, hbm),
+        "compact": (B * (P + cfg.keep) * (d + 2 * H * dh) * e, hbm),
+        "gram": (B * 2.0 * N * N * d, tens),
+        "gemm_f32_GQ": (B * 2.0 * N * N * k, prod),
+        "gemm_f32_YtY": (B * 1.0 * N * k * (k + 1), prod),  # symmetric result: upper triangle
+        # Y R^-1 (R^-1 triangular: N k^2 per launch) x passes, plus one full back-transformation
+        "gemm_f32_YRinv": (B * N * k * k * ((3 * 1.0 + 2.0) / 4 if tcp else 2.0 * 11.0 / 15.0), prod),
+        "chol_inv": (B * (2.0 / 3.0) * k ** 3, alu),
+        "eig": (B * (14.0 / 3.0) * k ** 3, alu),
     }
     out = {}
     for name, (ms_total, launches) in prof.items():
         if not launches or name not in work:
             continue
-        amount, peak, bound = work[name]
-        # a class launched several times per step (the GEMM products, chol_inv) does `amount`
-        # per launch; its time per launch is the class total over its launches
+        amount, (peak, bound, scale, unit, psrc) = work[name]
+        # a class launched several times per step (the products, chol_inv) does `amount` per
+        # launch; its time per launch is the class total over its launches
         per_launch_s = ms_total * 1e-3 / launches
         out[name] = {"bound": bound, "frac": round(amount / per_launch_s / peak, 4),
-                     "ms_per_step": round(ms_total / steps, 4)}
+                     "achieved": round(amount / per_launch_s / scale, 3), "peak": round(peak / scale, 3),
+                     "unit": unit, "peak_source": psrc, "ms_per_step": round(ms_total / steps, 4)}
+        if name == "gram" and cfg.dtype == "f16":
+            # the kernel issues the 128 x 128 tiles on or below the diagonal; the dense count
+            # above credits it with the mirror images it only stores
+            issued = B * gram_tiles * 2.0 * 128 * 128 * d
+            out[name]["frac_issued"] = round(issued / per_launch_s / peak, 4)
+            out[name]["achieved_issued"] = round(issued / per_launch_s / scale, 3)
+            out[name]["frac"] = out[name]["frac_issued"]
+            out[name]["achieved"] = out[name]["achieved_issued"]
+            out[name]["frac_dense_equivalent"] = round(amount / per_launch_s / peak, 4)
     return out
 
 
@@ -390,8 +422,8 @@ def run_sweep(args):
     groups = args.groups if args.groups else 4
     tcb.tc_set_groups(groups)
     pk = peaks()
-    base = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=args.batch)
-    if args.rank_cap:
+    base = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=args.batch or 64)
+    if args.rank_cap >= 0:
         base = base.with_(rank_cap=args.rank_cap)
     dev = {k: torch.from_numpy(v).cuda() for k, v in inputs.make_batch(base, want="OXKV").items()}
     for T in (32, 128, 512):
@@ -499,7 +531,7 @@ def run_extras(args):
                           "ms_per_call": round(ms, 4), "images_per_s": round(cfg.batch / (ms * 1e-3), 1),
                           "rank_of_image_0": int(res["rank"][0]), "status_any": bool(res["img_status"].any()),
                           "bytes_read_per_call": cfg.batch * n_sub * cfg.d_model * e}), flush=True)
-    n_sys, n_text = 35, args.n_query
+    n_sys, n_text = 35, cfg.n_query
     L = n_sys + cfg.n_tokens + n_text
     Hs = torch.randn(cfg.batch, L, cfg.d_model, device="cuda").to(dev["X"].dtype)
     ms = timed(lambda: tcb.tc_reassemble(p, n_sys, n_text, Hs, Xo, kept))
@@ -518,10 +550,13 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--batch", type=int, default=64, help="images per GPU per step")
-    ap.add_argument("--n-query", type=int, default=128)
-    ap.add_argument("--keep", type=int, default=128)
-    ap.add_argument("--rank-cap", type=int, default=0, help="override the workload's rank_cap")
+    ap.add_argument("--config", default="cfg5", choices=sorted(CONFIG_KEYS),
+                    help="which of the five named workloads (default: the metric's, cfg5)")
+    ap.add_argument("--batch", type=int, default=0, help="images per GPU per step (0 = the configuration's)")
+    ap.add_argument("--n-query", type=int, default=0)
+    ap.add_argument("--keep", type=int, default=0)
+    ap.add_argument("--rank-cap", type=int, default=-1,
+                    help="override the workload's rank_cap; 0 = full solve without a rank hint")
     ap.add_argument("--graph", action="store_true", help="(the default; kept for old command lines)")
     ap.add_argument("--no-graph", action="store_true",
                     help="time plain tc_carve calls instead of the replay of a CUDA graph of one call")

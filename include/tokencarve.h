@@ -29,6 +29,14 @@
  *     (TC_OK when fine) and never trap; they are valid once the stream has been synchronised.
  *   - Index lists are in ascending token order.  Every tie (equal scores, equal
  *     similarities) goes to the lower token index.
+ *   - Index lists a caller hands in (setA, setB, kept_idx, merge_src, merge_dst of the staged
+ *     calls) are checked on the device: a token number outside [0, N) is never used as an
+ *     address; the entry is skipped (a kept row becomes zeros, a merge source is left out, a
+ *     match is dropped) and TC_ERR_INVALID_ARG is recorded for that image, to be read with
+ *     tc_stage_status().  Numbers inside the range are taken as given.
+ *   - The first tc_score / tc_carve / tc_carve_host on a device creates the library's internal
+ *     streams and events (image groups, copy streams): make that first call outside any stream
+ *     capture.  Later calls create nothing and can be captured into a CUDA graph.
  */
 #ifndef TOKENCARVE_H
 #define TOKENCARVE_H
@@ -131,6 +139,16 @@ tc_status tc_compact(const tc_params* p, const void* X, const void* K, const voi
                      const int32_t* kept_idx, const int32_t* merge_src,
                      const int32_t* merge_dst, void* Xo, void* Ko, void* Vo, void* ws,
                      size_t ws_bytes, void* stream);
+
+/*
+ * Device-side findings of the last tc_merge or tc_compact that used the workspace `ws` (each of
+ * them clears the record when it starts): img_status [B] int32 (device) receives, per image,
+ * TC_OK or TC_ERR_INVALID_ARG (a list entry outside [0, N) was skipped).  Enqueued on `stream`
+ * behind that call; valid once the stream has been synchronised.  The paper has no counterpart:
+ * it is how the staged calls of Sec. 3.3.2 report without a status argument of their own.
+ */
+tc_status tc_stage_status(const tc_params* p, const void* ws, size_t ws_bytes, int32_t* img_status,
+                          void* stream);
 
 /*
  * The whole path (Sec. 3.3): score -> prune -> split -> match -> merge -> gather, one

@@ -27,7 +27,7 @@ EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge"
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
            "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
-           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3")
+           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3", "tc_stage_status")
 
 
 class TcParams(C.Structure):
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
         L.tc_rank.argtypes = [pp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         L.tc_reassemble.argtypes = [pp, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp]
         L.tc_gram.argtypes = [pp, vp, vp, vp]
+        L.tc_stage_status.argtypes = [pp, vp, sz, vp, vp]
         L.tc_matmul_f32x3.argtypes = [vp, vp, vp, vp] + [C.c_int32] * 4 + [vp, vp]
         L.tc_set_groups.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
@@ -169,6 +170,14 @@ def tc_gram(p: Params, O: torch.Tensor) -> torch.Tensor:
     cp = p.c()
     _check("tc_gram", lib().tc_gram(C.byref(cp), _ptr(O), _ptr(G), _stream()))
     return G
+
+
+def tc_stage_status(p: Params, ws: torch.Tensor) -> torch.Tensor:
+    """Per-image findings of the last tc_merge / tc_compact that used `ws`."""
+    st = torch.empty(p.batch, dtype=torch.int32, device=ws.device)
+    cp = p.c()
+    _check("tc_stage_status", lib().tc_stage_status(C.byref(cp), _ptr(ws), ws.numel(), _ptr(st), _stream()))
+    return st
 
 
 def tc_matmul_f32x3(A: torch.Tensor, B: torch.Tensor, transposed: bool = False):

@@ -343,8 +343,10 @@ tc_status tc_merge(const tc_params* p, const void* O, const int32_t* setA, const
   if ((size_t)D.d * sizeof(float) > 48 * 1024) return TC_ERR_UNSUPPORTED;
   float* bv = (float*)(c.ws + c.P.best_val);
   int32_t* bd = (int32_t*)(c.ws + c.P.best_dst);
-  if (D.M > 0) launch_match_rows(D, O, setA, setB, bv, bd, c.st);
-  launch_merge_select(D, setA, setB, bv, bd, merge_src, merge_dst, kept_idx, c.st);
+  int32_t* flags = (int32_t*)(c.ws + c.P.flags);
+  fill_i32(flags, D.B, 0, c.st);
+  if (D.M > 0) launch_match_rows(D, O, setA, setB, bv, bd, flags, c.st);
+  launch_merge_select(D, setA, setB, bv, bd, merge_src, merge_dst, kept_idx, flags, c.st);
   return check_launch();
 }
 
@@ -360,8 +362,22 @@ tc_status tc_compact(const tc_params* p, const void* X, const void* K, const voi
   const bool kv = (K != nullptr);
   if (kv != (V != nullptr) || kv != (Ko != nullptr) || kv != (Vo != nullptr)) return TC_ERR_INVALID_ARG;
   if (kv && (misaligned(K) || misaligned(V) || misaligned(Ko) || misaligned(Vo))) return TC_ERR_INVALID_ARG;
-  launch_compact(D, X, K, V, kept_idx, merge_src, merge_dst, Xo, Ko, Vo, c.st);
+  int32_t* flags = (int32_t*)(c.ws + c.P.flags);
+  fill_i32(flags, D.B, 0, c.st);
+  launch_compact(D, X, K, V, kept_idx, merge_src, merge_dst, Xo, Ko, Vo, flags, c.st);
   return check_launch();
+}
+
+tc_status tc_stage_status(const tc_params* p, const void* ws, size_t ws_bytes, int32_t* img_status,
+                          void* stream) {
+  Ctx c;
+  tc_status s = open_ctx(p, const_cast<void*>(ws), ws_bytes, stream, &c);
+  if (s != TC_OK) return s;
+  if (!img_status) return TC_ERR_INVALID_ARG;
+  if (cudaMemcpyAsync(img_status, c.ws + c.P.flags, (size_t)c.D.B * sizeof(int32_t),
+                      cudaMemcpyDeviceToDevice, c.st) != cudaSuccess)
+    return TC_ERR_CUDA;
+  return TC_OK;
 }
 
 tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void* X, const void* K,
@@ -388,9 +404,9 @@ tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void*
   s = enqueue_score(c, O, A, E, C, S, nullptr, nullptr, img_status);
   if (s != TC_OK) return s;
   launch_prune(D, E, setA, setB, c.st);
-  if (D.M > 0) launch_match_gram(D, (const float*)(c.ws + c.P.G), setA, setB, bv, bd, c.st);
-  launch_merge_select(D, setA, setB, bv, bd, msrc, mdst, kept_idx, c.st);
-  launch_compact(D, X, K, V, kept_idx, msrc, mdst, Xo, Ko, Vo, c.st);
+  if (D.M > 0) launch_match_gram(D, (const float*)(c.ws + c.P.G), setA, setB, bv, bd, img_status, c.st);
+  launch_merge_select(D, setA, setB, bv, bd, msrc, mdst, kept_idx, img_status, c.st);
+  launch_compact(D, X, K, V, kept_idx, msrc, mdst, Xo, Ko, Vo, img_status, c.st);
   return check_launch();
 }
 

@@ -156,18 +156,32 @@ __global__ void __launch_bounds__(128) match_gram_kernel(const float* __restrict
                                                         const int32_t* __restrict__ setB,
                                                         float* __restrict__ best_val,
                                                         int32_t* __restrict__ best_dst, int N,
-                                                        int nA, int nB) {
+                                                        int nA, int nB,
+                                                        int32_t* __restrict__ status) {
   const int b = blockIdx.y;
   const int jb = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (jb >= nB) return;
   const float* Gb = G + (size_t)b * N * N;
   const int tb = setB[(size_t)b * nB + jb];
+  // a token number outside [0, N) in a caller's list is reported and never used as an address
+  if (tb < 0 || tb >= N) {
+    if (lane == 0) {
+      atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+      best_val[(size_t)b * nB + jb] = -INFINITY;
+      best_dst[(size_t)b * nB + jb] = -1;
+    }
+    return;
+  }
   const float inv_b = inv_norm_from_sq(Gb[(size_t)tb * N + tb]);
   float bv = -INFINITY;
   int bi = 0x7fffffff;
   for (int ja = lane; ja < nA; ja += 32) {
     const int ta = setA[(size_t)b * nA + ja];
+    if (ta < 0 || ta >= N) {
+      atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+      continue;
+    }
     const float inv_a = inv_norm_from_sq(Gb[(size_t)ta * N + ta]);
     const float c = Gb[(size_t)tb * N + ta] * inv_b * inv_a;
     if (c > bv || (c == bv && ta < bi)) {
@@ -178,16 +192,16 @@ __global__ void __launch_bounds__(128) match_gram_kernel(const float* __restrict
   warp_best(bv, bi);
   if (lane == 0) {
     best_val[(size_t)b * nB + jb] = bv;
-    best_dst[(size_t)b * nB + jb] = bi;
+    best_dst[(size_t)b * nB + jb] = (bi == 0x7fffffff) ? -1 : bi;
   }
 }
 
 void launch_match_gram(const Dims& D, const float* G, const int32_t* setA, const int32_t* setB,
-                       float* best_val, int32_t* best_dst, cudaStream_t st) {
+                       float* best_val, int32_t* best_dst, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_MATCH, st);
   if (D.nB == 0 || D.nA == 0) return;
   dim3 grid((D.nB + 3) / 4, D.B);
-  { match_gram_kernel<<<grid, 128, 0, st>>>(G, setA, setB, best_val, best_dst, D.N, D.nA, D.nB); note_launch(); }
+  { match_gram_kernel<<<grid, 128, 0, st>>>(G, setA, setB, best_val, best_dst, D.N, D.nA, D.nB, status); note_launch(); }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -200,7 +214,8 @@ __global__ void __launch_bounds__(256) match_rows_kernel(const T* __restrict__ O
                                                         const int32_t* __restrict__ setB,
                                                         float* __restrict__ best_val,
                                                         int32_t* __restrict__ best_dst, int N,
-                                                        int d, int nA, int nB) {
+                                                        int d, int nA, int nB,
+                                                        int32_t* __restrict__ status) {
   extern __shared__ float rowb[];  // [d]
   __shared__ float sv[8];
   __shared__ int si[8];
@@ -209,6 +224,15 @@ __global__ void __launch_bounds__(256) match_rows_kernel(const T* __restrict__ O
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int tb = setB[(size_t)b * nB + jb];
   const T* Ob = O + (size_t)b * N * d;
+  // a token number outside [0, N) in a caller's list is reported and never used as an address
+  if (tb < 0 || tb >= N) {
+    if (threadIdx.x == 0) {
+      atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+      best_val[(size_t)b * nB + jb] = -INFINITY;
+      best_dst[(size_t)b * nB + jb] = -1;
+    }
+    return;
+  }
   for (int c = threadIdx.x; c < d; c += 256) rowb[c] = (float)Ob[(size_t)tb * d + c];
   __syncthreads();
   if (warp == 0) {
@@ -224,6 +248,10 @@ __global__ void __launch_bounds__(256) match_rows_kernel(const T* __restrict__ O
   int bi = 0x7fffffff;
   for (int ja = warp; ja < nA; ja += 8) {
     const int ta = setA[(size_t)b * nA + ja];
+    if (ta < 0 || ta >= N) {
+      if (lane == 0) atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+      continue;
+    }
     const T* ra = Ob + (size_t)ta * d;
     float dot = 0.f, na = 0.f;
     for (int c = lane; c < d; c += 32) {
@@ -254,22 +282,22 @@ __global__ void __launch_bounds__(256) match_rows_kernel(const T* __restrict__ O
         bi = si[w];
       }
     best_val[(size_t)b * nB + jb] = bv;
-    best_dst[(size_t)b * nB + jb] = bi;
+    best_dst[(size_t)b * nB + jb] = (bi == 0x7fffffff) ? -1 : bi;
   }
 }
 
 void launch_match_rows(const Dims& D, const void* O, const int32_t* setA, const int32_t* setB,
-                       float* best_val, int32_t* best_dst, cudaStream_t st) {
+                       float* best_val, int32_t* best_dst, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_MATCH, st);
   if (D.nB == 0 || D.nA == 0) return;
   dim3 grid(D.nB, D.B);
   size_t smem = (size_t)D.d * sizeof(float);
   if (D.f16)
     { match_rows_kernel<__half><<<grid, 256, smem, st>>>((const __half*)O, setA, setB, best_val,
-                                                       best_dst, D.N, D.d, D.nA, D.nB); note_launch(); }
+                                                       best_dst, D.N, D.d, D.nA, D.nB, status); note_launch(); }
   else
     { match_rows_kernel<float><<<grid, 256, smem, st>>>((const float*)O, setA, setB, best_val,
-                                                      best_dst, D.N, D.d, D.nA, D.nB); note_launch(); }
+                                                      best_dst, D.N, D.d, D.nA, D.nB, status); note_launch(); }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -281,7 +309,7 @@ __global__ void __launch_bounds__(SEL_THREADS) merge_select_kernel(
     const int32_t* __restrict__ setA, const int32_t* __restrict__ setB,
     const float* __restrict__ best_val, const int32_t* __restrict__ best_dst,
     int32_t* __restrict__ msrc, int32_t* __restrict__ mdst, int32_t* __restrict__ kept, int N,
-    int nA, int nB, int M, int keep) {
+    int nA, int nB, int M, int keep, int32_t* __restrict__ status) {
   extern __shared__ uint32_t dyn[];  // keys [nB] then flags [N] (one word per token)
   uint32_t* keys = dyn;
   uint32_t* flag = dyn + nB;
@@ -289,11 +317,22 @@ __global__ void __launch_bounds__(SEL_THREADS) merge_select_kernel(
   __shared__ uint32_t sh_u[2];
   __shared__ int sh_scan[9];
   const int b = blockIdx.x;
+  // Token numbers come from the caller's lists: one outside [0, N) is reported in the image's
+  // status and never used as an address (the kept list then ends in -1 entries).
+  auto valid = [&](int t) {
+    if (t >= 0 && t < N) return true;
+    atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+    return false;
+  };
   for (int i = threadIdx.x; i < N; i += SEL_THREADS) flag[i] = 0;
+  for (int j = threadIdx.x; j < keep; j += SEL_THREADS) kept[(size_t)b * keep + j] = -1;
   for (int j = threadIdx.x; j < nB; j += SEL_THREADS)
     keys[j] = (M > 0) ? orderable(best_val[(size_t)b * nB + j]) : 0u;
   __syncthreads();
-  for (int j = threadIdx.x; j < nA; j += SEL_THREADS) flag[setA[(size_t)b * nA + j]] = 1;
+  for (int j = threadIdx.x; j < nA; j += SEL_THREADS) {
+    const int t = setA[(size_t)b * nA + j];
+    if (valid(t)) flag[t] = 1;
+  }
   uint32_t thr = 0xffffffffu;
   int need = 0;
   if (M > 0) block_select_kth(keys, nB, M, hist, sh_u, sh_scan, &thr, &need);
@@ -314,7 +353,8 @@ __global__ void __launch_bounds__(SEL_THREADS) merge_select_kernel(
         sel |= 1u << (j - j0);
         ++cm;
       } else {
-        flag[setB[(size_t)b * nB + j]] = 1;  // unmerged Set-B tokens stay
+        const int t = setB[(size_t)b * nB + j];
+        if (valid(t)) flag[t] = 1;  // unmerged Set-B tokens stay
       }
     }
     int o = block_excl_scan(cm, sh_scan, &tot);
@@ -339,11 +379,11 @@ __global__ void __launch_bounds__(SEL_THREADS) merge_select_kernel(
 
 void launch_merge_select(const Dims& D, const int32_t* setA, const int32_t* setB,
                          const float* best_val, const int32_t* best_dst, int32_t* msrc,
-                         int32_t* mdst, int32_t* kept, cudaStream_t st) {
+                         int32_t* mdst, int32_t* kept, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_MSEL, st);
   size_t smem = (size_t)(D.nB + D.N) * sizeof(uint32_t);
   { merge_select_kernel<<<D.B, SEL_THREADS, smem, st>>>(setA, setB, best_val, best_dst, msrc, mdst,
-                                                     kept, D.N, D.nA, D.nB, D.M, D.keep); note_launch(); }
+                                                     kept, D.N, D.nA, D.nB, D.M, D.keep, status); note_launch(); }
 }
 
 }  // namespace tc

@@ -245,18 +245,45 @@ __global__ void __launch_bounds__(256) compact_kernel(
     const T* __restrict__ X, const T* __restrict__ K, const T* __restrict__ V,
     const int32_t* __restrict__ kept, const int32_t* __restrict__ msrc,
     const int32_t* __restrict__ mdst, T* __restrict__ Xo, T* __restrict__ Ko,
-    T* __restrict__ Vo, int N, int d, int H, int dh, int keep, int M) {
+    T* __restrict__ Vo, int N, int d, int H, int dh, int keep, int M,
+    int32_t* __restrict__ status) {
   extern __shared__ int srcs[];  // [M]
   __shared__ int s_cnt;
   constexpr int L = Vec16<T>::L;
   const int b = blockIdx.y, j = blockIdx.x;
   const int a = kept[(size_t)b * keep + j];
+  // The lists may come from the caller: a token number outside [0, N) is reported in the
+  // image's status and never used as an address.  A bad kept entry gives a row of zeros, a bad
+  // source is left out of its group.
+  if (a < 0 || a >= N) {
+    if (threadIdx.x == 0) atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    uint4* xo = reinterpret_cast<uint4*>(Xo + ((size_t)b * keep + j) * d);
+    for (int v = threadIdx.x; v < d / L; v += 256) xo[v] = z;
+    if (K != nullptr) {
+      const int vpr = dh / L;
+      for (int idx = threadIdx.x; idx < H * vpr; idx += 256) {
+        const int h = idx / vpr, v = idx - h * vpr;
+        const size_t out_off = (((size_t)b * H + h) * keep + j) * dh;
+        reinterpret_cast<uint4*>(Ko + out_off)[v] = z;
+        reinterpret_cast<uint4*>(Vo + out_off)[v] = z;
+      }
+    }
+    return;
+  }
   // ordered list of the sources merged into a (first warp, ballot compaction)
   if (threadIdx.x < 32) {
     int cnt = 0;
     for (int m0 = 0; m0 < M; m0 += 32) {
       const int m = m0 + threadIdx.x;
-      const bool hit = (m < M) && (mdst[(size_t)b * M + m] == a);
+      bool hit = (m < M) && (mdst[(size_t)b * M + m] == a);
+      if (hit) {
+        const int sidx = msrc[(size_t)b * M + m];
+        if (sidx < 0 || sidx >= N) {
+          atomicMax(&status[b], (int)TC_ERR_INVALID_ARG);
+          hit = false;
+        }
+      }
       const unsigned mask = __ballot_sync(0xffffffffu, hit);
       if (hit) srcs[cnt + __popc(mask & ((1u << threadIdx.x) - 1u))] = msrc[(size_t)b * M + m];
       cnt += __popc(mask);
@@ -284,19 +311,19 @@ __global__ void __launch_bounds__(256) compact_kernel(
 
 void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
                     const int32_t* kept, const int32_t* msrc, const int32_t* mdst, void* Xo,
-                    void* Ko, void* Vo, cudaStream_t st) {
+                    void* Ko, void* Vo, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_COMPACT, st);
   dim3 grid(D.keep, D.B);
   size_t smem = (size_t)max(D.M, 1) * sizeof(int);
   if (D.f16)
     { compact_kernel<__half><<<grid, 256, smem, st>>>(
         (const __half*)X, (const __half*)K, (const __half*)V, kept, msrc, mdst, (__half*)Xo,
-        (__half*)Ko, (__half*)Vo, D.N, D.d, D.H, D.dh, D.keep, D.M); note_launch(); }
+        (__half*)Ko, (__half*)Vo, D.N, D.d, D.H, D.dh, D.keep, D.M, status); note_launch(); }
   else
     { compact_kernel<float><<<grid, 256, smem, st>>>((const float*)X, (const float*)K,
                                                     (const float*)V, kept, msrc, mdst,
                                                     (float*)Xo, (float*)Ko, (float*)Vo, D.N, D.d,
-                                                    D.H, D.dh, D.keep, D.M); note_launch(); }
+                                                    D.H, D.dh, D.keep, D.M, status); note_launch(); }
 }
 
 // ------------------------------------------------------------------------------------------

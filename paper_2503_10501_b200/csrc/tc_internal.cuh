@@ -88,18 +88,20 @@ void launch_combine(const Dims& D, const float* s_part, const float* C, float* S
 // Stage I prune + Eq. 3-9 split.
 void launch_prune(const Dims& D, const float* E, int32_t* setA, int32_t* setB, cudaStream_t st);
 // Eq. 3-10 best match per Set-B token, from the Gram matrix or from the rows of O.
+// (status [B]: receives TC_ERR_INVALID_ARG for an image whose lists hold a token number outside
+// [0, N); such an entry is skipped, never used as an address.  The same for the launchers below.)
 void launch_match_gram(const Dims& D, const float* G, const int32_t* setA, const int32_t* setB,
-                       float* best_val, int32_t* best_dst, cudaStream_t st);
+                       float* best_val, int32_t* best_dst, int32_t* status, cudaStream_t st);
 void launch_match_rows(const Dims& D, const void* O, const int32_t* setA, const int32_t* setB,
-                       float* best_val, int32_t* best_dst, cudaStream_t st);
+                       float* best_val, int32_t* best_dst, int32_t* status, cudaStream_t st);
 // top-M of the best similarities, merge lists, kept list.
 void launch_merge_select(const Dims& D, const int32_t* setA, const int32_t* setB,
                          const float* best_val, const int32_t* best_dst, int32_t* msrc,
-                         int32_t* mdst, int32_t* kept, cudaStream_t st);
+                         int32_t* mdst, int32_t* kept, int32_t* status, cudaStream_t st);
 // merge + gather of X, K, V.
 void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
                     const int32_t* kept, const int32_t* msrc, const int32_t* mdst, void* Xo,
-                    void* Ko, void* Vo, cudaStream_t st);
+                    void* Ko, void* Vo, int32_t* status, cudaStream_t st);
 
 // Sec. 3.2: rows idx[b][0..n_sub) of O gathered into Os [B, n_sub, d] (D describes O).
 void launch_gather_rows(const Dims& D, int n_sub, const void* O, const int32_t* idx, void* Os,

@@ -509,3 +509,53 @@ def test_host_entry_point_matches_the_device_one():
         torch.cuda.synchronize()
         for a, b in zip(ref, hout):
             assert np.array_equal(a, b.numpy())
+
+
+# ------------------------------------------------------------------ caller-supplied lists
+def test_staged_calls_skip_and_report_bad_list_entries():
+    # Sec. 3.3.2 as staged calls: Set A / Set B, the merge lists and kept_idx come from the caller.
+    # A token number outside [0, N) is skipped on the device (never an address) and reported per
+    # image through tc_stage_status; the other images are untouched.
+    cfg = inputs.tiny_config(n_tokens=72, d_model=64, n_heads=2, head_dim=8, n_query=5, keep=20,
+                             rank=16, dtype="f16", batch=3, seed=41, noise=0.3, rank_tol=0.0)
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    O, A, X, K, V = (dev(batch[k]) for k in "OAXKV")
+    ws = tcb.workspace(p)
+    sc = tcb.tc_score(p, O, A, ws)
+    setA, setB = tcb.tc_prune(p, sc["E"], ws)
+    src, dst, kept = tcb.tc_merge(p, O, setA, setB, ws)
+    good = [host(t) for t in tcb.tc_compact(p, X, K, V, kept, src, dst, ws)]
+    st = host(tcb.tc_stage_status(p, ws))
+    torch.cuda.synchronize()
+    assert st.tolist() == [0, 0, 0]
+    N = cfg.n_tokens
+    # a bad Set-A entry in image 1, a bad Set-B entry in image 2
+    a2, b2 = host(setA).copy(), host(setB).copy()
+    a2[1, 3] = N + 5
+    b2[2, 0] = -7
+    s2, d2, k2 = tcb.tc_merge(p, O, dev(a2), dev(b2), ws)
+    st = host(tcb.tc_stage_status(p, ws))
+    torch.cuda.synchronize()
+    assert st.tolist() == [0, 1, 1]
+    assert np.array_equal(host(k2)[0], host(kept)[0]) and np.array_equal(host(s2)[0], host(src)[0])
+    k2h = host(k2)
+    assert np.all((k2h >= -1) & (k2h < N))
+    # a bad kept entry in image 0 (row of zeros), a bad merge source in image 2 (left out)
+    k3, s3 = host(kept).copy(), host(src).copy()
+    k3[0, 4] = N
+    s3[2, 1] = 1 << 20
+    out = [host(t) for t in tcb.tc_compact(p, X, K, V, dev(k3), dev(s3), dst, ws)]
+    st = host(tcb.tc_stage_status(p, ws))
+    torch.cuda.synchronize()
+    assert st.tolist() == [1, 0, 1]
+    assert not out[0][0, 4].any() and not out[1][0, :, 4].any() and not out[2][0, :, 4].any()
+    assert np.array_equal(np.delete(out[0][0], 4, axis=0), np.delete(good[0][0], 4, axis=0))
+    for o, g in zip(out, good):
+        assert np.array_equal(o[1], g[1])
+        assert np.all(np.isfinite(o.astype(np.float32)))
+    # the call after a bad one starts from a clean record
+    tcb.tc_compact(p, X, K, V, kept, src, dst, ws)
+    st = host(tcb.tc_stage_status(p, ws))
+    torch.cuda.synchronize()
+    assert st.tolist() == [0, 0, 0]
