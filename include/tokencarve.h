@@ -269,6 +269,20 @@ tc_status tc_reassemble(const tc_params* p, int32_t n_sys, int32_t n_text, const
                         void* stream);
 
 /*
+ * Conclusion (the surviving tokens keep their original position IDs): the rotary-encoding
+ * tables the layers after the compression need for the rows of the re-assembled sequence.
+ * Rotary position embedding as published: pair i of a head's dimensions turns by
+ * pos * base^(-2 i / head_dim).
+ *   pos      device, [n_rows] int32 position IDs (tc_reassemble's `pos`, flattened over the batch)
+ *   head_dim even, >= 2;  base > 1 (10000 for LLaVA-1.5's language model)
+ *   cos_out, sin_out  device, [n_rows, head_dim / 2] float32 out
+ * The angle is formed in double precision, so the tables are good to float32 rounding for any
+ * position.  Allocates nothing, only enqueues.
+ */
+tc_status tc_rope_tables(const int32_t* pos, int64_t n_rows, int32_t head_dim, float base,
+                         float* cos_out, float* sin_out, void* stream);
+
+/*
  * Number of image groups tc_score / tc_carve run side by side (1..8, default 4; the paper has no
  * counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
  * chains are enqueued on internal streams forked from `stream` and joined back into it before

@@ -23,7 +23,8 @@ Paper passages followed (TokenCarve, Sec. 3.3; Sec. 3.2 for `token_information`)
               the L_vc * rho Set-B tokens with the highest similarity are merged
               into their Set-A match with ToMe's average; the rest stay intact;
               L_vc tokens result.
-  Conclusion  surviving tokens keep their original positional relationships.
+  Conclusion  surviving tokens keep their original positional relationships
+              (`reassemble`, `rope_tables`).
 
 Readings taken where the paper is silent (each is a parameter or a stated rule):
   * r in Eq. 3-5/3-6 is the numerical rank  #{sigma_i > rank_tol * sigma_1};
@@ -177,6 +178,26 @@ def reassemble(Hs: np.ndarray, n_sys: int, n_vis: int, Xo: np.ndarray, kept_idx:
     rows = np.concatenate([Hs[:n_sys], np.asarray(Xo, Hs.dtype), Hs[n_sys + n_vis:]], axis=0)
     pos = np.concatenate([np.arange(n_sys), n_sys + kept, np.arange(n_sys + n_vis, L)])
     return rows, pos.astype(np.int64)
+
+
+def rope_tables(pos: Sequence[int], head_dim: int, base: float = 10000.0
+                ) -> Tuple[np.ndarray, np.ndarray]:
+    """Rotary-encoding tables for the rows of the re-assembled sequence (Conclusion: the
+    surviving tokens keep their original position IDs, so the layers after the compression
+    rotate queries and keys by those positions, not by the new row numbers).  Rotary position
+    embedding as published (RoFormer): pair i of a head's dimensions is rotated by the angle
+    pos * theta_i with theta_i = base^(-2 i / head_dim).  Returns (cos, sin), each
+    [len(pos), head_dim / 2], float64."""
+    assert head_dim % 2 == 0
+    half = head_dim // 2
+    cos = np.zeros((len(pos), half), F64)
+    sin = np.zeros((len(pos), half), F64)
+    for j, p in enumerate(pos):
+        for i in range(half):
+            theta = F64(base) ** (-2.0 * i / head_dim)
+            cos[j, i] = np.cos(F64(int(p)) * theta)
+            sin[j, i] = np.sin(F64(int(p)) * theta)
+    return cos, sin
 
 
 # --------------------------------------------------------------------------

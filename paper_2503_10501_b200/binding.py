@@ -27,7 +27,7 @@ EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge"
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
            "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
-           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3", "tc_stage_status")
+           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3", "tc_stage_status", "tc_rope_tables")
 
 
 class TcParams(C.Structure):
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
         L.tc_reassemble.argtypes = [pp, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp]
         L.tc_gram.argtypes = [pp, vp, vp, vp]
         L.tc_stage_status.argtypes = [pp, vp, sz, vp, vp]
+        L.tc_rope_tables.argtypes = [vp, C.c_int64, C.c_int32, C.c_float, vp, vp, vp]
         L.tc_matmul_f32x3.argtypes = [vp, vp, vp, vp] + [C.c_int32] * 4 + [vp, vp]
         L.tc_set_groups.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
@@ -170,6 +171,17 @@ def tc_gram(p: Params, O: torch.Tensor) -> torch.Tensor:
     cp = p.c()
     _check("tc_gram", lib().tc_gram(C.byref(cp), _ptr(O), _ptr(G), _stream()))
     return G
+
+
+def tc_rope_tables(pos: torch.Tensor, head_dim: int, base: float = 10000.0):
+    """cos / sin tables [..., head_dim / 2] (float32) for int32 position IDs of any shape."""
+    assert pos.dtype == torch.int32
+    shape = tuple(pos.shape) + (head_dim // 2,)
+    cos = torch.empty(shape, dtype=torch.float32, device=pos.device)
+    sin = torch.empty(shape, dtype=torch.float32, device=pos.device)
+    _check("tc_rope_tables", lib().tc_rope_tables(_ptr(pos), pos.numel(), head_dim, base, _ptr(cos),
+                                                  _ptr(sin), _stream()))
+    return cos, sin
 
 
 def tc_stage_status(p: Params, ws: torch.Tensor) -> torch.Tensor:

@@ -671,6 +671,15 @@ tc_status tc_reassemble(const tc_params* p, int32_t n_sys, int32_t n_text, const
   return check_launch();
 }
 
+tc_status tc_rope_tables(const int32_t* pos, int64_t n_rows, int32_t head_dim, float base,
+                         float* cos_out, float* sin_out, void* stream) {
+  if (!pos || !cos_out || !sin_out) return TC_ERR_INVALID_ARG;
+  if (n_rows < 1 || n_rows > 0x7fffffffLL || head_dim < 2 || (head_dim & 1) || !(base > 1.f))
+    return TC_ERR_INVALID_ARG;
+  launch_rope_tables(pos, n_rows, head_dim, (double)base, cos_out, sin_out, (cudaStream_t)stream);
+  return check_launch();
+}
+
 const char* tc_status_string(int32_t status) {
   switch (status) {
     case TC_OK: return "ok";

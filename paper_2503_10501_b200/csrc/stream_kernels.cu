@@ -393,4 +393,32 @@ void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, con
                                            n_sys, D.N, n_text, D.keep, D.d * D.esz / 16); note_launch(); }
 }
 
+// ------------------------------------------------------------------------------------------
+// Rotary-encoding tables for rows with given position IDs (Conclusion: the later layers rotate
+// by the original positions): cos / sin of pos * base^(-2 i / dh), i < dh / 2.  The angle is
+// formed and reduced in double precision (a float32 angle of a few thousand radians would cost
+// four digits); the tables are float32.  grid = rows, block = dh / 2 rounded up to a warp.
+// ------------------------------------------------------------------------------------------
+__global__ void rope_tables_kernel(const int32_t* __restrict__ pos, int half, double neg_log2_base_2_over_dh,
+                                   float* __restrict__ cosv, float* __restrict__ sinv) {
+  const size_t row = blockIdx.x;
+  const double p = (double)pos[row];
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    const double theta = exp2(neg_log2_base_2_over_dh * (double)i);
+    double sn, cs;
+    sincos(p * theta, &sn, &cs);
+    cosv[row * half + i] = (float)cs;
+    sinv[row * half + i] = (float)sn;
+  }
+}
+
+void launch_rope_tables(const int32_t* pos, long long rows, int head_dim, double base, float* cosv,
+                        float* sinv, cudaStream_t st) {
+  Scope scope_(KC_COMPACT, st);
+  const int half = head_dim / 2;
+  const int threads = min(256, (half + 31) / 32 * 32);
+  { rope_tables_kernel<<<(unsigned)rows, threads, 0, st>>>(pos, half, -2.0 * log2(base) / (double)head_dim,
+                                                         cosv, sinv); note_launch(); }
+}
+
 }  // namespace tc

@@ -111,6 +111,10 @@ void fill_i32(int32_t* p, int n, int v, cudaStream_t st);
 void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, const void* Xo,
                        const int32_t* kept, void* Ho, int32_t* pos, cudaStream_t st);
 
+// Conclusion: rotary tables cos / sin [rows][head_dim / 2] of the given position IDs.
+void launch_rope_tables(const int32_t* pos, long long rows, int head_dim, double base, float* cosv,
+                        float* sinv, cudaStream_t st);
+
 // G = O O^T (float32 out).
 tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 

@@ -453,6 +453,14 @@ def test_reassembled_sequence_and_positions():
         for b in range(3):
             rows, want = orc.reassemble(Hs[b], n_sys, cfg.n_tokens, host(Xo)[b], host(kept)[b])
             assert np.array_equal(host(Ho)[b], rows) and host(pos)[b].tolist() == want.tolist()
+        # rotary tables of the re-assembled rows, from their original positions
+        if n_sys == 35:
+            cos, sin = tcb.tc_rope_tables(pos, cfg.head_dim, 10000.0)
+            torch.cuda.synchronize()
+            for b in (0, 2):
+                co, so = orc.rope_tables(host(pos)[b].tolist(), cfg.head_dim, 10000.0)
+                assert np.max(np.abs(host(cos)[b] - co)) <= 1.5e-7
+                assert np.max(np.abs(host(sin)[b] - so)) <= 1.5e-7
 
 
 # ------------------------------------------------------------------ launch modes

@@ -482,3 +482,27 @@ def test_reassemble_closed_forms():
     rows, pos = orc.reassemble(vis, 0, n_vis, Xo, kept)
     assert np.array_equal(rows, Xo) and pos.tolist() == kept
 
+
+
+def test_rope_tables_closed_forms():
+    # Conclusion: rotary encodings of the layers after the compression use the original
+    # positions.  Pins: position 0 is the identity rotation; the first pair turns by exactly
+    # `pos` radians (theta_0 = 1); the last pair by pos * base^-(dh-2)/dh; every pair is a
+    # rotation (cos^2 + sin^2 = 1); rotating by a then by b is rotating by a + b.
+    dh, base = 16, 10000.0
+    pos = [0, 1, 7, 35, 611, 4095]
+    cos, sin = orc.rope_tables(pos, dh, base)
+    assert cos.shape == (6, 8) and sin.shape == (6, 8)
+    assert np.array_equal(cos[0], np.ones(8)) and np.array_equal(sin[0], np.zeros(8))
+    np.testing.assert_allclose(cos[:, 0], np.cos(np.array(pos, float)), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(sin[:, 0], np.sin(np.array(pos, float)), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(cos[3, 7], np.cos(35.0 / 10000.0 ** (14.0 / 16.0)), atol=1e-15)
+    np.testing.assert_allclose(cos ** 2 + sin ** 2, 1.0, atol=1e-14)
+    ca, sa = orc.rope_tables([13], dh, base)
+    cb, sb = orc.rope_tables([598], dh, base)
+    cc, sc = orc.rope_tables([611], dh, base)
+    np.testing.assert_allclose(ca * cb - sa * sb, cc, atol=1e-12)
+    np.testing.assert_allclose(sa * cb + ca * sb, sc, atol=1e-12)
+    # a different base changes every pair but the first
+    c2, _ = orc.rope_tables([35], dh, 500000.0)
+    assert c2[0, 0] == cos[3, 0] and np.all(c2[0, 1:] != cos[3, 1:])
