@@ -61,7 +61,20 @@ typedef enum {
   TC_ERR_SCRATCH_LIMIT = 8  /* tc_attn_score_noalloc: request larger than its built-in scratch */
 } tc_status;
 
-typedef enum { TC_F16 = 0, TC_F32 = 1 } tc_dtype;
+typedef enum { TC_F16 = 0, TC_F32 = 1, TC_BF16 = 2 } tc_dtype;
+
+/* tc_params.flags: variants kept beside the paper's own choices (0 = the paper's).
+ *   Eq. 3-10 matches on the rows of the attention output O.  TC_FLAG_SIM_X matches on the
+ *   hidden states X instead, TC_FLAG_SIM_MEAN_K on the mean over the heads of K (the features
+ *   ToMe, which Sec. 3.3.2 takes its merging from, matches on).
+ *   Sec. 3.3.2 merges with ToMe's plain average.  TC_FLAG_WEIGHTED_MERGE weights every token of
+ *   a merged group with its IPGS score E (Eq. 3-8); a group whose scores do not add up to a
+ *   positive number falls back to the plain average. */
+#define TC_FLAG_SIM_O 0u
+#define TC_FLAG_SIM_X 1u
+#define TC_FLAG_SIM_MEAN_K 2u
+#define TC_FLAG_SIM_MASK 3u
+#define TC_FLAG_WEIGHTED_MERGE 16u
 
 /* How Eq. 3-8 combines the two terms: on the raw C and S (the equation as printed), or on
  * C / sum(C) and S / sum(S) so that both terms have the same scale. */
@@ -87,7 +100,7 @@ typedef struct tc_params {
                          below k: only a k-dimensional dominant subspace is decomposed.  The
                          device checks r <= k - 8 and reports TC_ERR_RANK_CAP otherwise.
                          Singular values beyond the k-th are then reported as 0.             */
-  uint32_t flags;     /* reserved, 0                                                         */
+  uint32_t flags;     /* TC_FLAG_* variants, 0 = the paper's choices                         */
 } tc_params;
 
 /* Counts derived from the parameters (Sec. 3.3.1 last paragraph, Eq. 3-9):
@@ -120,7 +133,9 @@ tc_status tc_prune(const tc_params* p, const float* E, int32_t* setA, int32_t* s
  * Stage II matching (Eq. 3-10 and the paragraph after it).
  *   O [B,N,d], setA, setB in.  Cosine similarity of the L2-normalised rows of O between every
  *   Set-B and Set-A token; each Set-B token's best Set-A match; the M Set-B tokens with the
- *   highest best-similarity are merged.
+ *   highest best-similarity are merged.  The call matches on the rows of whatever [B,N,d]
+ *   matrix it is given (pass X with TC_FLAG_SIM_X); with TC_FLAG_SIM_MEAN_K the argument is
+ *   K [B,H,N,dh] and the features are its mean over the heads.
  *   merge_src [B,M] (ascending), merge_dst [B,M] (the match of merge_src[i]),
  *   kept_idx [B,keep] = Set A plus the unmerged Set-B tokens, ascending.
  */
@@ -139,6 +154,13 @@ tc_status tc_compact(const tc_params* p, const void* X, const void* K, const voi
                      const int32_t* kept_idx, const int32_t* merge_src,
                      const int32_t* merge_dst, void* Xo, void* Ko, void* Vo, void* ws,
                      size_t ws_bytes, void* stream);
+
+/* tc_compact with the score-weighted merge (TC_FLAG_WEIGHTED_MERGE as a staged call): E [B,N]
+ * float32 (device) are the weights, e.g. tc_score's E.  Everything else as tc_compact. */
+tc_status tc_compact_weighted(const tc_params* p, const void* X, const void* K, const void* V,
+                              const int32_t* kept_idx, const int32_t* merge_src,
+                              const int32_t* merge_dst, const float* E, void* Xo, void* Ko,
+                              void* Vo, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Device-side findings of the last tc_merge or tc_compact that used the workspace `ws` (each of

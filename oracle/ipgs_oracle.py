@@ -39,7 +39,9 @@ Readings taken where the paper is silent (each is a parameter or a stated rule):
   * "Norm" in Eq. 3-10 is the L2 row normalisation  x / max(|x|_2, 1e-12).
   * The merged token is the unweighted mean of the destination and every source
     that chose it; K and V get the same map per head (an extension: the paper
-    merges tokens, it does not say K/V).
+    merges tokens, it does not say K/V).  Variants kept beside the paper's choices:
+    matching on the hidden states or on the head-mean keys (ToMe's features), and a
+    mean weighted by the IPGS scores.
   * Output rows are in ascending original index; that index list is returned.
 
 Parity status: every function below is pinned by tests against closed forms,
@@ -282,8 +284,21 @@ def normalise_rows(O: np.ndarray) -> np.ndarray:
     return out
 
 
+def mean_heads(K: np.ndarray) -> np.ndarray:
+    """Mean over the heads of K [H, N, dh] -> [N, dh]: the token features ToMe matches on (the
+    paper's Sec. 3.3.2 takes its merging from ToMe but matches on the attention output; this is
+    the variant with ToMe's own choice of features)."""
+    K = np.asarray(K, F64)
+    out = np.zeros(K.shape[1:], F64)
+    for h in range(K.shape[0]):
+        out += K[h]
+    return out / K.shape[0]
+
+
 def similarity(O: np.ndarray, setA: Sequence[int], setB: Sequence[int]) -> np.ndarray:
-    """Simi_AB [nB, nA] = Norm(Z)[Set B] x Norm(Z)[Set A]^T  (Eq. 3-10)."""
+    """Simi_AB [nB, nA] = Norm(Z)[Set B] x Norm(Z)[Set A]^T  (Eq. 3-10).  Z is the matrix whose
+    rows describe the tokens: the attention output in the paper; the variants pass the hidden
+    states or the head-mean keys instead."""
     Zn = normalise_rows(O)
     return Zn[np.asarray(setB, int)] @ Zn[np.asarray(setA, int)].T
 
@@ -331,33 +346,65 @@ def merge(O: np.ndarray, setA: Sequence[int], setB: Sequence[int], M: int
 # --------------------------------------------------------------------------
 # merge + compaction of X, K, V
 # --------------------------------------------------------------------------
+def round_to_storage(x: np.ndarray, out_dtype) -> np.ndarray:
+    """Round float64 values once, to nearest even, to the storage type.  "bf16" (which numpy
+    does not have) gives float32 values that are exactly representable in bfloat16."""
+    if isinstance(out_dtype, str) and out_dtype == "bf16":
+        f = np.asarray(x, F64).astype(np.float32)
+        u = f.view(np.uint32).astype(np.uint64)
+        # float64 -> float32 -> bfloat16 is a double rounding only when the float32 lands
+        # exactly half-way between two bfloat16 values; redo those few from the float64
+        u16 = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint32) << 16
+        out = u16.astype(np.uint32).view(np.float32).reshape(f.shape)
+        tie = (u & 0xFFFF) == 0x8000
+        if np.any(tie):
+            x64 = np.asarray(x, F64)
+            lo = ((u >> 16) << 16).astype(np.uint32).view(np.float32).reshape(f.shape)
+            hi = (((u >> 16) + 1) << 16).astype(np.uint32).view(np.float32).reshape(f.shape)
+            mid = 0.5 * (lo.astype(F64) + hi.astype(F64))
+            fix = np.where(np.abs(x64) > np.abs(mid), hi, np.where(np.abs(x64) < np.abs(mid), lo, out))
+            out = np.where(tie.reshape(f.shape), fix, out).astype(np.float32)
+        return out
+    return np.asarray(x, F64).astype(out_dtype)
+
+
 def compact_rows(R: np.ndarray, kept_idx: Sequence[int], merge_src: Sequence[int],
-                 merge_dst: Sequence[int], out_dtype) -> np.ndarray:
+                 merge_dst: Sequence[int], out_dtype, weights: Optional[np.ndarray] = None
+                 ) -> np.ndarray:
     """Rows `kept_idx` of R [N, w]; a kept row that is a merge destination becomes the
     plain mean of itself and all its sources (ToMe average with unit sizes), computed
-    in float64 and rounded once (to nearest even) to the storage dtype."""
+    in float64 and rounded once (to nearest even) to the storage dtype.  With `weights`
+    [N] (the variant: IPGS scores, float32-rounded like every decision input) the mean is
+    weighted, sum(w_i R_i) / sum(w_i) over the group; a group whose weights do not add up to a
+    positive number falls back to the plain mean."""
     R = np.asarray(R, F64)
+    w = None if weights is None else np.asarray(weights, F64).astype(np.float32).astype(F64)
     out = np.empty((len(kept_idx), R.shape[1]), F64)
     for j, a in enumerate(kept_idx):
-        acc = R[int(a)].copy()
-        cnt = 1
-        for s, t in zip(merge_src, merge_dst):
-            if int(t) == int(a):
-                acc += R[int(s)]
-                cnt += 1
-        out[j] = acc / cnt
-    return out.astype(out_dtype)
+        group = [int(a)] + [int(s) for s, t in zip(merge_src, merge_dst) if int(t) == int(a)]
+        tot = sum(w[g] for g in group) if w is not None else 0.0
+        if w is not None and tot > 0.0 and len(group) > 1:
+            acc = np.zeros(R.shape[1], F64)
+            for g in group:
+                acc += w[g] * R[g]
+            out[j] = acc / tot
+        else:
+            acc = np.zeros(R.shape[1], F64)
+            for g in group:
+                acc += R[g]
+            out[j] = acc / len(group)
+    return round_to_storage(out, out_dtype)
 
 
 def compact(X: np.ndarray, K: Optional[np.ndarray], V: Optional[np.ndarray],
             kept_idx: Sequence[int], merge_src: Sequence[int], merge_dst: Sequence[int],
-            out_dtype) -> Dict[str, Optional[np.ndarray]]:
+            out_dtype, weights: Optional[np.ndarray] = None) -> Dict[str, Optional[np.ndarray]]:
     """X' [keep, d], K' / V' [H, keep, dh] under one merge map."""
     res: Dict[str, Optional[np.ndarray]] = {
-        "X": compact_rows(X, kept_idx, merge_src, merge_dst, out_dtype), "K": None, "V": None}
+        "X": compact_rows(X, kept_idx, merge_src, merge_dst, out_dtype, weights), "K": None, "V": None}
     for name, T in (("K", K), ("V", V)):
         if T is not None:
-            res[name] = np.stack([compact_rows(T[h], kept_idx, merge_src, merge_dst, out_dtype)
+            res[name] = np.stack([compact_rows(T[h], kept_idx, merge_src, merge_dst, out_dtype, weights)
                                   for h in range(T.shape[0])], axis=0)
     return res
 
@@ -368,16 +415,21 @@ def compact(X: np.ndarray, K: Optional[np.ndarray], V: Optional[np.ndarray],
 def carve(O: np.ndarray, A: np.ndarray, X: np.ndarray, K: Optional[np.ndarray],
           V: Optional[np.ndarray], keep: int, rho: float = 0.5, lam: float = 0.5,
           rank_tol: float = 0.0, score_norm: str = "none", n_merge: int = -1,
-          method: str = "lapack") -> Dict[str, object]:
+          method: str = "lapack", sim_source: str = "O", weighted: bool = False,
+          out_dtype=None) -> Dict[str, object]:
     """score -> prune -> split -> similarity -> match/select -> merge -> compact, one image.
 
     Inputs are taken as given (already rounded to their storage dtype); outputs X', K', V'
-    are rounded to X's dtype."""
+    are rounded to X's dtype (or `out_dtype`).  Variants beside the paper's choices:
+    sim_source "X" / "meanK" matches on the hidden states / the head-mean keys instead of the
+    attention output; weighted = True merges with the IPGS scores as weights."""
     N = O.shape[0]
     M, P, nA, nB = resolve_counts(N, keep, rho, n_merge)
     sc = score(O, A, lam, rank_tol, score_norm, method)
     setA, setB = prune_split(sc["E"], P, nA)
-    src, dst, kept = merge(O, setA, setB, M)
-    out = compact(X, K, V, kept, src, dst, X.dtype)
+    feats = {"O": O, "X": X, "meanK": None if K is None else mean_heads(K)}[sim_source]
+    src, dst, kept = merge(np.asarray(feats, F64), setA, setB, M)
+    out = compact(X, K, V, kept, src, dst, X.dtype if out_dtype is None else out_dtype,
+                  sc["E"] if weighted else None)
     return {**sc, "M": M, "P": P, "setA": setA, "setB": setB, "merge_src": src,
             "merge_dst": dst, "kept_idx": kept, "Xo": out["X"], "Ko": out["K"], "Vo": out["V"]}

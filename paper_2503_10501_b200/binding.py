@@ -16,7 +16,8 @@ import torch
 from . import build as _build
 
 TC_OK = 0
-TC_F16, TC_F32 = 0, 1
+TC_F16, TC_F32, TC_BF16 = 0, 1, 2
+TC_FLAG_SIM_X, TC_FLAG_SIM_MEAN_K, TC_FLAG_WEIGHTED_MERGE = 1, 2, 16
 TC_NORM_NONE, TC_NORM_SUM1 = 0, 1
 STATUS_NAMES = {0: "TC_OK", 1: "TC_ERR_INVALID_ARG", 2: "TC_ERR_UNSUPPORTED", 3: "TC_ERR_WORKSPACE",
                 4: "TC_ERR_NOT_CONVERGED", 5: "TC_ERR_CUDA", 6: "TC_ERR_RANK_CAP",
@@ -27,7 +28,8 @@ EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge"
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
            "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
-           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3", "tc_stage_status", "tc_rope_tables")
+           "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3", "tc_stage_status", "tc_rope_tables",
+           "tc_compact_weighted")
 
 
 class TcParams(C.Structure):
@@ -69,6 +71,7 @@ def lib() -> C.CDLL:
         L.tc_prune.argtypes = [pp, vp, vp, vp, vp, sz, vp]
         L.tc_merge.argtypes = [pp] + [vp] * 6 + [vp, sz, vp]
         L.tc_compact.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
+        L.tc_compact_weighted.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_carve.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_carve_host.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.tc_rank_workspace_bytes.argtypes = [pp, C.c_int32, C.POINTER(sz)]
@@ -111,17 +114,21 @@ class Params:
     score_norm: str = "none"
     max_sweeps: int = 30
     rank_cap: int = 0
+    sim_source: str = "O"      # "O" (Eq. 3-10 as printed), "X", "meanK"
+    weighted_merge: bool = False
 
     def c(self) -> TcParams:
         return TcParams(self.batch, self.n_tokens, self.d_model, self.n_heads, self.head_dim,
                         self.n_query, self.keep, self.n_merge, self.rho, self.lam, self.rank_tol,
-                        TC_F16 if self.dtype == "f16" else TC_F32,
+                        {"f16": TC_F16, "f32": TC_F32, "bf16": TC_BF16}[self.dtype],
                         TC_NORM_SUM1 if self.score_norm == "sum1" else TC_NORM_NONE,
-                        self.max_sweeps, self.rank_cap, 0)
+                        self.max_sweeps, self.rank_cap,
+                        {"O": 0, "X": TC_FLAG_SIM_X, "meanK": TC_FLAG_SIM_MEAN_K}[self.sim_source]
+                        | (TC_FLAG_WEIGHTED_MERGE if self.weighted_merge else 0))
 
     @property
     def torch_dtype(self):
-        return torch.float16 if self.dtype == "f16" else torch.float32
+        return {"f16": torch.float16, "bf16": torch.bfloat16, "f32": torch.float32}[self.dtype]
 
 
 def _check(fn: str, status: int) -> None:
@@ -318,6 +325,20 @@ def tc_compact(p: Params, X, K, V, kept, src, dst, ws=None):
                                           _ptr(src) if M else None, _ptr(dst) if M else None,
                                           _ptr(Xo), _ptr(Ko), _ptr(Vo), _ptr(ws), ws.numel(),
                                           _stream()))
+    return Xo, Ko, Vo
+
+
+def tc_compact_weighted(p: Params, X, K, V, kept, src, dst, E, ws=None):
+    """tc_compact with the IPGS scores E [B, N] as merge weights."""
+    dev = X.device
+    ws = ws if ws is not None else workspace(p, dev)
+    M = tc_counts(p)[0]
+    Xo, Ko, Vo = _outputs(p, dev, K is not None)
+    cp = p.c()
+    _check("tc_compact_weighted",
+           lib().tc_compact_weighted(C.byref(cp), _ptr(X), _ptr(K), _ptr(V), _ptr(kept),
+                                     _ptr(src) if M else None, _ptr(dst) if M else None, _ptr(E),
+                                     _ptr(Xo), _ptr(Ko), _ptr(Vo), _ptr(ws), ws.numel(), _stream()))
     return Xo, Ko, Vo
 
 

@@ -63,9 +63,12 @@ tc_status make_dims(const tc_params* p, Dims* out) {
   if (D.keep < 1 || D.keep > D.N) return TC_ERR_INVALID_ARG;
   if (!(p->lambda >= 0.f && p->lambda <= 1.f)) return TC_ERR_INVALID_ARG;
   if (!(p->rank_tol >= 0.f && p->rank_tol < 1.f)) return TC_ERR_INVALID_ARG;
-  if (p->dtype != TC_F16 && p->dtype != TC_F32) return TC_ERR_INVALID_ARG;
+  if (p->dtype != TC_F16 && p->dtype != TC_F32 && p->dtype != TC_BF16) return TC_ERR_INVALID_ARG;
   if (p->score_norm != TC_NORM_NONE && p->score_norm != TC_NORM_SUM1) return TC_ERR_INVALID_ARG;
-  if (p->flags != 0) return TC_ERR_INVALID_ARG;
+  if ((p->flags & ~(uint32_t)(TC_FLAG_SIM_MASK | TC_FLAG_WEIGHTED_MERGE)) != 0) return TC_ERR_INVALID_ARG;
+  D.sim_src = (int)(p->flags & TC_FLAG_SIM_MASK);
+  if (D.sim_src > 2) return TC_ERR_INVALID_ARG;
+  D.wmerge = (p->flags & TC_FLAG_WEIGHTED_MERGE) != 0;
   // M = floor(L_vc * rho), P = L_vc + M (Sec. 3.3.1 / 3.3.2), Set A = first half (Eq. 3-9)
   int M;
   if (p->n_merge < 0) {
@@ -82,7 +85,8 @@ tc_status make_dims(const tc_params* p, Dims* out) {
   D.nB = D.P - D.nA;
   if (D.M > D.nB) return TC_ERR_INVALID_ARG;
   D.f16 = (p->dtype == TC_F16);
-  D.esz = D.f16 ? 2 : 4;
+  D.bf16 = (p->dtype == TC_BF16);
+  D.esz = (D.f16 || D.bf16) ? 2 : 4;
   // rows must be whole 16-byte vectors for the gather; selection kernels cover N <= 4096
   if (((size_t)D.d * D.esz) % 16 != 0 || ((size_t)D.dh * D.esz) % 16 != 0) return TC_ERR_UNSUPPORTED;
   if (D.N > 4096) return TC_ERR_UNSUPPORTED;
@@ -158,13 +162,14 @@ Plan make_plan(const Dims& D) {
   P.kept = take(B * (size_t)D.keep * 4);
   P.rank = take(B * 4);
   P.flags = take(B * 4);
+  if (D.sim_src == 2) P.Kmean = take(B * N * (size_t)D.dh * 4);
   P.total = off;
   return P;
 }
 
 // float16 inputs go to the tensor cores; float32 inputs keep full precision on the plain ALUs
 tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st) {
-  if (D.f16) return launch_gram_tc(D, O, G, status, st);
+  if (D.f16 || D.bf16) return launch_gram_tc(D, O, G, status, st);
   return launch_gram_simt(D, O, G, st);
 }
 
@@ -345,14 +350,24 @@ tc_status tc_merge(const tc_params* p, const void* O, const int32_t* setA, const
   int32_t* bd = (int32_t*)(c.ws + c.P.best_dst);
   int32_t* flags = (int32_t*)(c.ws + c.P.flags);
   fill_i32(flags, D.B, 0, c.st);
-  if (D.M > 0) launch_match_rows(D, O, setA, setB, bv, bd, flags, c.st);
+  if (D.M > 0) {
+    if (D.sim_src == 2) {
+      // the features are the head-mean keys: `O` is K [B, H, N, dh]
+      float* Km = (float*)(c.ws + c.P.Kmean);
+      launch_mean_heads(D, O, Km, c.st);
+      launch_match_rows_f32(D, Km, D.dh, setA, setB, bv, bd, flags, c.st);
+    } else {
+      launch_match_rows(D, O, setA, setB, bv, bd, flags, c.st);  // rows of O, or of X
+    }
+  }
   launch_merge_select(D, setA, setB, bv, bd, merge_src, merge_dst, kept_idx, flags, c.st);
   return check_launch();
 }
 
-tc_status tc_compact(const tc_params* p, const void* X, const void* K, const void* V,
-                     const int32_t* kept_idx, const int32_t* merge_src, const int32_t* merge_dst,
-                     void* Xo, void* Ko, void* Vo, void* ws, size_t ws_bytes, void* stream) {
+static tc_status compact_impl(const tc_params* p, const void* X, const void* K, const void* V,
+                              const int32_t* kept_idx, const int32_t* merge_src,
+                              const int32_t* merge_dst, const float* E, void* Xo, void* Ko,
+                              void* Vo, void* ws, size_t ws_bytes, void* stream) {
   Ctx c;
   tc_status s = open_ctx(p, ws, ws_bytes, stream, &c);
   if (s != TC_OK) return s;
@@ -364,8 +379,23 @@ tc_status tc_compact(const tc_params* p, const void* X, const void* K, const voi
   if (kv && (misaligned(K) || misaligned(V) || misaligned(Ko) || misaligned(Vo))) return TC_ERR_INVALID_ARG;
   int32_t* flags = (int32_t*)(c.ws + c.P.flags);
   fill_i32(flags, D.B, 0, c.st);
-  launch_compact(D, X, K, V, kept_idx, merge_src, merge_dst, Xo, Ko, Vo, flags, c.st);
+  launch_compact(D, X, K, V, kept_idx, merge_src, merge_dst, Xo, Ko, Vo, E, flags, c.st);
   return check_launch();
+}
+
+tc_status tc_compact(const tc_params* p, const void* X, const void* K, const void* V,
+                     const int32_t* kept_idx, const int32_t* merge_src, const int32_t* merge_dst,
+                     void* Xo, void* Ko, void* Vo, void* ws, size_t ws_bytes, void* stream) {
+  return compact_impl(p, X, K, V, kept_idx, merge_src, merge_dst, nullptr, Xo, Ko, Vo, ws, ws_bytes,
+                      stream);
+}
+
+tc_status tc_compact_weighted(const tc_params* p, const void* X, const void* K, const void* V,
+                              const int32_t* kept_idx, const int32_t* merge_src,
+                              const int32_t* merge_dst, const float* E, void* Xo, void* Ko,
+                              void* Vo, void* ws, size_t ws_bytes, void* stream) {
+  if (E == nullptr) return TC_ERR_INVALID_ARG;
+  return compact_impl(p, X, K, V, kept_idx, merge_src, merge_dst, E, Xo, Ko, Vo, ws, ws_bytes, stream);
 }
 
 tc_status tc_stage_status(const tc_params* p, const void* ws, size_t ws_bytes, int32_t* img_status,
@@ -392,6 +422,9 @@ tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void*
   const bool kv = (K != nullptr);
   if (kv != (V != nullptr) || kv != (Ko != nullptr) || kv != (Vo != nullptr)) return TC_ERR_INVALID_ARG;
   if (kv && (misaligned(K) || misaligned(V) || misaligned(Ko) || misaligned(Vo))) return TC_ERR_INVALID_ARG;
+  if (D.sim_src == 2 && !kv) return TC_ERR_INVALID_ARG;  // the head-mean keys need K
+  if (D.sim_src != 0 && (size_t)(D.sim_src == 1 ? D.d : D.dh) * sizeof(float) > 48 * 1024)
+    return TC_ERR_UNSUPPORTED;
   float* E = (float*)(c.ws + c.P.E);
   float* C = (float*)(c.ws + c.P.C);
   float* S = (float*)(c.ws + c.P.S);
@@ -404,9 +437,19 @@ tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void*
   s = enqueue_score(c, O, A, E, C, S, nullptr, nullptr, img_status);
   if (s != TC_OK) return s;
   launch_prune(D, E, setA, setB, c.st);
-  if (D.M > 0) launch_match_gram(D, (const float*)(c.ws + c.P.G), setA, setB, bv, bd, img_status, c.st);
+  if (D.M > 0) {
+    if (D.sim_src == 0) {
+      launch_match_gram(D, (const float*)(c.ws + c.P.G), setA, setB, bv, bd, img_status, c.st);
+    } else if (D.sim_src == 1) {
+      launch_match_rows(D, X, setA, setB, bv, bd, img_status, c.st);
+    } else {
+      float* Km = (float*)(c.ws + c.P.Kmean);
+      launch_mean_heads(D, K, Km, c.st);
+      launch_match_rows_f32(D, Km, D.dh, setA, setB, bv, bd, img_status, c.st);
+    }
+  }
   launch_merge_select(D, setA, setB, bv, bd, msrc, mdst, kept_idx, img_status, c.st);
-  launch_compact(D, X, K, V, kept_idx, msrc, mdst, Xo, Ko, Vo, img_status, c.st);
+  launch_compact(D, X, K, V, kept_idx, msrc, mdst, Xo, Ko, Vo, D.wmerge ? E : nullptr, img_status, c.st);
   return check_launch();
 }
 

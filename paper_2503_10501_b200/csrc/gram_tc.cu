@@ -1,4 +1,5 @@
-// G = O O^T for float16 O on the 5th-generation tensor cores (tcgen05), float32 accumulate.
+// G = O O^T for float16 or bfloat16 O on the 5th-generation tensor cores (tcgen05), float32
+// accumulate.
 //
 // The SVD of Sec. 3.3.1 is taken through the Gram matrix (O O^T = U Sigma^2 U^T) and the cosine
 // similarities of Eq. 3-10 are its normalised entries, so this is the one dense contraction of
@@ -35,21 +36,24 @@ constexpr uint32_t SMEM_BYTES = STAGES * 2 * TILE_BYTES + 1024;  // + alignment 
 constexpr uint32_t TMEM_COLS = 256;  // two 128-column accumulators
 constexpr int DRAIN_KB = 2;          // stages per accumulation chunk (128 elements of K)
 
-// Instruction descriptor: D float32, A and B float16, both K-major, M = 128, N = 128.
-constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+// Instruction descriptor: D float32, A and B both float16 or both bfloat16 (operand format 0 / 1),
+// both K-major, M = 128, N = 128.
+constexpr uint32_t IDESC_F16 = (1u << 4) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+constexpr uint32_t IDESC_BF16 = IDESC_F16 | (1u << 7) | (1u << 10);
 
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accum) {
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc,
+                                         uint32_t accum) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accum)
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accum)
       : "memory");
 }
 
 __global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CUtensorMap map,
                                                      float* __restrict__ G, int N, int d,
-                                                     int tiles_per_image,
+                                                     int tiles_per_image, int bf16,
                                                      int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[STAGES];
@@ -141,7 +145,7 @@ __global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CU
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // 16 halves = 32 bytes further along K inside the swizzled row: +2 in 16-byte units
-            umma_f16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
+            umma_f16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), bf16 ? IDESC_BF16 : IDESC_F16,
                      (kb > c * DRAIN_KB || k > 0) ? 1u : 0u);
           }
           umma_commit(smem_u32(&bar_empty[s]));
@@ -232,7 +236,8 @@ tc_status launch_gram_tc(const Dims& D, const void* O, float* G, int32_t* status
   const cuuint64_t strides[2] = {(cuuint64_t)D.d * 2, (cuuint64_t)D.N * D.d * 2};
   const cuuint32_t box[3] = {BK, TILE, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(O), dims, strides, box,
+  CUresult r = enc(&map, D.bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+                   const_cast<void*>(O), dims, strides, box,
                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return TC_ERR_CUDA;
@@ -242,7 +247,7 @@ tc_status launch_gram_tc(const Dims& D, const void* O, float* G, int32_t* status
   const int nt = (D.N + TILE - 1) / TILE;
   const int tiles = nt * (nt + 1) / 2;
   Scope scope_(KC_GRAM, st);
-  gram_tc_kernel<<<D.B * tiles, 192, SMEM_BYTES, st>>>(map, G, D.N, D.d, tiles, status);
+  gram_tc_kernel<<<D.B * tiles, 192, SMEM_BYTES, st>>>(map, G, D.N, D.d, tiles, D.bf16 ? 1 : 0, status);
   note_launch();
   return TC_OK;
 }

@@ -35,6 +35,7 @@ __device__ __forceinline__ void cp_async_wait() {
 // ==========================================================================================
 __device__ inline float ld_f32(const float* p) { return __ldg(p); }
 __device__ inline float ld_f32(const __half* p) { return __half2float(__ldg(p)); }
+__device__ inline float ld_f32(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
 // flags for structured products
 constexpr int GEMM_SYM = 1;       // C is symmetric (A^T A): tiles below the diagonal are mirrored
@@ -651,12 +652,9 @@ static void gemm_tn_sym(const float* A, const float* B, float* C, int n, int K, 
 // G = O O^T for float32 inputs (and, until the tensor-core kernel takes over, float16 ones).
 tc_status launch_gram_simt(const Dims& D, const void* O, float* G, cudaStream_t st) {
   const size_t sO = (size_t)D.N * D.d, sG = (size_t)D.N * D.N;
-  if (D.f16)
-    gemm<__half, __half, false, true>((const __half*)O, (const __half*)O, G, D.N, D.N, D.d, D.d,
-                                      D.d, D.N, sO, sO, sG, D.B, st, KC_GRAM);
-  else
-    gemm<float, float, false, true>((const float*)O, (const float*)O, G, D.N, D.N, D.d, D.d, D.d,
-                                    D.N, sO, sO, sG, D.B, st, KC_GRAM);
+  TC_WITH_STORAGE_TYPE(D,
+    gemm<T, T, false, true>((const T*)O, (const T*)O, G, D.N, D.N, D.d, D.d, D.d, D.N, sO, sO, sG, D.B,
+                            st, KC_GRAM););
   return TC_OK;
 }
 
@@ -2453,23 +2451,21 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
   }
   auto sketch_into = [&](float* Y0) {
     Scope scope_(KC_SKETCH, st);
-    const int L = D.f16 ? 8 : 4;
+    const int L = 16 / D.esz;
     if (k % L == 0 && k / L <= 256 && (size_t)D.d * sizeof(float) <= 48 * 1024) {
       const int kg = k / L;
       const int rows = max(1, 256 / kg);
       dim3 block(kg, rows), grid((N + rows - 1) / rows, B);
       const size_t smem = (size_t)D.d * sizeof(float);
-      if (D.f16)
-        { sketch_vec_kernel<__half, 8><<<grid, block, smem, st>>>((const __half*)O, Y0, N, D.d, k); note_launch(); }
-      else
-        { sketch_vec_kernel<float, 4><<<grid, block, smem, st>>>((const float*)O, Y0, N, D.d, k); note_launch(); }
+      TC_WITH_STORAGE_TYPE(D,
+        sketch_vec_kernel<T, 16 / sizeof(T)><<<grid, block, smem, st>>>((const T*)O, Y0, N, D.d, k);
+        note_launch(););
     } else {
       dim3 grid(N, B);
       const int threads = (k + 31) / 32 * 32;
-      if (D.f16)
-        { sketch_kernel<__half><<<grid, threads, 0, st>>>((const __half*)O, Y0, N, D.d, k); note_launch(); }
-      else
-        { sketch_kernel<float><<<grid, threads, 0, st>>>((const float*)O, Y0, N, D.d, k); note_launch(); }
+      TC_WITH_STORAGE_TYPE(D,
+        sketch_kernel<T><<<grid, threads, 0, st>>>((const T*)O, Y0, N, D.d, k);
+        note_launch(););
     }
   };
   if (D.tcp) {

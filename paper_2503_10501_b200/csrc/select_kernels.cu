@@ -292,12 +292,20 @@ void launch_match_rows(const Dims& D, const void* O, const int32_t* setA, const 
   if (D.nB == 0 || D.nA == 0) return;
   dim3 grid(D.nB, D.B);
   size_t smem = (size_t)D.d * sizeof(float);
-  if (D.f16)
-    { match_rows_kernel<__half><<<grid, 256, smem, st>>>((const __half*)O, setA, setB, best_val,
-                                                       best_dst, D.N, D.d, D.nA, D.nB, status); note_launch(); }
-  else
-    { match_rows_kernel<float><<<grid, 256, smem, st>>>((const float*)O, setA, setB, best_val,
-                                                      best_dst, D.N, D.d, D.nA, D.nB, status); note_launch(); }
+  TC_WITH_STORAGE_TYPE(D,
+    match_rows_kernel<T><<<grid, 256, smem, st>>>((const T*)O, setA, setB, best_val, best_dst, D.N,
+                                                  D.d, D.nA, D.nB, status);
+    note_launch(););
+}
+
+void launch_match_rows_f32(const Dims& D, const float* F, int f, const int32_t* setA,
+                           const int32_t* setB, float* best_val, int32_t* best_dst,
+                           int32_t* status, cudaStream_t st) {
+  Scope scope_(KC_MATCH, st);
+  if (D.nB == 0 || D.nA == 0) return;
+  dim3 grid(D.nB, D.B);
+  { match_rows_kernel<float><<<grid, 256, (size_t)f * sizeof(float), st>>>(F, setA, setB, best_val, best_dst,
+                                                                         D.N, f, D.nA, D.nB, status); note_launch(); }
 }
 
 // ------------------------------------------------------------------------------------------

@@ -30,6 +30,26 @@ struct Vec16<__half> {
   }
 };
 template <>
+struct Vec16<__nv_bfloat16> {
+  static constexpr int L = 8;
+  __device__ static void unpack(const uint4& v, float* f) {
+    // a bfloat16 is the upper half of a float32
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static uint4 pack(const float* f) {
+    uint4 v;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    return v;
+  }
+};
+template <>
 struct Vec16<float> {
   static constexpr int L = 4;
   __device__ static void unpack(const uint4& v, float* f) {
@@ -45,6 +65,7 @@ struct Vec16<float> {
 };
 
 __device__ inline float to_f32(__half v) { return __half2float(v); }
+__device__ inline float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 __device__ inline float to_f32(float v) { return v; }
 
 // ------------------------------------------------------------------------------------------
@@ -116,7 +137,7 @@ __global__ void attn_colsum_kernel(const T* __restrict__ A, float* __restrict__ 
 void launch_attn_colsum(const Dims& D, const void* A, float* s_part, cudaStream_t st) {
   Scope scope_(KC_ATTN, st);
   const int R = D.H * D.T;
-  const int L = D.f16 ? 8 : 4;
+  const int L = 16 / D.esz;
   const bool vec = (D.N % L) == 0;
   const int ncg = vec ? D.N / L : D.N;
   int bx = min(ncg, 128);
@@ -125,17 +146,10 @@ void launch_attn_colsum(const Dims& D, const void* A, float* s_part, cudaStream_
   const int rpc = (R + D.chunks - 1) / D.chunks;
   dim3 grid(D.chunks, D.B), block(bx, by);
   size_t smem = (size_t)bx * by * (vec ? L : 1) * sizeof(float);
-  if (D.f16) {
-    if (vec)
-      { attn_colsum_kernel<__half, true><<<grid, block, smem, st>>>((const __half*)A, s_part, R, D.N, rpc); note_launch(); }
-    else
-      { attn_colsum_kernel<__half, false><<<grid, block, smem, st>>>((const __half*)A, s_part, R, D.N, rpc); note_launch(); }
-  } else {
-    if (vec)
-      { attn_colsum_kernel<float, true><<<grid, block, smem, st>>>((const float*)A, s_part, R, D.N, rpc); note_launch(); }
-    else
-      { attn_colsum_kernel<float, false><<<grid, block, smem, st>>>((const float*)A, s_part, R, D.N, rpc); note_launch(); }
-  }
+  TC_WITH_STORAGE_TYPE(D,
+    if (vec) { attn_colsum_kernel<T, true><<<grid, block, smem, st>>>((const T*)A, s_part, R, D.N, rpc); }
+    else { attn_colsum_kernel<T, false><<<grid, block, smem, st>>>((const T*)A, s_part, R, D.N, rpc); }
+    note_launch(););
 }
 
 // ------------------------------------------------------------------------------------------
@@ -215,7 +229,9 @@ void launch_combine(const Dims& D, const float* s_part, const float* C, float* S
 template <typename T>
 __device__ inline void merge_row(const T* __restrict__ base, size_t row_stride, int a,
                                  const int* srcs, int cnt, T* __restrict__ out, int nvec,
-                                 int v0, int vstep) {
+                                 int v0, int vstep, const float* wts) {
+  // wts: null for the plain mean, else wts[0] = weight of a, wts[1 + s] of source s, and
+  // wts[cnt + 1] = 1 / their sum
   constexpr int L = Vec16<T>::L;
   const uint4* pa = reinterpret_cast<const uint4*>(base + (size_t)a * row_stride);
   uint4* po = reinterpret_cast<uint4*>(out);
@@ -227,15 +243,32 @@ __device__ inline void merge_row(const T* __restrict__ base, size_t row_stride, 
     }
     float acc[8], f[8];
     Vec16<T>::unpack(va, acc);
+    if (wts != nullptr) {
+      const float wa = wts[0];
+#pragma unroll
+      for (int i = 0; i < L; ++i) acc[i] *= wa;
+    }
     for (int s = 0; s < cnt; ++s) {
       uint4 vs = __ldg(reinterpret_cast<const uint4*>(base + (size_t)srcs[s] * row_stride) + v);
       Vec16<T>::unpack(vs, f);
+      if (wts != nullptr) {
+        const float w = wts[1 + s];
 #pragma unroll
-      for (int i = 0; i < L; ++i) acc[i] += f[i];
+        for (int i = 0; i < L; ++i) acc[i] = fmaf(w, f[i], acc[i]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < L; ++i) acc[i] += f[i];
+      }
     }
-    const float den = (float)(cnt + 1);
+    if (wts != nullptr) {
+      const float inv = wts[cnt + 1];
 #pragma unroll
-    for (int i = 0; i < L; ++i) acc[i] = acc[i] / den;
+      for (int i = 0; i < L; ++i) acc[i] *= inv;
+    } else {
+      const float den = (float)(cnt + 1);
+#pragma unroll
+      for (int i = 0; i < L; ++i) acc[i] = acc[i] / den;
+    }
     po[v] = Vec16<T>::pack(acc);
   }
 }
@@ -246,9 +279,11 @@ __global__ void __launch_bounds__(256) compact_kernel(
     const int32_t* __restrict__ kept, const int32_t* __restrict__ msrc,
     const int32_t* __restrict__ mdst, T* __restrict__ Xo, T* __restrict__ Ko,
     T* __restrict__ Vo, int N, int d, int H, int dh, int keep, int M,
-    int32_t* __restrict__ status) {
-  extern __shared__ int srcs[];  // [M]
+    const float* __restrict__ E, int32_t* __restrict__ status) {
+  extern __shared__ int srcs[];  // [M] sources, then [M + 2] floats of weights
+  float* wts_sm = reinterpret_cast<float*>(srcs + M);
   __shared__ int s_cnt;
+  __shared__ int s_weighted;
   constexpr int L = Vec16<T>::L;
   const int b = blockIdx.y, j = blockIdx.x;
   const int a = kept[(size_t)b * keep + j];
@@ -288,14 +323,34 @@ __global__ void __launch_bounds__(256) compact_kernel(
       if (hit) srcs[cnt + __popc(mask & ((1u << threadIdx.x) - 1u))] = msrc[(size_t)b * M + m];
       cnt += __popc(mask);
     }
-    if (threadIdx.x == 0) s_cnt = cnt;
+    if (threadIdx.x == 0) {
+      s_cnt = cnt;
+      // score-weighted variant: the group's weights and the reciprocal of their sum; a sum
+      // that is not positive falls back to the plain mean
+      int weighted = 0;
+      if (E != nullptr && cnt > 0) {
+        const float* Eb = E + (size_t)b * N;
+        float tot = Eb[a];
+        wts_sm[0] = Eb[a];
+        for (int q = 0; q < cnt; ++q) {
+          wts_sm[1 + q] = Eb[srcs[q]];
+          tot += Eb[srcs[q]];
+        }
+        if (tot > 0.f) {
+          wts_sm[cnt + 1] = 1.0f / tot;
+          weighted = 1;
+        }
+      }
+      s_weighted = weighted;
+    }
   }
   __syncthreads();
   const int cnt = s_cnt;
+  const float* wts = s_weighted ? wts_sm : nullptr;
 
   // X row
   merge_row<T>(X + (size_t)b * N * d, d, a, srcs, cnt, Xo + ((size_t)b * keep + j) * d, d / L,
-               threadIdx.x, 256);
+               threadIdx.x, 256, wts);
   // K, V rows of every head
   if (K != nullptr) {
     const int vpr = dh / L;
@@ -303,27 +358,48 @@ __global__ void __launch_bounds__(256) compact_kernel(
       const int h = idx / vpr, v = idx - h * vpr;
       const size_t in_off = ((size_t)b * H + h) * N * dh;
       const size_t out_off = (((size_t)b * H + h) * keep + j) * dh;
-      merge_row<T>(K + in_off, dh, a, srcs, cnt, Ko + out_off, v + 1, v, vpr + 1);
-      merge_row<T>(V + in_off, dh, a, srcs, cnt, Vo + out_off, v + 1, v, vpr + 1);
+      merge_row<T>(K + in_off, dh, a, srcs, cnt, Ko + out_off, v + 1, v, vpr + 1, wts);
+      merge_row<T>(V + in_off, dh, a, srcs, cnt, Vo + out_off, v + 1, v, vpr + 1, wts);
     }
   }
 }
 
 void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
                     const int32_t* kept, const int32_t* msrc, const int32_t* mdst, void* Xo,
-                    void* Ko, void* Vo, int32_t* status, cudaStream_t st) {
+                    void* Ko, void* Vo, const float* E, int32_t* status, cudaStream_t st) {
   Scope scope_(KC_COMPACT, st);
   dim3 grid(D.keep, D.B);
-  size_t smem = (size_t)max(D.M, 1) * sizeof(int);
-  if (D.f16)
-    { compact_kernel<__half><<<grid, 256, smem, st>>>(
-        (const __half*)X, (const __half*)K, (const __half*)V, kept, msrc, mdst, (__half*)Xo,
-        (__half*)Ko, (__half*)Vo, D.N, D.d, D.H, D.dh, D.keep, D.M, status); note_launch(); }
-  else
-    { compact_kernel<float><<<grid, 256, smem, st>>>((const float*)X, (const float*)K,
-                                                    (const float*)V, kept, msrc, mdst,
-                                                    (float*)Xo, (float*)Ko, (float*)Vo, D.N, D.d,
-                                                    D.H, D.dh, D.keep, D.M, status); note_launch(); }
+  size_t smem = (size_t)max(D.M, 1) * sizeof(int) + (size_t)(D.M + 2) * sizeof(float);
+  TC_WITH_STORAGE_TYPE(D,
+    compact_kernel<T><<<grid, 256, smem, st>>>((const T*)X, (const T*)K, (const T*)V, kept, msrc, mdst,
+                                               (T*)Xo, (T*)Ko, (T*)Vo, D.N, D.d, D.H, D.dh, D.keep,
+                                               D.M, E, status);
+    note_launch(););
+}
+
+// ------------------------------------------------------------------------------------------
+// Km[b][x][:] = mean over the heads h of K[b][h][x][:], float32 (the features ToMe matches on).
+// grid (N, B), block dh (rounded up to a warp).
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void mean_heads_kernel(const T* __restrict__ K, float* __restrict__ Km, int H, int N,
+                                  int dh) {
+  const int x = blockIdx.x, b = blockIdx.y;
+  const float inv = 1.0f / (float)H;
+  for (int c = threadIdx.x; c < dh; c += blockDim.x) {
+    float s = 0.f;
+    for (int h = 0; h < H; ++h) s += to_f32(K[(((size_t)b * H + h) * N + x) * dh + c]);
+    Km[((size_t)b * N + x) * dh + c] = s * inv;
+  }
+}
+
+void launch_mean_heads(const Dims& D, const void* K, float* Km, cudaStream_t st) {
+  Scope scope_(KC_MATCH, st);
+  dim3 grid(D.N, D.B);
+  const int threads = min(256, (D.dh + 31) / 32 * 32);
+  TC_WITH_STORAGE_TYPE(D,
+    mean_heads_kernel<T><<<grid, threads, 0, st>>>((const T*)K, Km, D.H, D.N, D.dh);
+    note_launch(););
 }
 
 // ------------------------------------------------------------------------------------------

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libtokencarve.
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
@@ -17,7 +18,10 @@ struct Dims {
   bool full;      // rank_cap == 0
   bool tcp;       // the subspace solve runs its products on the tensor cores (split panels)
   int esz;        // bytes per element of O, A, X, K, V
-  bool f16;
+  bool f16;       // float16 storage
+  bool bf16;      // bfloat16 storage (neither: float32)
+  int sim_src;    // Eq. 3-10 features: 0 rows of O (the paper), 1 rows of X, 2 head-mean of K
+  bool wmerge;    // merge with the IPGS scores as weights instead of the plain mean
   int chunks;     // row chunks of the attention column-mean
   int max_sweeps;
   float lambda, rank_tol;
@@ -38,6 +42,7 @@ struct Plan {
   size_t setA, setB, best_val, best_dst, msrc, mdst, kept;  // int32 / f32 lists
   size_t rank;     // [B] int32
   size_t flags;    // [B] int32 device status scratch
+  size_t Kmean;    // [B, N, dh] f32: head-mean keys (sim_src == 2 only)
   // tensor-core subspace solve (Dims::tcp)
   size_t PA, PB;   // two sets of tall panels: [B][N][k] row-major and, panel_T_off bytes
                    // further on, [B][k][N] transposed
@@ -61,6 +66,21 @@ __device__ __forceinline__ float tf32_round(float x) {
 int tn_parts(int k);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Runs `...` with T bound to the storage type of the call.
+#define TC_WITH_STORAGE_TYPE(D, ...)      \
+  do {                                    \
+    if ((D).bf16) {                       \
+      using T = __nv_bfloat16;            \
+      __VA_ARGS__                         \
+    } else if ((D).f16) {                 \
+      using T = __half;                   \
+      __VA_ARGS__                         \
+    } else {                              \
+      using T = float;                    \
+      __VA_ARGS__                         \
+    }                                     \
+  } while (0)
 
 // Running count of kernels this library has launched (host side, all streams).
 void note_launch(int n = 1);
@@ -99,9 +119,16 @@ void launch_merge_select(const Dims& D, const int32_t* setA, const int32_t* setB
                          const float* best_val, const int32_t* best_dst, int32_t* msrc,
                          int32_t* mdst, int32_t* kept, int32_t* status, cudaStream_t st);
 // merge + gather of X, K, V.
+// E: the per-token weights [B, N] of the score-weighted merge, or null for the plain mean.
 void launch_compact(const Dims& D, const void* X, const void* K, const void* V,
                     const int32_t* kept, const int32_t* msrc, const int32_t* mdst, void* Xo,
-                    void* Ko, void* Vo, int32_t* status, cudaStream_t st);
+                    void* Ko, void* Vo, const float* E, int32_t* status, cudaStream_t st);
+// Km [B, N, dh] float32 = mean over the heads of K [B, H, N, dh].
+void launch_mean_heads(const Dims& D, const void* K, float* Km, cudaStream_t st);
+// launch_match_rows on float32 features F [B, N, f] whatever the storage type of the call.
+void launch_match_rows_f32(const Dims& D, const float* F, int f, const int32_t* setA,
+                           const int32_t* setB, float* best_val, int32_t* best_dst,
+                           int32_t* status, cudaStream_t st);
 
 // Sec. 3.2: rows idx[b][0..n_sub) of O gathered into Os [B, n_sub, d] (D describes O).
 void launch_gather_rows(const Dims& D, int n_sub, const void* O, const int32_t* idx, void* Os,

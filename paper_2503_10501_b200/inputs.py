@@ -46,7 +46,7 @@ class CarveConfig:
     n_heads: int           # H
     head_dim: int          # dh
     n_query: int           # T
-    dtype: str             # "f16" | "f32"
+    dtype: str             # "f16" | "f32" | "bf16"
     rank: int              # r of the low-rank part of O
     noise: float           # sigma_n
     tau: float             # std of the attention logits
@@ -88,9 +88,21 @@ CONFIGS: Dict[str, CarveConfig] = {
 def np_dtype(dtype: str):
     if dtype == "f16":
         return np.float16
-    if dtype == "f32":
-        return np.float32
+    if dtype in ("f32", "bf16"):
+        return np.float32   # numpy has no bfloat16: its values are held in float32 (see to_storage)
     raise ValueError(f"unknown dtype {dtype!r}")
+
+
+def to_storage(a: np.ndarray, dtype: str) -> np.ndarray:
+    """One rounding (to nearest even) to the storage type.  "bf16" returns float32 values that
+    are exactly representable in bfloat16 (the top 16 bits of a float32), so that a torch
+    tensor made from them converts to torch.bfloat16 without a second rounding."""
+    if dtype != "bf16":
+        return a.astype(np_dtype(dtype))
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
+    return u.astype(np.uint32).view(np.float32).reshape(f.shape)
 
 
 def _softmax_last(z: np.ndarray) -> np.ndarray:
@@ -108,7 +120,7 @@ def make_image(cfg: CarveConfig, b: int, want: str = "OAXKV") -> Dict[str, np.nd
     depend on which others were requested.
     """
     N, d, H, dh, T, r = cfg.n_tokens, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.n_query, cfg.rank
-    dt = np_dtype(cfg.dtype)
+    dt = cfg.dtype
     root = np.random.SeedSequence(cfg.seed + 1000 * b)
     s_o, s_a, s_x, s_k, s_v, s_d = [np.random.default_rng(s) for s in root.spawn(6)]
     out: Dict[str, np.ndarray] = {}
@@ -157,26 +169,26 @@ def make_image(cfg: CarveConfig, b: int, want: str = "OAXKV") -> Dict[str, np.nd
         Om += cfg.noise * s_o.standard_normal((N, d))
         row_rms = float(np.sqrt(np.mean(Om * Om)))
         apply_copies(Om, 0, 0.1 * row_rms)
-        out["O"] = Om.astype(dt)
+        out["O"] = to_storage(Om, dt)
     if "A" in want:
         z = s_a.standard_normal((H, T, N), dtype=np.float32)
         z *= np.float32(cfg.tau)
         if cfg.hot:
             hot_idx = s_a.choice(N, size=cfg.hot, replace=False)
             z[:, :, hot_idx] += np.float32(cfg.hot_bias)
-        out["A"] = _softmax_last(z).astype(dt)
+        out["A"] = to_storage(_softmax_last(z), dt)
     if "X" in want:
         Xm = s_x.standard_normal((N, d), dtype=np.float32)
         apply_copies(Xm, 0, 0.1)
-        out["X"] = Xm.astype(dt)
+        out["X"] = to_storage(Xm, dt)
     if "K" in want:
         Km = s_k.standard_normal((H, N, dh), dtype=np.float32)
         apply_copies(Km, 1, 0.1)
-        out["K"] = Km.astype(dt)
+        out["K"] = to_storage(Km, dt)
     if "V" in want:
         Vm = s_v.standard_normal((H, N, dh), dtype=np.float32)
         apply_copies(Vm, 1, 0.1)
-        out["V"] = Vm.astype(dt)
+        out["V"] = to_storage(Vm, dt)
     return out
 
 

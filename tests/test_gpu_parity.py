@@ -11,12 +11,18 @@ import parity_util as pu
 pytestmark = pytest.mark.gpu
 
 
-def dev(a):
-    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+def dev(a, bf16=False):
+    """Device tensor of a numpy array; bf16: the float32 array holds bfloat16 values."""
+    if a is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t.to(torch.bfloat16) if bf16 else t
 
 
 def host(t):
-    return None if t is None else t.cpu().numpy()
+    if t is None:
+        return None
+    return (t.float() if t.dtype == torch.bfloat16 else t).cpu().numpy()
 
 
 def params_of(cfg, **over):
@@ -29,14 +35,19 @@ def params_of(cfg, **over):
 
 def run_staged(p, batch, with_kv=True):
     """Every stage through its own entry point, each fed with the previous stage's CUDA output."""
-    O, A, X = dev(batch["O"]), dev(batch["A"]), dev(batch["X"])
-    K = dev(batch["K"]) if with_kv else None
-    V = dev(batch["V"]) if with_kv else None
+    bf = p.dtype == "bf16"
+    O, A, X = dev(batch["O"], bf), dev(batch["A"], bf), dev(batch["X"], bf)
+    K = dev(batch["K"], bf) if with_kv else None
+    V = dev(batch["V"], bf) if with_kv else None
     ws = tcb.workspace(p)
     sc = tcb.tc_score(p, O, A, ws)
     setA, setB = tcb.tc_prune(p, sc["E"], ws)
-    src, dst, kept = tcb.tc_merge(p, O, setA, setB, ws)
-    Xo, Ko, Vo = tcb.tc_compact(p, X, K, V, kept, src, dst, ws)
+    feats = {"O": O, "X": X, "meanK": K}[p.sim_source]     # what Eq. 3-10 is taken on
+    src, dst, kept = tcb.tc_merge(p, feats, setA, setB, ws)
+    if p.weighted_merge:
+        Xo, Ko, Vo = tcb.tc_compact_weighted(p, X, K, V, kept, src, dst, sc["E"], ws)
+    else:
+        Xo, Ko, Vo = tcb.tc_compact(p, X, K, V, kept, src, dst, ws)
     cX, cK, cV, ckept, cstatus = tcb.tc_carve(p, O, A, X, K, V, ws)
     torch.cuda.synchronize()
     res = {k: host(v) for k, v in sc.items()}
@@ -56,7 +67,8 @@ def image_slice(res, b, with_kv=True):
 
 def cfgp_of(p):
     return dict(keep=p.keep, rho=p.rho, n_merge=p.n_merge, lam=p.lam, rank_tol=p.rank_tol,
-                score_norm=p.score_norm)
+                score_norm=p.score_norm, sim_source=p.sim_source, weighted=p.weighted_merge,
+                dtype=p.dtype)
 
 
 def check_config(cfg, images, with_kv=True, max_flips=0, **over):
@@ -567,3 +579,39 @@ def test_staged_calls_skip_and_report_bad_list_entries():
     st = host(tcb.tc_stage_status(p, ws))
     torch.cuda.synchronize()
     assert st.tolist() == [0, 0, 0]
+
+
+# ------------------------------------------------------------------ variants beside the paper's choices
+@pytest.mark.parametrize("sim_source,weighted", [("X", False), ("meanK", False), ("O", True),
+                                                 ("meanK", True)])
+def test_variants_similarity_source_and_weighted_merge(sim_source, weighted):
+    # Eq. 3-10 on the hidden states or on the head-mean keys (ToMe's features) instead of the
+    # attention output, and the merge of Sec. 3.3.2 weighted by the IPGS scores of Eq. 3-8:
+    # staged and fused calls against the oracle's same variant, ragged shapes and twins
+    cfg = inputs.tiny_config(n_tokens=200, d_model=264, n_heads=3, head_dim=24, n_query=37, keep=61,
+                             rank=40, dtype="f16", batch=3, seed=29, noise=0.01, tau=2.0,
+                             rank_tol=2e-3, dup_frac=0.05)
+    check_config(cfg, range(3), rank_cap=96, max_flips=2, sim_source=sim_source,
+                 weighted_merge=weighted)
+
+
+def test_variants_at_a_named_workload():
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=4)
+    check_config(cfg, [0, 3], max_flips=2, sim_source="meanK", weighted_merge=True, score_norm="sum1")
+
+
+@pytest.mark.parametrize("rank_cap", [0, 96])
+def test_bfloat16_storage(rank_cap):
+    # bfloat16 in and out (the storage type of most LLaVA checkpoints): the Gram matrix comes from
+    # the same tensor-core kernel with bfloat16 operands, the scores obey the same float32
+    # tolerances (the inputs are taken as given), the merged rows are one bfloat16 rounding of the
+    # float32 mean
+    cfg = inputs.tiny_config(n_tokens=200, d_model=264, n_heads=3, head_dim=24, n_query=37, keep=61,
+                             rank=40, dtype="bf16", batch=3, seed=37, noise=0.01, tau=2.0,
+                             rank_tol=2e-3, dup_frac=0.05)
+    check_config(cfg, range(3), rank_cap=rank_cap, max_flips=2)
+
+
+def test_bfloat16_at_a_named_workload():
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=4, dtype="bf16")
+    check_config(cfg, [1, 2], max_flips=2)

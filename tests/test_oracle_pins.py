@@ -506,3 +506,55 @@ def test_rope_tables_closed_forms():
     # a different base changes every pair but the first
     c2, _ = orc.rope_tables([35], dh, 500000.0)
     assert c2[0, 0] == cos[3, 0] and np.all(c2[0, 1:] != cos[3, 1:])
+
+
+def test_variant_weighted_merge_and_mean_key_similarity():
+    # Variants beside Sec. 3.3.2's choices.  Weighted merge: equal weights give the plain mean;
+    # a source of weight zero leaves its destination untouched; the weighted sum is preserved
+    # (sum_j W_j X'_j = sum over the survivors of w_x X_x); weights that add up to nothing fall
+    # back to the plain mean.  Mean-key features: with one head they are the keys themselves; the
+    # similarity on them is the brute-force cosine.
+    rng = np.random.default_rng(12)
+    N, w = 10, 6
+    R = rng.standard_normal((N, w))
+    kept, src, dst = [0, 2, 5, 7], [3, 4, 9], [2, 2, 7]
+    plain = orc.compact_rows(R, kept, src, dst, np.float64)
+    same = orc.compact_rows(R, kept, src, dst, np.float64, weights=np.full(N, 0.25))
+    np.testing.assert_allclose(same, plain, rtol=1e-15)
+    wts = rng.uniform(0.5, 2.0, N)
+    wts32 = wts.astype(np.float32).astype(np.float64)
+    out = orc.compact_rows(R, kept, src, dst, np.float64, weights=wts)
+    np.testing.assert_allclose(out[1], (wts32[2] * R[2] + wts32[3] * R[3] + wts32[4] * R[4])
+                               / (wts32[2] + wts32[3] + wts32[4]), rtol=1e-14)
+    assert np.array_equal(out[0], R[0]) and np.array_equal(out[2], R[5])
+    W = np.array([wts32[0], wts32[2] + wts32[3] + wts32[4], wts32[5], wts32[7] + wts32[9]])
+    surv = [0, 2, 3, 4, 5, 7, 9]
+    np.testing.assert_allclose((W[:, None] * out).sum(0), sum(wts32[x] * R[x] for x in surv), rtol=1e-13)
+    w0 = wts.copy()
+    w0[9] = 0.0
+    np.testing.assert_allclose(orc.compact_rows(R, kept, src, dst, np.float64, weights=w0)[3], R[7], rtol=1e-15)
+    np.testing.assert_allclose(orc.compact_rows(R, kept, src, dst, np.float64, weights=np.zeros(N)), plain)
+    K = rng.standard_normal((3, N, 4))
+    np.testing.assert_allclose(orc.mean_heads(K), K.mean(axis=0), rtol=1e-15)
+    assert np.array_equal(orc.mean_heads(K[:1]), K[0])
+    F = orc.mean_heads(K)
+    sim = orc.similarity(F, [1, 4], [0, 6, 8])
+    for j, b in enumerate([0, 6, 8]):
+        for i, a in enumerate([1, 4]):
+            want = F[b] @ F[a] / (np.linalg.norm(F[b]) * np.linalg.norm(F[a]))
+            assert abs(sim[j, i] - want) < 1e-14
+
+
+def test_round_to_storage_bf16_is_round_to_nearest_even():
+    # bfloat16 keeps the top 16 bits of a float32: 1 + 2^-8 is half-way between 1 and 1 + 2^-7
+    # (goes to the even one, 1), 1 + 3 * 2^-8 half-way between 1 + 2^-7 and 1 + 2^-6 (goes up)
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -30, -2.5, 3.0e38, 1e-40])
+    got = orc.round_to_storage(x, "bf16")
+    assert got.dtype == np.float32
+    assert got[0] == 1.0 and got[1] == 1.0 and got[2] == 1.0 + 2.0 ** -6 and got[3] == 1.0 + 2.0 ** -7
+    assert got[4] == -2.5
+    assert np.all((got.view(np.uint32) & 0xFFFF) == 0)
+    rng = np.random.default_rng(2)
+    y = rng.standard_normal(2000) * 10.0
+    r = orc.round_to_storage(y, "bf16").astype(np.float64)
+    assert np.all(np.abs(r - y) <= np.abs(y) * 2.0 ** -8)
