@@ -10,7 +10,8 @@ the paper itself names (an SVD, a matrix product, a sort); there is no blocking,
 fusion or reordering.  A LAPACK-free one-sided Jacobi SVD (`svd_jacobi`) is kept
 beside the LAPACK call so each can check the other.
 
-Paper passages followed (TokenCarve, Sec. 3.3; Sec. 3.2 for `token_information`):
+Paper passages followed (TokenCarve, Sec. 3.3; Sec. 3.2 for `token_information`; Sec. 3.1
+Eq. 3-1 / 3-2 for `layer2_probe`, the producer of the matrices the compression reads):
   Sec. 3.2    the information quantity of the visual tokens is measured by the
               matrix rank of their rows of the attention-output matrix, followed
               as tokens are removed (Visual Token Information curve; appendix
@@ -43,6 +44,9 @@ Readings taken where the paper is silent (each is a parameter or a stated rule):
     matching on the hidden states or on the head-mean keys (ToMe's features), and a
     mean weighted by the IPGS scores.
   * Output rows are in ascending original index; that index list is returned.
+  * `layer2_probe`: the attention is causal (a decoder-only LLM), Q and K arrive with
+    their rotary encodings applied, Z is taken before the output projection with the
+    heads side by side, and the rows whose attention Eq. 3-7 averages are a parameter.
 
 Parity status: every function below is pinned by tests against closed forms,
 invariants, brute force or an independent routine, except `carve` as a whole
@@ -200,6 +204,77 @@ def rope_tables(pos: Sequence[int], head_dim: int, base: float = 10000.0
             cos[j, i] = np.cos(F64(int(p)) * theta)
             sin[j, i] = np.sin(F64(int(p)) * theta)
     return cos, sin
+
+
+# --------------------------------------------------------------------------
+# the layer-2 probe: what IPGS reads from the second LLM layer (Sec. 3.1, Sec. 3.2)
+# --------------------------------------------------------------------------
+def layer2_probe(Q: np.ndarray, K: np.ndarray, V: np.ndarray, n_sys: int, n_vis: int,
+                 probe_rows: Sequence[int], causal: bool = True
+                 ) -> Tuple[np.ndarray, np.ndarray]:
+    """Attention of one layer on the sequence [system, visual, prompt] (Sec. 3.1):
+    A = Softmax(Q K^T / sqrt(d_k)) per head (Eq. 3-1), Z = A V (Eq. 3-2), and from them the two
+    things the compression reads (Sec. 3.2, Sec. 3.3.1): the visual rows of Z with the heads
+    side by side, O [n_vis, H * dh], and the attention the rows `probe_rows` pay to the visual
+    tokens, A_slice [H, len(probe_rows), n_vis] (the slice Eq. 3-7 averages).
+    Q, K, V: [H, L, dh], L = n_sys + n_vis + n_text, taken as given (rotary encodings, if any,
+    already applied).  causal: row i attends to the keys j <= i, as in a decoder-only LLM (the
+    paper's LLaVA models); False lets every row see every key.
+    Plain loops over heads and rows; nothing is blocked or fused."""
+    Q = np.asarray(Q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    H, L, dh = Q.shape
+    scale = 1.0 / np.sqrt(F64(dh))
+    O = np.zeros((n_vis, H * dh), F64)
+    A_slice = np.zeros((H, len(probe_rows), n_vis), F64)
+    for h in range(H):
+        for i in list(range(n_sys, n_sys + n_vis)) + [int(r) for r in probe_rows]:
+            last = i + 1 if causal else L
+            logits = np.array([np.dot(Q[h, i], K[h, j]) * scale for j in range(last)])
+            logits -= logits.max()
+            w = np.exp(logits)
+            w /= w.sum()
+            if n_sys <= i < n_sys + n_vis:
+                z = np.zeros(dh, F64)
+                for j in range(last):
+                    z += w[j] * V[h, j]
+                O[i - n_sys, h * dh:(h + 1) * dh] = z
+        for t, i in enumerate(probe_rows):
+            last = int(i) + 1 if causal else L
+            logits = np.array([np.dot(Q[h, int(i)], K[h, j]) * scale for j in range(last)])
+            logits -= logits.max()
+            w = np.exp(logits)
+            w /= w.sum()
+            for x in range(n_vis):
+                j = n_sys + x
+                A_slice[h, t, x] = w[j] if j < last else 0.0
+    return O, A_slice
+
+
+def layer2_probe_matrix(Q: np.ndarray, K: np.ndarray, V: np.ndarray, n_sys: int, n_vis: int,
+                        probe_rows: Sequence[int], causal: bool = True
+                        ) -> Tuple[np.ndarray, np.ndarray]:
+    """The same quantities by the textbook route (one matrix product per head, a masked
+    softmax over whole rows): fast enough for the benchmark-sized checks, and a second route
+    the loop version is pinned against."""
+    Q = np.asarray(Q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    H, L, dh = Q.shape
+    O = np.zeros((n_vis, H * dh), F64)
+    A_slice = np.zeros((H, len(probe_rows), n_vis), F64)
+    rows = np.array(list(range(n_sys, n_sys + n_vis)) + [int(r) for r in probe_rows])
+    for h in range(H):
+        S = (Q[h, rows] @ K[h].T) / np.sqrt(F64(dh))
+        if causal:
+            S = np.where(np.arange(L)[None, :] <= rows[:, None], S, -np.inf)
+        S = S - S.max(axis=1, keepdims=True)
+        W = np.exp(S)
+        W /= W.sum(axis=1, keepdims=True)
+        O[:, h * dh:(h + 1) * dh] = W[:n_vis] @ V[h]
+        A_slice[h] = W[n_vis:, n_sys:n_sys + n_vis]
+    return O, A_slice
 
 
 # --------------------------------------------------------------------------

@@ -558,3 +558,49 @@ def test_round_to_storage_bf16_is_round_to_nearest_even():
     y = rng.standard_normal(2000) * 10.0
     r = orc.round_to_storage(y, "bf16").astype(np.float64)
     assert np.all(np.abs(r - y) <= np.abs(y) * 2.0 ** -8)
+
+
+def test_layer2_probe_closed_forms():
+    # Eq. 3-1 / 3-2 on [system, visual, prompt].  Pins: every probability row sums to one over
+    # the keys it may see, so its visual part sums to at most one; all keys equal => uniform
+    # probabilities and Z = the running mean of V (causal) or the mean of V (not causal); one key
+    # that dominates a row => that row of Z is that key's V; causal rows do not change when later
+    # keys and values change; the loop route and the matrix route agree.
+    rng = np.random.default_rng(21)
+    H, dh, n_sys, n_vis, n_text = 2, 8, 3, 6, 4
+    L = n_sys + n_vis + n_text
+    Q = rng.standard_normal((H, L, dh))
+    K = rng.standard_normal((H, L, dh))
+    V = rng.standard_normal((H, L, dh))
+    probe = list(range(n_sys + n_vis, L))
+    O, A = orc.layer2_probe(Q, K, V, n_sys, n_vis, probe)
+    O2, A2 = orc.layer2_probe_matrix(Q, K, V, n_sys, n_vis, probe)
+    np.testing.assert_allclose(O, O2, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(A, A2, rtol=1e-12, atol=1e-14)
+    assert O.shape == (n_vis, H * dh) and A.shape == (H, n_text, n_vis)
+    assert np.all(A >= 0) and np.all(A.sum(axis=2) <= 1.0 + 1e-12)
+    # equal keys: uniform attention
+    Ke = np.broadcast_to(K[:, :1], K.shape).copy()
+    Oe, Ae = orc.layer2_probe(Q, Ke, V, n_sys, n_vis, probe)
+    for x in range(n_vis):
+        i = n_sys + x
+        np.testing.assert_allclose(Oe[x, :dh], V[0, :i + 1].mean(axis=0), rtol=1e-12)
+    for t, i in enumerate(probe):
+        np.testing.assert_allclose(Ae[:, t, :], 1.0 / (i + 1), rtol=1e-12)
+    On, An = orc.layer2_probe(Q, Ke, V, n_sys, n_vis, probe, causal=False)
+    np.testing.assert_allclose(On[:, dh:], np.broadcast_to(V[1].mean(axis=0), (n_vis, dh)), rtol=1e-12)
+    np.testing.assert_allclose(An, 1.0 / L, rtol=1e-12)
+    # a dominating key
+    Kd = K.copy()
+    Kd[0, 2] = 80.0 * Q[0, n_sys + 4] / np.linalg.norm(Q[0, n_sys + 4])
+    Od, _ = orc.layer2_probe(Q, Kd, V, n_sys, n_vis, probe)
+    np.testing.assert_allclose(Od[4, :dh], V[0, 2], atol=1e-6)
+    # causality: later keys / values do not reach earlier rows
+    K2, V2 = K.copy(), V.copy()
+    K2[:, n_sys + 3:] += 1.0
+    V2[:, n_sys + 3:] -= 2.0
+    O3, _ = orc.layer2_probe(Q, K2, V2, n_sys, n_vis, probe)
+    assert np.array_equal(O3[:3], O[:3]) and not np.allclose(O3[3:], O[3:])
+    # a probe row in front of some visual tokens sees nothing of them
+    _, Ap = orc.layer2_probe(Q, K, V, n_sys, n_vis, [n_sys + 1])
+    assert np.all(Ap[:, 0, 2:] == 0.0) and np.all(Ap[:, 0, :2] > 0.0)
