@@ -291,6 +291,30 @@ tc_status tc_reassemble(const tc_params* p, int32_t n_sys, int32_t n_text, const
                         void* stream);
 
 /*
+ * The layer-2 probe (Sec. 3.1, Eq. 3-1 and 3-2; Sec. 3.2: the visual slice): what the compression
+ * reads from the second LLM layer, produced from that layer's queries, keys and values without
+ * writing its probability matrix out.  The sequence is [n_sys system, n_tokens visual, n_text
+ * prompt] tokens, L = n_sys + n_tokens + n_text.
+ *   p        batch, n_tokens, n_heads, head_dim (128), d_model (= n_heads * head_dim), dtype
+ *            (TC_F16 or TC_BF16), n_query = the number T of probe rows
+ *   Q, K, V  device, [B, H, L, dh], taken as given (rotary encodings already applied)
+ *   O        device out, [B, n_tokens, H * dh]: the visual rows of Z = Softmax(Q K^T / sqrt(dh)) V,
+ *            heads side by side (tc_score's O); NULL = not wanted (V and ws may then be NULL)
+ *   A        device out, [B, H, T, n_tokens]: the attention the rows probe_start .. probe_start +
+ *            T - 1 of the sequence pay to the visual tokens (tc_score's A); NULL = not wanted
+ *   The attention is causal (row i sees the keys j <= i); a visual token a probe row cannot see
+ *   gets probability 0.  float32 scores and sums, probabilities rounded to the storage type
+ *   before they multiply V.
+ *   img_status [B] as in tc_score.  ws: device scratch of tc_probe_workspace_bytes() bytes (the
+ *   transposed V), owned by the caller; nothing is allocated; asynchronous on `stream`.
+ * Returns TC_ERR_UNSUPPORTED for float32 storage or head_dim != 128.
+ */
+tc_status tc_probe_workspace_bytes(const tc_params* p, int32_t n_sys, int32_t n_text, size_t* bytes);
+tc_status tc_probe(const tc_params* p, int32_t n_sys, int32_t n_text, int32_t probe_start,
+                   const void* Q, const void* K, const void* V, void* O, void* A,
+                   int32_t* img_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Conclusion (the surviving tokens keep their original position IDs): the rotary-encoding
  * tables the layers after the compression need for the rows of the re-assembled sequence.
  * Rotary position embedding as published: pair i of a head's dimensions turns by

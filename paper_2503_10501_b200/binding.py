@@ -29,7 +29,7 @@ EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge"
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
            "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
            "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3", "tc_stage_status", "tc_rope_tables",
-           "tc_compact_weighted")
+           "tc_compact_weighted", "tc_probe", "tc_probe_workspace_bytes")
 
 
 class TcParams(C.Structure):
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         L.tc_gram.argtypes = [pp, vp, vp, vp]
         L.tc_stage_status.argtypes = [pp, vp, sz, vp, vp]
         L.tc_rope_tables.argtypes = [vp, C.c_int64, C.c_int32, C.c_float, vp, vp, vp]
+        L.tc_probe_workspace_bytes.argtypes = [pp, C.c_int32, C.c_int32, C.POINTER(sz)]
+        L.tc_probe.argtypes = [pp, C.c_int32, C.c_int32, C.c_int32] + [vp] * 7 + [sz, vp]
         L.tc_matmul_f32x3.argtypes = [vp, vp, vp, vp] + [C.c_int32] * 4 + [vp, vp]
         L.tc_set_groups.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
@@ -178,6 +180,28 @@ def tc_gram(p: Params, O: torch.Tensor) -> torch.Tensor:
     cp = p.c()
     _check("tc_gram", lib().tc_gram(C.byref(cp), _ptr(O), _ptr(G), _stream()))
     return G
+
+
+def tc_probe(p: Params, n_sys: int, n_text: int, probe_start: int, Q, K, V, want_o=True, want_a=True,
+             ws=None, out=None):
+    """Layer-2 probe: returns (O [B, N, H*dh] or None, A [B, H, T, N] or None, img_status)."""
+    dev = Q.device
+    cp = p.c()
+    if ws is None and want_o:
+        n = C.c_size_t(0)
+        _check("tc_probe_workspace_bytes",
+               lib().tc_probe_workspace_bytes(C.byref(cp), n_sys, n_text, C.byref(n)))
+        ws = torch.empty(max(int(n.value), 256), dtype=torch.uint8, device=dev)
+    if out is None:
+        O = torch.empty(p.batch, p.n_tokens, p.n_heads * p.head_dim, dtype=p.torch_dtype, device=dev) if want_o else None
+        A = torch.empty(p.batch, p.n_heads, p.n_query, p.n_tokens, dtype=p.torch_dtype, device=dev) if want_a else None
+        st = torch.empty(p.batch, dtype=torch.int32, device=dev)
+    else:
+        O, A, st = out
+    _check("tc_probe", lib().tc_probe(C.byref(cp), n_sys, n_text, probe_start, _ptr(Q), _ptr(K), _ptr(V),
+                                      _ptr(O), _ptr(A), _ptr(st), _ptr(ws), ws.numel() if ws is not None else 0,
+                                      _stream()))
+    return O, A, st
 
 
 def tc_rope_tables(pos: torch.Tensor, head_dim: int, base: float = 10000.0):

@@ -714,6 +714,38 @@ tc_status tc_reassemble(const tc_params* p, int32_t n_sys, int32_t n_text, const
   return check_launch();
 }
 
+tc_status tc_probe_workspace_bytes(const tc_params* p, int32_t n_sys, int32_t n_text, size_t* bytes) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  if (!bytes || n_sys < 0 || n_text < 0) return TC_ERR_INVALID_ARG;
+  *bytes = probe_workspace_bytes(D.B, D.H, n_sys + D.N + n_text, D.dh);
+  return TC_OK;
+}
+
+tc_status tc_probe(const tc_params* p, int32_t n_sys, int32_t n_text, int32_t probe_start,
+                   const void* Q, const void* K, const void* V, void* O, void* A,
+                   int32_t* img_status, void* ws, size_t ws_bytes, void* stream) {
+  Dims D;
+  tc_status s = make_dims(p, &D);
+  if (s != TC_OK) return s;
+  if (n_sys < 0 || n_text < 0) return TC_ERR_INVALID_ARG;
+  const int L = n_sys + D.N + n_text;
+  if (!Q || !K || !img_status || (!O && !A) || (O && (!V || !ws))) return TC_ERR_INVALID_ARG;
+  if (misaligned(Q) || misaligned(K) || (V && misaligned(V)) || (O && misaligned(O)) ||
+      (A && misaligned(A)) || (ws && misaligned(ws)))
+    return TC_ERR_INVALID_ARG;
+  if (A && (probe_start < 0 || probe_start + D.T > L)) return TC_ERR_INVALID_ARG;
+  if (D.esz != 2 || D.dh != 128 || D.d != D.H * D.dh) return TC_ERR_UNSUPPORTED;
+  if (O && ws_bytes < probe_workspace_bytes(D.B, D.H, L, D.dh)) return TC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  fill_i32(img_status, D.B, 0, st);
+  s = launch_probe(D.B, D.H, D.dh, L, n_sys, D.N, probe_start, D.T, Q, K, V, O, A, ws, img_status, st,
+                   D.bf16 ? 1 : 0);
+  if (s != TC_OK) return s;
+  return check_launch();
+}
+
 tc_status tc_rope_tables(const int32_t* pos, int64_t n_rows, int32_t head_dim, float base,
                          float* cos_out, float* sin_out, void* stream) {
   if (!pos || !cos_out || !sin_out) return TC_ERR_INVALID_ARG;

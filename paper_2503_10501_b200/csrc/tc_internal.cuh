@@ -142,6 +142,13 @@ void launch_reassemble(const Dims& D, int n_sys, int n_text, const void* Hs, con
 void launch_rope_tables(const int32_t* pos, long long rows, int head_dim, double base, float* cosv,
                         float* sinv, cudaStream_t st);
 
+// Layer-2 probe (Eq. 3-1 / 3-2): visual rows of the attention output and the probe rows'
+// attention to the visual tokens, from Q, K, V [B, H, L, dh] (16-bit storage, dh = 128).
+size_t probe_workspace_bytes(int B, int H, int L, int dh);
+tc_status launch_probe(int B, int H, int dh, int L, int n_sys, int n_vis, int probe_start, int n_probe,
+                       const void* Q, const void* K, const void* V, void* O, void* A, void* ws,
+                       int32_t* status, cudaStream_t st, int bf);
+
 // G = O O^T (float32 out).
 tc_status launch_gram(const Dims& D, const void* O, float* G, int32_t* status, cudaStream_t st);
 
