@@ -544,6 +544,67 @@ def run_extras(args):
                                    "note": "the call also allocates its two outputs"}}), flush=True)
 
 
+def run_probe(args):
+    """One JSON line for the layer-2 probe (tc_probe) at the LLaVA-1.5 layout of the bench point:
+    35 system + 576 visual + 64 prompt tokens, 32 heads x 128, the prompt rows probing; event-timed
+    with the inputs resident (Q, K, V of a 64-image batch are 1.06 GB, larger than L2)."""
+    import torch
+    from paper_2503_10501_b200 import binding as tcb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the probe")
+    torch.cuda.set_device(0)
+    tcb.lib()
+    pk = peaks()
+    B, H, dh, n_sys, N, n_text = args.batch or 64, 32, 128, 35, 576, 64
+    L = n_sys + N + n_text
+    g = torch.Generator(device="cuda").manual_seed(7)
+    Q, K, V = (torch.randn(B, H, L, dh, device="cuda", generator=g).half() for _ in range(3))
+    p = tcb.Params(batch=B, n_tokens=N, d_model=H * dh, n_heads=H, head_dim=dh, n_query=n_text, keep=128,
+                   dtype="f16")
+    n = __import__("ctypes").c_size_t(0)
+    cp = p.c()
+    tcb.lib().tc_probe_workspace_bytes(__import__("ctypes").byref(cp), n_sys, n_text, __import__("ctypes").byref(n))
+    ws = torch.empty(int(n.value), dtype=torch.uint8, device="cuda")
+    out = (torch.empty(B, N, H * dh, dtype=torch.float16, device="cuda"),
+           torch.empty(B, H, n_text, N, dtype=torch.float16, device="cuda"),
+           torch.empty(B, dtype=torch.int32, device="cuda"))
+
+    def step():
+        tcb.tc_probe(p, n_sys, n_text, n_sys + N, Q, K, V, ws=ws, out=out)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if int(out[2].abs().sum()):
+        raise SystemExit("probe reported a per-image status")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    # algorithmic flops: row i sees i + 1 keys; Q K^T and P V, 2 flops per multiply-add
+    vis = sum(i + 1 for i in range(n_sys, n_sys + N))
+    prb = sum(i + 1 for i in range(n_sys + N, L))
+    flops = B * H * (4.0 * vis * dh + 2.0 * 2 * prb * dh)
+    # issued: 128 x 128 key blocks up to the last row of each 128-row tile
+    tiles = sum(((min(N, (t + 1) * 128) + n_sys - 1) // 128 + 1) for t in range((N + 127) // 128))
+    issued = B * H * tiles * 2 * 2.0 * 128 * 128 * dh
+    byts = (3 * Q.numel() + out[0].numel() + out[1].numel()) * 2 + 2 * V.numel() * 2
+    print(json.dumps({
+        "entry": "tc_probe", "workload": f"B={B} H={H} dh={dh} n_sys={n_sys} N={N} n_text={n_text} f16",
+        "ms_per_call": round(ms, 4), "images_per_s": round(B / (ms * 1e-3), 1),
+        "roofline": {"bound": "tensor", "achieved": round(flops / (ms * 1e-3) / 1e12, 2),
+                     "achieved_issued": round(issued / (ms * 1e-3) / 1e12, 2),
+                     "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": round(flops / (ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"], 4),
+                     "peak_source": pk["source"] + " (sustained bf16)"},
+        "hbm_bytes_per_call": byts,
+        "hbm_frac": round(byts / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], 4)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -565,10 +626,14 @@ def main():
                     help="images the CPU oracle is timed on (0 = skip)")
     ap.add_argument("--sweep", action="store_true",
                     help="one line per point of the T x keep sweep instead of the bench line")
+    ap.add_argument("--probe", action="store_true",
+                    help="time the layer-2 probe (tc_probe) at the bench point's layout instead of the bench line")
     ap.add_argument("--extras", action="store_true",
                     help="time tc_rank and tc_reassemble at the bench point instead of the bench line")
     args = ap.parse_args()
-    if args.extras:
+    if args.probe:
+        run_probe(args)
+    elif args.extras:
         run_extras(args)
     elif args.sweep:
         run_sweep(args)

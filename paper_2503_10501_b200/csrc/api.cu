@@ -203,7 +203,7 @@ static tc_status open_ctx(const tc_params* p, void* ws, size_t ws_bytes, void* s
 // Gram -> eigen-solve chains run on separate internal streams, forked from and joined back into
 // the caller's stream with events: one group's single-block kernels overlap another group's
 // GEMMs.  Per-image results do not depend on the grouping.
-constexpr int kMaxGroups = 8;
+constexpr int kMaxGroups = 16;
 struct GroupStreams {
   bool ready = false;
   cudaStream_t s[kMaxGroups];    // a group's sketch -> Cholesky-QR -> eigen-solve chain

@@ -1538,7 +1538,11 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
                                                          float* __restrict__ u0g, float* __restrict__ u1g,
                                                          float* __restrict__ u2g, float* yg, float* __restrict__ mlg,
                                                          size_t ml_stride,
-                                                         int32_t* __restrict__ status, int nparts) {
+                                                         int32_t* __restrict__ status, int nparts,
+                                                         int emit_factors) {
+  // emit_factors: instead of Z = Q Y the kernel leaves its two factors for the tensor-core
+  // products: ZTg receives Q^T ([j][i] = Q[i][j]) and u0g receives Y^T ([p][j] = component j of
+  // the eigenvector p of T)
   const int n = NT ? NT : n_rt;
   extern __shared__ __align__(16) float sm[];
   const int ld = n | 1;
@@ -2153,6 +2157,26 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     }
     __syncthreads();
     for (int p = tid; p < n; p += 512) theta[(size_t)b * n + p] = fmaxf(e2[p], 0.f);
+    if (emit_factors) {
+      float* QT = ZTg + img;
+      for (int e = tid; e < n * n; e += 512) {
+        const int j = e / n, i = e - j * n;
+        QT[e] = A[i * ld + j];
+      }
+      __syncthreads();
+      for (int e = tid; e < n * n; e += 512) {   // Y through shared memory, to turn it over
+        const int j = e / n, p = e - j * n;
+        A[j * ld + p] = __ldcg(y + e);
+      }
+      __syncthreads();
+      float* YT = u0;  // the factorisations kept there are no longer needed
+      for (int e = tid; e < n * n; e += 512) {
+        const int p = e / n, j = e - p * n;
+        YT[e] = A[j * ld + p];
+      }
+      if (tid == 0 && s_fail) atomicMax(&status[b], (int)TC_ERR_NOT_CONVERGED);
+      return;
+    }
     // ---------------- Z = Q Y:  ZT[p][i] = sum_j Q[i][j] Y[j][p] ----------------
     // thread = (four eigenvectors p, twelve rows i): per j one 16-byte load of Y (coalesced over
     // p) and twelve broadcast reads of Q from shared memory feed 48 multiply-adds
@@ -2235,14 +2259,14 @@ constexpr size_t SMEM_LIMIT = 220 * 1024;  // leaves room for the static shared 
 static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int n, int batch,
                           int max_sweeps, float rank_tol, float* scr1, float* scr2, float* scr3,
                           float* scr4, size_t scr4_stride, int32_t* status, cudaStream_t st,
-                          int nparts = 1) {
+                          int nparts = 1, int emit_factors = 0) {
   Scope scope_(KC_JACOBI, st);
   {
     const size_t tri = ((size_t)n * (n | 1) + 27 * (size_t)((n + 3) & ~3)) * sizeof(float);
     if (n >= 3 && tri <= SMEM_LIMIT && scr1 != nullptr) {
       auto go = [&](auto kernel) {
         cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri);
-        { kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts); note_launch(); }
+        { kernel<<<batch, 512, tri, st>>>(H, ZT, theta, n, rank_tol, W, scr1, scr2, scr3, scr4, scr4_stride, status, nparts, emit_factors); note_launch(); }
       };
       switch (n) {
         case 128: go(tridiag_eig_kernel<128>); break;
@@ -2508,12 +2532,17 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
     mm(G, At, N, N, nullptr, Bt, KC_GEMM_GQ);
     mm(At, Bt, k, N, Hk, nullptr, KC_GEMM_TN);
     if (err != TC_OK) return err;
-    float* ZTk = Sk;  // the k x k matrices of the passes are free now
-    launch_jacobi(Hk, Es, ZTk, theta, k, B, D.max_sweeps, D.rank_tol, Es + (size_t)B * sK,
-                  Es + 2 * (size_t)B * sK, Rinv, Es + 3 * (size_t)B * sK, sK, stp, st, 1);
-    // 5. PT[p][x] = sum_i ZT[p][i] Q1[x][i]: the product Q1 ZT^T written transposed
-    float* PT = Br;
-    mm(Ar, ZTk, N, k, nullptr, PT, KC_GEMM);
+    // The solver leaves the eigenvectors of H as the two factors Z = Q Y (Q from the reduction
+    // to tridiagonal form, Y the eigenvectors of the tridiagonal matrix): Q^T in QTk, Y^T in YTk.
+    float* QTk = Sk;  // the k x k matrices of the passes are free now
+    float* YTk = Es;  // (the solver's first work array, handed back as Y^T)
+    launch_jacobi(Hk, Es, QTk, theta, k, B, D.max_sweeps, D.rank_tol, Es + (size_t)B * sK,
+                  Es + 2 * (size_t)B * sK, Rinv, Es + 3 * (size_t)B * sK, sK, stp, st, 1, 1);
+    // 5. eigenvectors of G in the subspace, U = Q1 Q Y, as two products:
+    //    W = Q1 Q, then PT[p][x] = sum_j Y[j][p] W[x][j] (W Y written transposed)
+    mm(Ar, QTk, N, k, Br, nullptr, KC_GEMM);
+    float* PT = Bt;
+    mm(Br, YTk, N, k, nullptr, PT, KC_GEMM);
     if (err != TC_OK) return err;
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
