@@ -2368,7 +2368,9 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
                                                  float* __restrict__ sigma_sorted,
                                                  int32_t* __restrict__ rank_out,
                                                  int32_t* __restrict__ status, int N, int k, int q,
-                                                 float rank_tol, int full) {
+                                                 float rank_tol, int full,
+                                                 const float* __restrict__ G) {
+  // G (subspace solve only): the Gram matrix, for the energy check below
   // grid (token chunks of 256, images): every block ranks the k singular values again (k^2
   // comparisons, cheap) and sums Eq. 3-6 for its own tokens; chunk 0 writes sigma and the rank.
   extern __shared__ float sig[];  // [k] sigma, then [k] weights (sigma or 0)
@@ -2414,6 +2416,23 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
     for (int w = 0; w < 8; ++w) r += s_cnt[w];
     if (rank_out) rank_out[b] = r;
     if (!full && r > k - 8) atomicMax(&status[b], (int)TC_ERR_RANK_CAP);
+  }
+  if (writer && !full && G != nullptr && warp == 0) {
+    // What the subspace did not capture: trace(G) - sum(theta) is the energy of O outside it.
+    // If the directions left out were all under the rank cut-off, that is at most
+    // (q - k) (rank_tol sigma_1)^2; more means a direction above the cut-off was missed (a
+    // rank above the hint that the count above could not see), and Eq. 3-6 would be truncated.
+    float tr = 0.f, st = 0.f;
+    const float* Gb = G + (size_t)b * N * N;
+    for (int x = lane; x < N; x += 32) tr += Gb[(size_t)x * N + x];
+    for (int p = lane; p < k; p += 32) st += sig[p] * sig[p];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      tr += __shfl_xor_sync(0xffffffffu, tr, o);
+      st += __shfl_xor_sync(0xffffffffu, st, o);
+    }
+    const float allow = (float)max(q - k, 0) * cut * cut + 1e-5f * tr;
+    if (lane == 0 && tr - st > allow) atomicMax(&status[b], (int)TC_ERR_RANK_CAP);
   }
   const float* PTb = PT + (size_t)b * k * N;
   const int x = blockIdx.x * 256 + tid;
@@ -2470,7 +2489,7 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
                   img_status, st);
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)N * sizeof(float), st>>>(
-          theta, ZT, C_out, sigma_out, rank_out, img_status, N, N, q, D.rank_tol, 1); note_launch(); }
+          theta, ZT, C_out, sigma_out, rank_out, img_status, N, N, q, D.rank_tol, 1, nullptr); note_launch(); }
     return TC_OK;
   }
   auto sketch_into = [&](float* Y0) {
@@ -2546,7 +2565,7 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
     if (err != TC_OK) return err;
     Scope scope_(KC_ICS, st);
     { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
-          theta, PT, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0); note_launch(); }
+          theta, PT, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0, G); note_launch(); }
     return TC_OK;
   }
   float* Y0 = (float*)(ws + P.Y0) + b0 * sY;
@@ -2585,7 +2604,7 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
   gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
   Scope scope_(KC_ICS, st);
   { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
-        theta, Y0, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0); note_launch(); }
+        theta, Y0, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0, G); note_launch(); }
   return TC_OK;
 }
 
