@@ -34,7 +34,7 @@ constexpr int UMMA_K = 16;
 constexpr uint32_t TILE_BYTES = TILE * BK * 2;  // 16 KB
 constexpr uint32_t SMEM_BYTES = STAGES * 2 * TILE_BYTES + 1024;  // + alignment slack
 constexpr uint32_t TMEM_COLS = 256;  // two 128-column accumulators
-constexpr int DRAIN_KB = 2;          // stages per accumulation chunk (128 elements of K)
+constexpr int DRAIN_KB = 4;          // stages per accumulation chunk (256 elements of K; 512 breaks the 2e-6 bound)
 
 // Instruction descriptor: D float32, A and B both float16 or both bfloat16 (operand format 0 / 1),
 // both K-major, M = 128, N = 128.

@@ -13,9 +13,11 @@
 //   - warp 5 (one lane): S = Q K^T into TMEM; later O_blk = P V into a second accumulator;
 //   - warps 0-3: thread = query row.  The scores of the row come back with tcgen05.ld, get the
 //     causal mask, and feed an online softmax in the exp2 domain; the probabilities are written as
-//     float16 / bfloat16 into the shared-memory tile the keys have just left (in the swizzled
-//     layout the tensor core expects), and the block's P V is folded into a float32 row of Z held
-//     in registers, rescaled when the running maximum moves.
+//     float16 / bfloat16 into a shared-memory tile of their own (in the swizzled layout the
+//     tensor core expects), and the block's P V is folded into a float32 row of Z held in
+//     registers, rescaled when the running maximum moves.
+// The scores have two accumulators and V^T two tiles: while the softmax warps work on block i the
+// tensor core already forms the scores of block i + 1, and the loads of block i + 1 are in flight.
 // The probe rows take two passes over the keys instead (first the row maxima and sums, then the
 // normalised probabilities of the visual columns) and need no V.
 // Every mbarrier wait is bounded; a wait that runs out records an error for the image and the
@@ -34,9 +36,10 @@ constexpr int KB = 128;          // keys per block
 constexpr int DH = 128;          // head dimension the kernel is built for
 constexpr uint32_t ATOM = 128 * 128;        // bytes of one 128-row x 64-element swizzle atom
 constexpr uint32_t TILE_B = 2 * ATOM;       // a 128 x 128 tile of 16-bit elements
-constexpr uint32_t SMEM_O = 3 * TILE_B + 1024;   // Q, K (later P), V^T
+constexpr uint32_t SMEM_O = 5 * TILE_B + 1024;   // Q, K, P, two tiles of V^T
 constexpr uint32_t SMEM_A = 2 * TILE_B + 1024;   // Q, K
-constexpr uint32_t TMEM_COLS = 256;              // S and the block's P V
+constexpr uint32_t TMEM_COLS_O = 512;            // two score accumulators and the block's P V
+constexpr uint32_t TMEM_COLS_A = 256;            // two score accumulators
 
 // D float32, A and B float16 (bf = 0) or bfloat16 (bf = 1), both K-major, M = N = 128
 __device__ __forceinline__ uint32_t idesc(int bf) {
@@ -110,7 +113,13 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
     const __grid_constant__ CUtensorMap mapVt, ProbeArgs pa, T* __restrict__ out,
     int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_q, bar_k, bar_v, bar_s, bar_p, bar_pv, bar_sfree;
+  // bar_k: key tile landed; bar_kfree: its scores are formed (the tile may be reloaded);
+  // bar_v[2]: V^T tile landed; bar_s[2]: scores ready in accumulator 0 / 1; bar_sfree[2]: the
+  // softmax warps are done with that accumulator; bar_p: P written; bar_pv: P V done (O_blk
+  // ready, P free); bar_vfree[2]: the same event per V^T tile (so that no waiter can fall two
+  // completions behind)
+  __shared__ __align__(8) uint64_t bar_q, bar_k, bar_kfree, bar_v[2], bar_vfree[2], bar_s[2], bar_sfree[2], bar_p, bar_pv;
+  constexpr uint32_t TMEM_COLS = WANT_O ? TMEM_COLS_O : TMEM_COLS_A;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
 
@@ -122,17 +131,22 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
   const int nkb = q_last / KB + 1;                        // causal: keys up to the last row's position
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t sQ = smem_base, sK = smem_base + TILE_B, sV = smem_base + 2 * TILE_B;
+  const uint32_t sQ = smem_base, sK = smem_base + TILE_B, sP = smem_base + 2 * TILE_B;
+  auto sV = [&](int i) { return smem_base + (uint32_t)(3 + (i & 1)) * TILE_B; };
   const uint32_t id = idesc(pa.bf);
 
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&bar_q), 1);
     mbar_init(smem_u32(&bar_k), 1);
-    mbar_init(smem_u32(&bar_v), 1);
-    mbar_init(smem_u32(&bar_s), 1);
+    mbar_init(smem_u32(&bar_kfree), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bar_v[i]), 1);
+      mbar_init(smem_u32(&bar_vfree[i]), 1);
+      mbar_init(smem_u32(&bar_s[i]), 1);
+      mbar_init(smem_u32(&bar_sfree[i]), 4);
+    }
     mbar_init(smem_u32(&bar_p), 4);
     mbar_init(smem_u32(&bar_pv), 1);
-    mbar_init(smem_u32(&bar_sfree), 4);
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -146,7 +160,8 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_s = s_tmem, tmem_o = s_tmem + 128u;
+  auto tmem_s = [&](int i) { return s_tmem + (uint32_t)(i & 1) * 128u; };
+  const uint32_t tmem_o = s_tmem + 256u;
 
   // key blocks in the order they are walked: all of them once (WANT_O), or all of them for the
   // row statistics and then those that hold visual columns once more
@@ -156,46 +171,50 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
   auto block_of = [&](int it) { return it < nkb ? it : vb0 + (it - nkb); };
 
   if (warp == 4) {
-    // ---- TMA producer ----
+    // ---- TMA producer: the key tile of block it + 1 as soon as the scores of block it are
+    //      formed, the V^T tile of block it + 1 as soon as P V of block it - 1 is done ----
     if (lane == 0) {
       mbar_expect_tx(smem_u32(&bar_q), TILE_B);
       tma_load_3d(sQ, &mapQ, 0, q0, bh, smem_u32(&bar_q));
       tma_load_3d(sQ + ATOM, &mapQ, 64, q0, bh, smem_u32(&bar_q));
-      for (int it = 0; it < n_iter; ++it) {
+      bool ok = true;
+      for (int it = 0; it < n_iter && ok; ++it) {
         const int kb = block_of(it);
-        if (it > 0) {
-          // the key tile is free once its scores have been read (and, with Z, once P V has run)
-          const bool okw = WANT_O ? mbar_wait(smem_u32(&bar_pv), (uint32_t)(it - 1) & 1u)
-                                  : mbar_wait(smem_u32(&bar_sfree), (uint32_t)(it - 1) & 1u);
-          if (!okw) {
-            s_fail = 1;
-            break;
-          }
-        }
+        if (it > 0 && !mbar_wait(smem_u32(&bar_kfree), (uint32_t)(it - 1) & 1u)) { ok = false; break; }
         mbar_expect_tx(smem_u32(&bar_k), TILE_B);
         tma_load_3d(sK, &mapK, 0, kb * KB, bh, smem_u32(&bar_k));
         tma_load_3d(sK + ATOM, &mapK, 64, kb * KB, bh, smem_u32(&bar_k));
         if (WANT_O) {
-          mbar_expect_tx(smem_u32(&bar_v), TILE_B);
-          tma_load_3d(sV, &mapVt, kb * KB, 0, bh, smem_u32(&bar_v));
-          tma_load_3d(sV + ATOM, &mapVt, kb * KB + 64, 0, bh, smem_u32(&bar_v));
+          if (it >= 2 && !mbar_wait(smem_u32(&bar_vfree[it & 1]), ((uint32_t)(it - 2) >> 1) & 1u)) { ok = false; break; }
+          mbar_expect_tx(smem_u32(&bar_v[it & 1]), TILE_B);
+          tma_load_3d(sV(it), &mapVt, kb * KB, 0, bh, smem_u32(&bar_v[it & 1]));
+          tma_load_3d(sV(it) + ATOM, &mapVt, kb * KB + 64, 0, bh, smem_u32(&bar_v[it & 1]));
         }
       }
+      if (!ok) s_fail = 1;
     }
   } else if (warp == 5) {
-    // ---- MMA issuer ----
+    // ---- MMA issuer: scores one block ahead of the softmax ----
     if (lane == 0) {
       bool ok = mbar_wait(smem_u32(&bar_q), 0);
-      for (int it = 0; it < n_iter && ok; ++it) {
-        const uint32_t ph = (uint32_t)it & 1u;
-        if (!mbar_wait(smem_u32(&bar_k), ph)) { ok = false; break; }
+      auto scores = [&](int it) {   // S[it & 1] = Q K(it)^T
+        if (!mbar_wait(smem_u32(&bar_k), (uint32_t)it & 1u)) return false;
+        if (it >= 2 && !mbar_wait(smem_u32(&bar_sfree[it & 1]), ((uint32_t)(it - 2) >> 1) & 1u)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        mma_tile(tmem_s, sQ, sK, id);                 // S = Q K^T
-        umma_commit(smem_u32(&bar_s));
-        if (WANT_O) {
-          if (!mbar_wait(smem_u32(&bar_p), ph) || !mbar_wait(smem_u32(&bar_v), ph)) { ok = false; break; }
+        mma_tile(tmem_s(it), sQ, sK, id);
+        umma_commit(smem_u32(&bar_kfree));
+        umma_commit(smem_u32(&bar_s[it & 1]));
+        return true;
+      };
+      if (ok) ok = scores(0);
+      for (int it = 0; it < n_iter && ok; ++it) {
+        if (it + 1 < n_iter) ok = scores(it + 1);
+        if (WANT_O && ok) {
+          if (!mbar_wait(smem_u32(&bar_p), (uint32_t)it & 1u) ||
+              !mbar_wait(smem_u32(&bar_v[it & 1]), ((uint32_t)it >> 1) & 1u)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          mma_tile(tmem_o, sK, sV, id);               // O_blk = P V  (P stands where the keys were)
+          mma_tile(tmem_o, sP, sV(it), id);             // O_blk = P V
+          umma_commit(smem_u32(&bar_vfree[it & 1]));
           umma_commit(smem_u32(&bar_pv));
         }
       }
@@ -218,7 +237,8 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
       const uint32_t ph = (uint32_t)it & 1u;
       const int kb = block_of(it);
       const bool second = it >= nkb;
-      if (!mbar_wait(smem_u32(&bar_s), ph)) { ok = false; break; }
+      const uint32_t ts = tmem_s(it);
+      if (!mbar_wait(smem_u32(&bar_s[it & 1]), ((uint32_t)it >> 1) & 1u)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int jmax = min(qpos, pa.L - 1) - kb * KB;   // columns 0 .. jmax of this block are visible
       float alpha = 1.f;
@@ -228,7 +248,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t r[32];
-          tmem_ld32_issue(tmem_s + lane_addr + (uint32_t)(c * 32), r);
+          tmem_ld32_issue(ts + lane_addr + (uint32_t)(c * 32), r);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; ++j)
@@ -245,7 +265,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t r[32];
-          tmem_ld32_issue(tmem_s + lane_addr + (uint32_t)(c * 32), r);
+          tmem_ld32_issue(ts + lane_addr + (uint32_t)(c * 32), r);
           tmem_wait_ld();
           float pr[32];
 #pragma unroll
@@ -256,7 +276,8 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
           }
           if (WANT_O) {
             // 32 columns = four 16-byte chunks of the row; chunk ch of atom a lies at
-            // a * ATOM + row * 128 + ((ch ^ (row & 7)) * 16)
+            // a * ATOM + row * 128 + ((ch ^ (row & 7)) * 16).  (P V of the block before, which
+            // read this tile, was waited for when its result was folded in.)
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               const int kk = c * 32 + q * 8;             // first key of the chunk
@@ -266,7 +287,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
               v.y = pack2<T>(pr[q * 8 + 2], pr[q * 8 + 3]);
               v.z = pack2<T>(pr[q * 8 + 4], pr[q * 8 + 5]);
               v.w = pack2<T>(pr[q * 8 + 6], pr[q * 8 + 7]);
-              *reinterpret_cast<uint4*>(smem_gen + TILE_B + atom * ATOM + (uint32_t)row * 128u +
+              *reinterpret_cast<uint4*>(smem_gen + 2 * TILE_B + atom * ATOM + (uint32_t)row * 128u +
                                         ((ch ^ ((uint32_t)row & 7u)) << 4)) = v;
             }
           }
@@ -278,7 +299,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t r[32];
-          tmem_ld32_issue(tmem_s + lane_addr + (uint32_t)(c * 32), r);
+          tmem_ld32_issue(ts + lane_addr + (uint32_t)(c * 32), r);
           tmem_wait_ld();
           if (live) {
             T* dst = out + (((size_t)bh * pa.n_rows + (qpos - pa.row0)) * pa.n_vis);
@@ -293,7 +314,11 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
           }
         }
       }
+      // this score accumulator may be overwritten
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_sfree[it & 1])) : "memory");
       if (WANT_O) {
         // hand P to the tensor core, then fold the block's P V into the row of Z
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -311,10 +336,6 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
           for (int j = 0; j < 32; ++j) o[c * 32 + j] = fmaf(o[c * 32 + j], alpha, __uint_as_float(r[j]));
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      } else {
-        __syncwarp();
-        if (lane == 0)
-          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_sfree)) : "memory");
       }
     }
     if (ok && s_fail == 0) {
@@ -340,7 +361,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 5) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_s),
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(s_tmem),
                  "r"(TMEM_COLS)
                  : "memory");
   }
