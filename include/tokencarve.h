@@ -210,17 +210,23 @@ tc_status tc_carve_host(const tc_params* p, const void* O, const void* A, const 
  *   n_tokens, n_heads, n_query and dtype of `p` matter, but `p` must be valid as a whole.
  *
  * The partial column sums go into a fixed array of TC_NOALLOC_SCRATCH_BYTES that is part of
- * the library image: every GPU that loads the library holds that much memory until the
- * process exits, whether or not this function is ever called.  The call needs
+ * the library image: a GPU holds that much memory from the moment the part of the library that
+ * contains the array is loaded onto it (with the CUDA runtime's lazy loading that is this
+ * function's first call on the device) until the process exits.  The call needs
  * B * chunks * N floats of it, where chunks = min(64, (H*T)/32, ceil(592/B)) (at least 1);
  * a larger request returns TC_ERR_SCRATCH_LIMIT and enqueues nothing.
  *
  * The first call on each device looks up the array's device address (a host-side runtime
- * query, done with that device current); make that first call outside any stream capture.
- * No call allocates or frees memory.  All calls on a device share the one array, which keeps
- * whatever the previous call left in it; each call overwrites the part it uses before reading
- * it, so nothing has to be cleared, but two calls that overlap on the GPU (different streams,
- * or different host threads without ordering) race on it.  Order them on one stream.
+ * query, done with that device current).  That query, and the loading of the code it may
+ * trigger, can allocate and synchronise inside the driver: make the first call at start-up,
+ * outside any stream capture and outside latency-critical code.  After it, no call of this
+ * function allocates or frees memory (it calls neither cudaMalloc nor cudaFree nor any library
+ * that does).  `stream` must belong to the device that is current at the call: the address is
+ * remembered per current device.  The remembered address is not valid across cudaDeviceReset.
+ * All calls on a device share the one array, which keeps whatever the previous call left in
+ * it; each call overwrites the part it uses before reading it, so nothing has to be cleared,
+ * but two calls that overlap on the GPU (different streams, or different host threads without
+ * ordering) race on it.  Order them on one stream.
  */
 #define TC_NOALLOC_SCRATCH_BYTES (4u << 20)
 tc_status tc_attn_score_noalloc(const tc_params* p, const void* A, float* S, void* stream);
@@ -329,14 +335,15 @@ tc_status tc_rope_tables(const int32_t* pos, int64_t n_rows, int32_t head_dim, f
                          float* cos_out, float* sin_out, void* stream);
 
 /*
- * Number of image groups tc_score / tc_carve run side by side (1..8, default 4; the paper has no
- * counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
+ * Number of image groups tc_score / tc_carve run side by side (1..16, default 4; the paper has
+ * no counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
  * chains are enqueued on internal streams forked from `stream` and joined back into it before
  * the call's remaining kernels, so that the one-block-per-image solver kernels of one group
- * overlap the GEMMs of another.  Results do not depend on the setting.  Process-wide.  Each
- * group costs the host a few dozen launches per call: more than four groups pay only when the
- * call is replayed from a CUDA graph (measured at B = 64: 1.86 ms with 4 groups and 2.80 ms with
- * 8 for plain calls, 1.82 ms with 8 under replay).
+ * overlap the products of another.  Results do not depend on the setting.  The setting is
+ * process-wide state (one value for all threads and devices), and calls that use groups are
+ * serialised on a lock while they enqueue.  Each group costs the host a few dozen launches per
+ * call: more than four groups pay only when the call is replayed from a CUDA graph, where eight
+ * is the measured optimum at B = 64 (twelve and sixteen are within 1 % of it).
  */
 tc_status tc_set_groups(int32_t groups);
 

@@ -7,12 +7,14 @@
 // Both products run on the 5th-generation tensor cores (tcgen05.mma kind::f16, M = N = 128,
 // float32 accumulators in TMEM, operands staged by TMA with the 128-byte swizzle).  One CTA owns
 // 128 query rows of one head of one image and walks the keys in blocks of 128:
-//   - warp 4 (one lane): TMA loads of the query tile (once), then per block the key tile and,
+//   - warp 8 (one lane): TMA loads of the query tile (once), then per block the key tile and,
 //     when Z is wanted, the tile of V^T (V is transposed into the workspace first, so that both
 //     operands of P V have their contraction index contiguous);
-//   - warp 5 (one lane): S = Q K^T into TMEM; later O_blk = P V into a second accumulator;
-//   - warps 0-3: thread = query row.  The scores of the row come back with tcgen05.ld, get the
-//     causal mask, and feed an online softmax in the exp2 domain; the probabilities are written as
+//   - warp 9 (one lane): S = Q K^T into TMEM; later O_blk = P V into a second accumulator;
+//   - warps 0-7: two threads per query row, each with half of the block's 128 columns (and half
+//     of the row of Z).  The scores come back with tcgen05.ld, get the causal mask, and feed an
+//     online softmax in the exp2 domain (the two halves of a row exchange their block maxima
+//     through shared memory); the probabilities are written as
 //     float16 / bfloat16 into a shared-memory tile of their own (in the swizzled layout the
 //     tensor core expects), and the block's P V is folded into a float32 row of Z held in
 //     registers, rescaled when the running maximum moves.
@@ -108,7 +110,7 @@ struct ProbeArgs {
 // WANT_O: visual query rows -> rows of Z (O_out [B][n_vis][H * dh]).
 // !WANT_O: probe rows -> probabilities of the visual columns (A_out [B][H][n_rows][n_vis]).
 template <typename T, bool WANT_O>
-__global__ void __launch_bounds__(192, 1) probe_kernel(
+__global__ void __launch_bounds__(320, 1) probe_kernel(
     const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
     const __grid_constant__ CUtensorMap mapVt, ProbeArgs pa, T* __restrict__ out,
     int32_t* __restrict__ status) {
@@ -122,6 +124,8 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
   constexpr uint32_t TMEM_COLS = WANT_O ? TMEM_COLS_O : TMEM_COLS_A;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
+  __shared__ float s_xm[2][2][QT];   // block maxima of the two column halves, double-buffered
+  __shared__ float s_xl[2][QT];      // row sums of the two halves
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -143,14 +147,14 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
       mbar_init(smem_u32(&bar_v[i]), 1);
       mbar_init(smem_u32(&bar_vfree[i]), 1);
       mbar_init(smem_u32(&bar_s[i]), 1);
-      mbar_init(smem_u32(&bar_sfree[i]), 4);
+      mbar_init(smem_u32(&bar_sfree[i]), 8);
     }
-    mbar_init(smem_u32(&bar_p), 4);
+    mbar_init(smem_u32(&bar_p), 8);
     mbar_init(smem_u32(&bar_pv), 1);
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 5) {
+  if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&s_tmem)),
                  "r"(TMEM_COLS)
@@ -170,7 +174,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
   const int n_iter = nkb + n_second;
   auto block_of = [&](int it) { return it < nkb ? it : vb0 + (it - nkb); };
 
-  if (warp == 4) {
+  if (warp == 8) {
     // ---- TMA producer: the key tile of block it + 1 as soon as the scores of block it are
     //      formed, the V^T tile of block it + 1 as soon as P V of block it - 1 is done ----
     if (lane == 0) {
@@ -193,7 +197,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
       }
       if (!ok) s_fail = 1;
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ---- MMA issuer: scores one block ahead of the softmax ----
     if (lane == 0) {
       bool ok = mbar_wait(smem_u32(&bar_q), 0);
@@ -221,51 +225,68 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
       if (!ok) s_fail = 1;
     }
   } else {
-    // ---- warps 0-3: softmax; thread = query row = TMEM lane ----
-    const int row = warp * 32 + lane;
+    // ---- warps 0-7: softmax.  Thread = (query row = TMEM lane, column half) ----
+    constexpr int HC = KB / 2;                      // columns of a block per thread
+    const int row = (warp & 3) * 32 + lane, half = warp >> 2;
     const int qpos = q0 + row;                       // sequence position of this row
     const bool live = qpos <= q_last;
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-    float m = -INFINITY, l = 0.f;
-    float o[WANT_O ? DH : 1];
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t col0 = (uint32_t)(half * HC);
+    float m = -INFINITY, l = 0.f;                    // l: this thread's half of the row sum
+    float o[WANT_O ? HC : 1];
     if (WANT_O) {
 #pragma unroll
-      for (int i = 0; i < DH; ++i) o[i] = 0.f;
+      for (int i = 0; i < HC; ++i) o[i] = 0.f;
     }
+    auto pair_sync = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };
     bool ok = true;
+    float inv_l = 0.f;
     for (int it = 0; it < n_iter; ++it) {
       const uint32_t ph = (uint32_t)it & 1u;
       const int kb = block_of(it);
       const bool second = it >= nkb;
-      const uint32_t ts = tmem_s(it);
-      if (!mbar_wait(smem_u32(&bar_s[it & 1]), ((uint32_t)it >> 1) & 1u)) { ok = false; break; }
+      const uint32_t ts = tmem_s(it) + lane_addr + col0;
+      if (!WANT_O && it == nkb) {
+        // between the two passes of the probe rows: the whole row sum
+        s_xl[half][row] = l;
+        pair_sync();
+        const float lt = s_xl[0][row] + s_xl[1][row];
+        inv_l = (lt > 0.f) ? 1.0f / lt : 0.f;
+      }
+      // A wait that runs out must not take this thread out of the loop: its partner would wait
+      // for it at the pair barrier for ever.  It goes on (on whatever the accumulators hold)
+      // without waiting again, and the image is reported at the end.
+      if (ok && !mbar_wait(smem_u32(&bar_s[it & 1]), ((uint32_t)it >> 1) & 1u)) ok = false;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int jmax = min(qpos, pa.L - 1) - kb * KB;   // columns 0 .. jmax of this block are visible
+      const int jmax = min(qpos, pa.L - 1) - kb * KB - (int)col0;   // own columns 0 .. jmax are visible
       float alpha = 1.f;
       if (!second) {
-        // pass over the block for its maximum
+        // pass over the block for its maximum: own half, then the partner's through shared memory
         float bm = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < HC / 32; ++c) {
           uint32_t r[32];
-          tmem_ld32_issue(ts + lane_addr + (uint32_t)(c * 32), r);
+          tmem_ld32_issue(ts + (uint32_t)(c * 32), r);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; ++j)
             if (c * 32 + j <= jmax) bm = fmaxf(bm, __uint_as_float(r[j]));
         }
+        s_xm[it & 1][half][row] = bm;
+        pair_sync();
+        bm = fmaxf(bm, s_xm[it & 1][half ^ 1][row]);
         const float m_new = fmaxf(m, bm * pa.scale2);
         alpha = (m_new == -INFINITY) ? 1.f : exp2f(m - m_new);
         m = m_new;
         l *= alpha;
       }
       if (WANT_O || !second) {
-        // probabilities of the block (unnormalised), their sum, and, with Z, the tile of P
+        // probabilities of the own columns (unnormalised), their sum, and, with Z, the tile of P
         float ls = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < HC / 32; ++c) {
           uint32_t r[32];
-          tmem_ld32_issue(ts + lane_addr + (uint32_t)(c * 32), r);
+          tmem_ld32_issue(ts + (uint32_t)(c * 32), r);
           tmem_wait_ld();
           float pr[32];
 #pragma unroll
@@ -275,19 +296,18 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
             ls += pr[j];
           }
           if (WANT_O) {
-            // 32 columns = four 16-byte chunks of the row; chunk ch of atom a lies at
-            // a * ATOM + row * 128 + ((ch ^ (row & 7)) * 16).  (P V of the block before, which
-            // read this tile, was waited for when its result was folded in.)
+            // The half's 64 columns are one swizzle atom of the P tile; chunk ch (8 columns) of
+            // the row lies at atom * ATOM + row * 128 + ((ch ^ (row & 7)) * 16).  (P V of the
+            // block before, which read this tile, was waited for when its result was folded in.)
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const int kk = c * 32 + q * 8;             // first key of the chunk
-              const uint32_t atom = (uint32_t)(kk >> 6), ch = (uint32_t)((kk & 63) >> 3);
+              const uint32_t ch = (uint32_t)(c * 4 + q);
               uint4 v;
               v.x = pack2<T>(pr[q * 8], pr[q * 8 + 1]);
               v.y = pack2<T>(pr[q * 8 + 2], pr[q * 8 + 3]);
               v.z = pack2<T>(pr[q * 8 + 4], pr[q * 8 + 5]);
               v.w = pack2<T>(pr[q * 8 + 6], pr[q * 8 + 7]);
-              *reinterpret_cast<uint4*>(smem_gen + 2 * TILE_B + atom * ATOM + (uint32_t)row * 128u +
+              *reinterpret_cast<uint4*>(smem_gen + 2 * TILE_B + (uint32_t)half * ATOM + (uint32_t)row * 128u +
                                         ((ch ^ ((uint32_t)row & 7u)) << 4)) = v;
             }
           }
@@ -295,17 +315,16 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
         l += ls;
       } else {
         // second pass of the probe rows: normalised probabilities of the visual columns
-        const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < HC / 32; ++c) {
           uint32_t r[32];
-          tmem_ld32_issue(ts + lane_addr + (uint32_t)(c * 32), r);
+          tmem_ld32_issue(ts + (uint32_t)(c * 32), r);
           tmem_wait_ld();
           if (live) {
             T* dst = out + (((size_t)bh * pa.n_rows + (qpos - pa.row0)) * pa.n_vis);
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const int key = kb * KB + c * 32 + j, x = key - pa.n_sys;
+              const int key = kb * KB + (int)col0 + c * 32 + j, x = key - pa.n_sys;
               if (x >= 0 && x < pa.n_vis) {
                 const float e = exp2f(fmaf(__uint_as_float(r[j]), pa.scale2, -m)) * inv_l;
                 dst[x] = (T)((c * 32 + j <= jmax) ? e : 0.f);
@@ -320,17 +339,17 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
       if (lane == 0)
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_sfree[it & 1])) : "memory");
       if (WANT_O) {
-        // hand P to the tensor core, then fold the block's P V into the row of Z
+        // hand P to the tensor core, then fold the block's P V into the own half of the row of Z
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0)
           asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_p)) : "memory");
-        if (!mbar_wait(smem_u32(&bar_pv), ph)) { ok = false; break; }
+        if (ok && !mbar_wait(smem_u32(&bar_pv), ph)) ok = false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < HC / 32; ++c) {
           uint32_t r[32];
-          tmem_ld32_issue(tmem_o + lane_addr + (uint32_t)(c * 32), r);
+          tmem_ld32_issue(tmem_o + lane_addr + col0 + (uint32_t)(c * 32), r);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; ++j) o[c * 32 + j] = fmaf(o[c * 32 + j], alpha, __uint_as_float(r[j]));
@@ -338,14 +357,22 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       }
     }
-    if (ok && s_fail == 0) {
+    if (WANT_O) {
+      // the whole row sum (every thread of the team comes here, whatever happened above)
+      s_xl[half][row] = l;
+      pair_sync();
+      const float lt = s_xl[0][row] + s_xl[1][row];
+      inv_l = (lt > 0.f) ? 1.0f / lt : 0.f;
+    }
+    if (!ok) s_fail = 1;
+    pair_sync();
+    if (s_fail == 0) {
       if (WANT_O && live) {
-        // row qpos - n_sys of O, columns h * dh ..
-        const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
+        // row qpos - n_sys of O, columns h * dh + 64 half ..
         uint4* dst = reinterpret_cast<uint4*>(
-            out + (((size_t)b * pa.n_vis + (qpos - pa.n_sys)) * pa.H + h) * DH);
+            out + (((size_t)b * pa.n_vis + (qpos - pa.n_sys)) * pa.H + h) * DH + half * HC);
 #pragma unroll
-        for (int q = 0; q < DH / 8; ++q) {
+        for (int q = 0; q < HC / 8; ++q) {
           uint4 v;
           v.x = pack2<T>(o[q * 8] * inv_l, o[q * 8 + 1] * inv_l);
           v.y = pack2<T>(o[q * 8 + 2] * inv_l, o[q * 8 + 3] * inv_l);
@@ -360,7 +387,7 @@ __global__ void __launch_bounds__(192, 1) probe_kernel(
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(s_tmem),
                  "r"(TMEM_COLS)
                  : "memory");
@@ -426,7 +453,7 @@ tc_status run_probe(int B, int H, int L, int n_sys, int n_vis, int probe_start, 
     note_launch();
     pa.row0 = n_sys; pa.n_rows = n_vis;
     dim3 grid((n_vis + QT - 1) / QT, H, B);
-    probe_kernel<T, true><<<grid, 192, SMEM_O, st>>>(mq, mk, mv, pa, (T*)O, status);
+    probe_kernel<T, true><<<grid, 320, SMEM_O, st>>>(mq, mk, mv, pa, (T*)O, status);
     note_launch();
   }
   if (A != nullptr && n_probe > 0) {
@@ -435,7 +462,7 @@ tc_status run_probe(int B, int H, int L, int n_sys, int n_vis, int probe_start, 
     if (cudaMemsetAsync(A, 0, (size_t)B * H * n_probe * n_vis * sizeof(T), st) != cudaSuccess) return TC_ERR_CUDA;
     pa.row0 = probe_start; pa.n_rows = n_probe;
     dim3 grid((n_probe + QT - 1) / QT, H, B);
-    probe_kernel<T, false><<<grid, 192, SMEM_A, st>>>(mq, mk, mv, pa, (T*)A, status);
+    probe_kernel<T, false><<<grid, 320, SMEM_A, st>>>(mq, mk, mv, pa, (T*)A, status);
     note_launch();
   }
   return TC_OK;
