@@ -246,8 +246,8 @@ def run_ours(args):
 
     # The timed step replays a CUDA graph of one tc_carve call (same kernels, same streams: the
     # fork/join of the library's internal streams is captured as graph dependencies), which
-    # takes the ~25 dependent launches of a group's chain off the host: 1.82 ms against 1.86 ms
-    # per step for plain calls (--no-graph).
+    # takes the ~25 dependent launches of a group's chain off the host (a few per cent of the
+    # step against plain calls, --no-graph).
     eager_step = step
     graph = None
     if use_graph:
@@ -303,9 +303,11 @@ def run_ours(args):
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of
     # this kernel at B=16, scaled by the batch: the traffic of these kernels grows in proportion);
     # null for a kernel that changed after its counters were taken
-    ncu_dram_per_image = {"gram": (75.57e6 + 3.8e6) / 16, "attn_colsum": (75.52e6 + 1.7e6) / 16,
-                          "compact": (75.58e6 + 17.7e6) / 16}
-    same_shape = (cfg.n_tokens, cfg.d_model, cfg.n_query, cfg.keep, k) == (576, 4096, 128, 128, 144)
+    ncu_dram_per_image = {"gram": (75.58e6 + 3.49e6) / 16, "attn_colsum": (75.52e6 + 1.38e6) / 16,
+                          "compact": (75.56e6 + 18.61e6) / 16, "eig": 1.396e6 / 16,
+                          "sketch": (75.51e6 + 1.85e6) / 16}
+    same_shape = (cfg.n_tokens, cfg.d_model, cfg.n_query, cfg.keep, k, cfg.dtype) == \
+        (576, 4096, 128, 128, 144, "f16")
     roof["traffic"] = (ncu_dram_per_image[top_name] * cfg.batch
                        if same_shape and top_name in ncu_dram_per_image else None)
     # the whole path against the slower of its HBM bytes and its Gram flops
