@@ -1807,7 +1807,6 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
     float* Vb = qf;              // [NBQ][n]  Vb[i][r] = entry r of reflector j0+i (0 above its support)
     float* Wp = qf + NBQ * n;    // [3][NBQ][n] partial products V^T Q per row range
     __shared__ float s_vv[NBQ][NBQ];  // v_a . v_b for a < b
-    __shared__ float s_T[NBQ][NBQ];
     for (int j1 = n - 3; j1 >= 0; j1 -= NBQ) {
       const int j0 = max(0, j1 - NBQ + 1), nbk = j1 - j0 + 1;
       // (1) copy the block's reflectors out of the columns that are about to be overwritten
@@ -1838,18 +1837,6 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         }
       }
       bar_named(1, QT);
-      if (qt == 0) {
-        // T_ii = beta_i ;  T[0:i, i] = -beta_i T[0:i, 0:i] (V[:, 0:i]^T v_i)
-        for (int i = 0; i < nbk; ++i) {
-          const float bi = beta[j0 + i];
-          for (int a2 = 0; a2 < i; ++a2) {
-            float acc = 0.f;
-            for (int l = a2; l < i; ++l) acc = fmaf(s_T[a2][l], s_vv[l][i], acc);
-            s_T[a2][i] = -bi * acc;
-          }
-          s_T[i][i] = bi;
-        }
-      }
       // (3) W = V^T Q on the columns c >= j0+1, rows split into up to three ranges
       const int ncols = n - j0 - 1;
       const int cw = (ncols + 31) >> 5;
@@ -1878,14 +1865,25 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
           for (int q = 0; q < G; ++q) t += Wp[(q * NBQ + i) * n + c];
           w[i] = (i < nbk) ? t : 0.f;
         }
-#pragma unroll
-        for (int i = 0; i < NBQ; ++i) {
-          float t = 0.f;
-#pragma unroll
-          for (int l = 0; l < NBQ; ++l)
-            if (l >= i && l < nbk && i < nbk) t = fmaf(s_T[i][l], w[l], t);
-          tw[i] = t;
-        }
+        // T (upper triangular, 4 x 4) of the compact WY form, in registers of every thread:
+        //   T_ii = beta_i ;  T[0:i, i] = -beta_i T[0:i, 0:i] (V[:, 0:i]^T v_i)
+        // (a reflector the block does not have gets beta = 0, which zeroes its row and column)
+        const float b0 = beta[j0], b1 = (nbk > 1) ? beta[j0 + 1] : 0.f;
+        const float b2 = (nbk > 2) ? beta[j0 + 2] : 0.f, b3 = (nbk > 3) ? beta[j0 + 3] : 0.f;
+        const float v01 = (nbk > 1) ? s_vv[0][1] : 0.f;
+        const float v02 = (nbk > 2) ? s_vv[0][2] : 0.f, v12 = (nbk > 2) ? s_vv[1][2] : 0.f;
+        const float v03 = (nbk > 3) ? s_vv[0][3] : 0.f, v13 = (nbk > 3) ? s_vv[1][3] : 0.f;
+        const float v23 = (nbk > 3) ? s_vv[2][3] : 0.f;
+        const float t01 = -b1 * (b0 * v01);
+        const float t02 = -b2 * fmaf(t01, v12, b0 * v02);
+        const float t12 = -b2 * (b1 * v12);
+        const float t03 = -b3 * fmaf(t02, v23, fmaf(t01, v13, b0 * v03));
+        const float t13 = -b3 * fmaf(t12, v23, b1 * v13);
+        const float t23 = -b3 * (b2 * v23);
+        tw[0] = fmaf(t03, w[3], fmaf(t02, w[2], fmaf(t01, w[1], b0 * w[0])));
+        tw[1] = fmaf(t13, w[3], fmaf(t12, w[2], b1 * w[1]));
+        tw[2] = fmaf(t23, w[3], b2 * w[2]);
+        tw[3] = b3 * w[3];
         for (int r = r_lo; r < r_hi; ++r) {
           float qv = A[r * ld + c];
 #pragma unroll
@@ -2013,9 +2011,13 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
       // eigenvalue number tid (0 = smallest): plain bisection, one thread per eigenvalue (the
       // counts are bound by instruction issue, so evaluating several points per round on
       // neighbouring lanes costs more than the rounds it saves)
+      // An interval that lies wholly under the floor below which no eigenvector is computed
+      // stops at a thousandth of that floor: such an eigenvalue only enters the energy check.
+      const float floor_n = 0.25f * rank_tol * rank_tol;
       for (int it = 0; it < 48; ++it) {
         const float x = 0.5f * (a + bhi);
         if (!(x > a) || !(x < bhi)) break;
+        if (bhi < floor_n && bhi - a < 1e-3f * floor_n) break;
         if (sturm(x) > tid) bhi = x; else a = x;
       }
       lam[tid] = 0.5f * (a + bhi) * tn;
