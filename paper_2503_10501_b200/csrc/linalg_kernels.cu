@@ -1804,15 +1804,16 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
   // reflectors; everything else of Q is still the identity, which the block first writes out.
   {
     constexpr int NBQ = 4;
-    float* Vb = qf;              // [NBQ][n]  Vb[i][r] = entry r of reflector j0+i (0 above its support)
+    float* Vb = qf;              // [n][NBQ]  Vb[r][i] = entry r of reflector j0+i (0 above its support
+                                 // and for a reflector the block does not have): one 16-byte read per row
     float* Wp = qf + NBQ * n;    // [3][NBQ][n] partial products V^T Q per row range
     __shared__ float s_vv[NBQ][NBQ];  // v_a . v_b for a < b
     for (int j1 = n - 3; j1 >= 0; j1 -= NBQ) {
       const int j0 = max(0, j1 - NBQ + 1), nbk = j1 - j0 + 1;
       // (1) copy the block's reflectors out of the columns that are about to be overwritten
-      for (int idx = qt; idx < nbk * n; idx += QT) {
-        const int i = idx / n, r = idx - i * n, jj = j0 + i;
-        Vb[i * n + r] = (r >= jj + 1) ? A[r * ld + jj] : 0.f;
+      for (int idx = qt; idx < NBQ * n; idx += QT) {
+        const int r = idx / NBQ, i = idx - r * NBQ, jj = j0 + i;
+        Vb[idx] = (i < nbk && r >= jj + 1) ? A[r * ld + jj] : 0.f;
       }
       bar_named(1, QT);
       // (2) identity columns j0+1 .. j1+1, zero rows j0+1 .. j1+1 right of them; v_a . v_b
@@ -1830,7 +1831,7 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         const int b2 = (qw < 3) ? qw + 1 : (qw < 5 ? qw - 1 : 3);
         if (b2 < nbk) {
           float d2 = 0.f;
-          for (int r = lane; r < n; r += 32) d2 = fmaf(Vb[a2 * n + r], Vb[b2 * n + r], d2);
+          for (int r = lane; r < n; r += 32) d2 = fmaf(Vb[r * NBQ + a2], Vb[r * NBQ + b2], d2);
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) d2 += __shfl_xor_sync(0xffffffffu, d2, o);
           if (lane == 0) s_vv[a2][b2] = d2;
@@ -1849,8 +1850,11 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         float acc[NBQ] = {0.f, 0.f, 0.f, 0.f};
         for (int r = r_lo; r < r_hi; ++r) {
           const float qv = A[r * ld + c];
-#pragma unroll
-          for (int i = 0; i < NBQ; ++i) acc[i] = fmaf(Vb[i * n + r], qv, acc[i]);
+          const float4 v4 = *reinterpret_cast<const float4*>(Vb + r * NBQ);
+          acc[0] = fmaf(v4.x, qv, acc[0]);
+          acc[1] = fmaf(v4.y, qv, acc[1]);
+          acc[2] = fmaf(v4.z, qv, acc[2]);
+          acc[3] = fmaf(v4.w, qv, acc[3]);
         }
 #pragma unroll
         for (int i = 0; i < NBQ; ++i) Wp[(g * NBQ + i) * n + c] = acc[i];
@@ -1884,10 +1888,29 @@ __global__ void __launch_bounds__(512) tridiag_eig_kernel(const float* Hin,
         tw[1] = fmaf(t13, w[3], fmaf(t12, w[2], b1 * w[1]));
         tw[2] = fmaf(t23, w[3], b2 * w[2]);
         tw[3] = b3 * w[3];
-        for (int r = r_lo; r < r_hi; ++r) {
+        int r = r_lo;
+        for (; r + 3 < r_hi; r += 4) {  // all loads of a trip before its stores
+          float qv[4];
+          float4 vb[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            qv[u] = A[(r + u) * ld + c];
+            vb[u] = *reinterpret_cast<const float4*>(Vb + (r + u) * NBQ);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            qv[u] = fmaf(-vb[u].x, tw[0], qv[u]);
+            qv[u] = fmaf(-vb[u].y, tw[1], qv[u]);
+            qv[u] = fmaf(-vb[u].z, tw[2], qv[u]);
+            qv[u] = fmaf(-vb[u].w, tw[3], qv[u]);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) A[(r + u) * ld + c] = qv[u];
+        }
+        for (; r < r_hi; ++r) {
           float qv = A[r * ld + c];
 #pragma unroll
-          for (int i = 0; i < NBQ; ++i) qv = fmaf(-Vb[i * n + r], tw[i], qv);
+          for (int i = 0; i < NBQ; ++i) qv = fmaf(-Vb[r * NBQ + i], tw[i], qv);
           A[r * ld + c] = qv;
         }
       }
