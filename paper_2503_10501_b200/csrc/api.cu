@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <functional>
 #include <mutex>
 #include <vector>
 
@@ -209,6 +210,7 @@ struct GroupStreams {
   cudaStream_t s[kMaxGroups];    // a group's sketch -> Cholesky-QR -> eigen-solve chain
   cudaStream_t s2[kMaxGroups];   // its Gram matrix, which the chain needs only from G Q on
   cudaEvent_t fork, join[kMaxGroups], gram_done[kMaxGroups];
+  cudaEvent_t attn_done;         // the attention partial sums of the whole batch are written
 };
 static std::mutex g_groups_mu;
 static GroupStreams g_groups[64];
@@ -226,6 +228,7 @@ static GroupStreams* group_streams() {
       if (cudaEventCreateWithFlags(&g.gram_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     }
     if (cudaEventCreateWithFlags(&g.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&g.attn_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     g.ready = true;
   }
   return &g;
@@ -235,8 +238,12 @@ static GroupStreams* group_streams() {
 // A launcher that refuses (tensor map, function attribute) stops the enqueue: the group streams
 // forked so far are joined back, the status words of the images not reached are set, and the
 // caller gets the status.
+// tail: what follows the scores of an image group on that group's stream (images b0 .. b0 + Dg.B),
+// so that one group's selection and gather run beside another group's eigen-solve; null for none.
+using GroupTail = std::function<void(const Dims& Dg, int b0, cudaStream_t st)>;
 static tc_status enqueue_score(const Ctx& c, const void* O, const void* A, float* E, float* C, float* S,
-                               float* sigma, int32_t* rank, int32_t* img_status) {
+                               float* sigma, int32_t* rank, int32_t* img_status,
+                               const GroupTail* tail = nullptr) {
   const Dims& D = c.D;
   const int q = D.N < D.d ? D.N : D.d;
   fill_i32(img_status, D.B, 0, c.st);
@@ -247,6 +254,8 @@ static tc_status enqueue_score(const Ctx& c, const void* O, const void* A, float
   if (gs == nullptr) ng = 1;
   if (ng > 1) cudaEventRecord(gs->fork, c.st);
   launch_attn_colsum(D, A, (float*)(c.ws + c.P.s_part), c.st);
+  const bool group_tail = (tail != nullptr) && ng > 1;
+  if (group_tail) cudaEventRecord(gs->attn_done, c.st);
   const int base = D.B / ng, extra = D.B % ng;
   int b0 = 0;
   tc_status err = TC_OK;
@@ -274,6 +283,12 @@ static tc_status enqueue_score(const Ctx& c, const void* O, const void* A, float
                        rank ? rank + b0 : nullptr, img_status + b0, st, nullptr, gram_done);
     else if (gram_done)
       cudaStreamWaitEvent(st, gram_done, 0);  // the side stream still joins the group's stream
+    if (group_tail && err == TC_OK) {
+      cudaStreamWaitEvent(st, gs->attn_done, 0);
+      const size_t o = (size_t)b0 * D.N;
+      launch_combine(Dg, (const float*)(c.ws + c.P.s_part) + o * D.chunks, C + o, S + o, E + o, st);
+      (*tail)(Dg, b0, st);
+    }
     if (ng > 1) {
       cudaEventRecord(gs->join[g], st);
       cudaStreamWaitEvent(c.st, gs->join[g], 0);
@@ -282,7 +297,10 @@ static tc_status enqueue_score(const Ctx& c, const void* O, const void* A, float
     b0 += nb;
   }
   if (err != TC_OK) return err;
-  launch_combine(D, (const float*)(c.ws + c.P.s_part), C, S, E, c.st);
+  if (!group_tail) {
+    launch_combine(D, (const float*)(c.ws + c.P.s_part), C, S, E, c.st);
+    if (tail) (*tail)(D, 0, c.st);
+  }
   return TC_OK;
 }
 
@@ -434,22 +452,40 @@ tc_status tc_carve(const tc_params* p, const void* O, const void* A, const void*
   int32_t* bd = (int32_t*)(c.ws + c.P.best_dst);
   int32_t* msrc = (int32_t*)(c.ws + c.P.msrc);
   int32_t* mdst = (int32_t*)(c.ws + c.P.mdst);
-  s = enqueue_score(c, O, A, E, C, S, nullptr, nullptr, img_status);
-  if (s != TC_OK) return s;
-  launch_prune(D, E, setA, setB, c.st);
-  if (D.M > 0) {
-    if (D.sim_src == 0) {
-      launch_match_gram(D, (const float*)(c.ws + c.P.G), setA, setB, bv, bd, img_status, c.st);
-    } else if (D.sim_src == 1) {
-      launch_match_rows(D, X, setA, setB, bv, bd, img_status, c.st);
-    } else {
-      float* Km = (float*)(c.ws + c.P.Kmean);
-      launch_mean_heads(D, K, Km, c.st);
-      launch_match_rows_f32(D, Km, D.dh, setA, setB, bv, bd, img_status, c.st);
+  // selection and gather of images b0 .. b0 + Dg.B on the stream their scores were computed on
+  const GroupTail tail = [&](const Dims& Dg, int b0, cudaStream_t st) {
+    const size_t b = (size_t)b0, esz = D.esz;
+    const size_t kv_in = (size_t)D.H * D.N * D.dh * esz, kv_out = (size_t)D.H * D.keep * D.dh * esz;
+    int32_t* sA = setA + b * D.nA;
+    int32_t* sB = setB + b * D.nB;
+    float* gbv = bv + b * D.nB;
+    int32_t* gbd = bd + b * D.nB;
+    int32_t* gst = img_status + b0;
+    const char* Xg = (const char*)X + b * D.N * D.d * esz;
+    const char* Kg = kv ? (const char*)K + b * kv_in : nullptr;
+    const char* Vg = kv ? (const char*)V + b * kv_in : nullptr;
+    launch_prune(Dg, E + b * D.N, sA, sB, st);
+    if (D.M > 0) {
+      if (D.sim_src == 0) {
+        launch_match_gram(Dg, (const float*)(c.ws + c.P.G) + b * D.N * D.N, sA, sB, gbv, gbd, gst, st);
+      } else if (D.sim_src == 1) {
+        launch_match_rows(Dg, Xg, sA, sB, gbv, gbd, gst, st);
+      } else {
+        float* Km = (float*)(c.ws + c.P.Kmean) + b * D.N * D.dh;
+        launch_mean_heads(Dg, Kg, Km, st);
+        launch_match_rows_f32(Dg, Km, D.dh, sA, sB, gbv, gbd, gst, st);
+      }
     }
-  }
-  launch_merge_select(D, setA, setB, bv, bd, msrc, mdst, kept_idx, img_status, c.st);
-  launch_compact(D, X, K, V, kept_idx, msrc, mdst, Xo, Ko, Vo, D.wmerge ? E : nullptr, img_status, c.st);
+    int32_t* gms = msrc + b * D.M;
+    int32_t* gmd = mdst + b * D.M;
+    int32_t* gk = kept_idx + b * D.keep;
+    launch_merge_select(Dg, sA, sB, gbv, gbd, gms, gmd, gk, gst, st);
+    launch_compact(Dg, Xg, Kg, Vg, gk, gms, gmd, (char*)Xo + b * D.keep * D.d * esz,
+                   kv ? (char*)Ko + b * kv_out : nullptr, kv ? (char*)Vo + b * kv_out : nullptr,
+                   D.wmerge ? E + b * D.N : nullptr, gst, st);
+  };
+  s = enqueue_score(c, O, A, E, C, S, nullptr, nullptr, img_status, &tail);
+  if (s != TC_OK) return s;
   return check_launch();
 }
 
