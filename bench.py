@@ -190,8 +190,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     tcb.lib()
     use_graph = not args.no_graph
-    # concurrent image groups: measured best is 8 under graph replay, the library's 4 otherwise
-    groups = args.groups if args.groups else (8 if use_graph else 4)
+    # concurrent image groups: measured best is 16 under graph replay, the library's 4 otherwise
+    groups = args.groups if args.groups else (16 if use_graph else 4)
     tcb.tc_set_groups(groups)
 
     cfg, name = workload(args)

@@ -336,14 +336,17 @@ tc_status tc_rope_tables(const int32_t* pos, int64_t n_rows, int32_t head_dim, f
 
 /*
  * Number of image groups tc_score / tc_carve run side by side (1..16, default 4; the paper has
- * no counterpart).  The batch is cut into that many contiguous groups whose Gram -> eigen-solve
- * chains are enqueued on internal streams forked from `stream` and joined back into it before
- * the call's remaining kernels, so that the one-block-per-image solver kernels of one group
- * overlap the products of another.  Results do not depend on the setting.  The setting is
- * process-wide state (one value for all threads and devices), and calls that use groups are
- * serialised on a lock while they enqueue.  Each group costs the host a few dozen launches per
- * call: more than four groups pay only when the call is replayed from a CUDA graph, where eight
- * is the measured optimum at B = 64 (twelve and sixteen are within 1 % of it).
+ * no counterpart).  The batch is cut into that many contiguous groups whose chains (Gram ->
+ * eigen-solve -> scores, and in tc_carve the selection and gather as well) are enqueued on
+ * internal streams forked from `stream` and joined back into it, so that the
+ * one-block-per-image solver kernels of one group overlap the products of another.  With four
+ * or more groups they start in waves (two; four from eight groups on), a wave's Gram products
+ * behind the previous wave's, so that the groups are not all in the same phase of the chain.
+ * Results do not depend on the setting.  The setting is process-wide state (one value for all
+ * threads and devices), and calls that use groups are serialised on a lock while they enqueue.
+ * Each group costs the host a few dozen launches per call: more than four groups pay only when
+ * the call is replayed from a CUDA graph, where sixteen is the measured optimum at B = 64
+ * (1.29 ms per carve against 1.31 ms with eight and 1.35 ms with eight in one wave).
  */
 tc_status tc_set_groups(int32_t groups);
 
