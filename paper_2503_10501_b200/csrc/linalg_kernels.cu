@@ -2396,12 +2396,14 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
                                                  float rank_tol, int full,
                                                  const float* __restrict__ G) {
   // G (subspace solve only): the Gram matrix, for the energy check below
-  // grid (token chunks of 256, images): every block ranks the k singular values again (k^2
-  // comparisons, cheap) and sums Eq. 3-6 for its own tokens; chunk 0 writes sigma and the rank.
+  // grid (token chunks of 64, images): every block ranks the k singular values again (k^2
+  // comparisons, cheap) and sums Eq. 3-6 for its own tokens, four threads to a token (each a
+  // quarter of the range of p, its loads in flight together); chunk 0 writes sigma and the rank.
   extern __shared__ float sig[];  // [k] sigma, then [k] weights (sigma or 0)
   float* wgt = sig + k;
   __shared__ float s_red[8];
   __shared__ int s_cnt[8];
+  __shared__ float s_part[4][64];
   const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool writer = blockIdx.x == 0;
   float mx = 0.f;
@@ -2449,7 +2451,16 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
     // rank above the hint that the count above could not see), and Eq. 3-6 would be truncated.
     float tr = 0.f, st = 0.f;
     const float* Gb = G + (size_t)b * N * N;
-    for (int x = lane; x < N; x += 32) tr += Gb[(size_t)x * N + x];
+    for (int x0 = 0; x0 < N; x0 += 256) {  // eight loads in flight
+      float dgl[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int x = x0 + u * 32 + lane;
+        dgl[u] = (x < N) ? Gb[(size_t)x * N + x] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) tr += dgl[u];
+    }
     for (int p = lane; p < k; p += 32) st += sig[p] * sig[p];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -2460,21 +2471,27 @@ __global__ void __launch_bounds__(256) ics_kernel(const float* __restrict__ thet
     if (lane == 0 && tr - st > allow) atomicMax(&status[b], (int)TC_ERR_RANK_CAP);
   }
   const float* PTb = PT + (size_t)b * k * N;
-  const int x = blockIdx.x * 256 + tid;
+  const int xl = tid & 63, part = tid >> 6;
+  const int x = blockIdx.x * 64 + xl;
+  const int per = (k + 3) >> 2;
+  const int p_lo = part * per, p_hi = min(k, p_lo + per);
+  float acc = 0.f;
   if (x < N) {
-    // terms in the order p = 0, 1, ...; eight loads in flight
-    float acc = 0.f;
-    int p = 0;
-    for (; p + 7 < k; p += 8) {
-      float v[8];
+    // terms of a quarter in the order p = p_lo, p_lo + 1, ...; twelve loads in flight
+    int p = p_lo;
+    for (; p + 11 < p_hi; p += 12) {
+      float v[12];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = PTb[(size_t)(p + u) * N + x];
+      for (int u = 0; u < 12; ++u) v[u] = PTb[(size_t)(p + u) * N + x];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) acc = fmaf(fabsf(v[u]), wgt[p + u], acc);
+      for (int u = 0; u < 12; ++u) acc = fmaf(fabsf(v[u]), wgt[p + u], acc);
     }
-    for (; p < k; ++p) acc = fmaf(fabsf(PTb[(size_t)p * N + x]), wgt[p], acc);
-    C[(size_t)b * N + x] = acc;
+    for (; p < p_hi; ++p) acc = fmaf(fabsf(PTb[(size_t)p * N + x]), wgt[p], acc);
   }
+  s_part[part][xl] = acc;
+  __syncthreads();
+  if (part == 0 && x < N)
+    C[(size_t)b * N + x] = (s_part[0][xl] + s_part[1][xl]) + (s_part[2][xl] + s_part[3][xl]);
 }
 
 __global__ void fill_i32_kernel(int32_t* p, int n, int v) {
@@ -2513,7 +2530,7 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
                   fs ? fs + 2 * (size_t)B * sG : nullptr, fs ? fs + 3 * (size_t)B * sG : nullptr, sG,
                   img_status, st);
     Scope scope_(KC_ICS, st);
-    { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)N * sizeof(float), st>>>(
+    { ics_kernel<<<dim3((N + 63) / 64, B), 256, 2 * (size_t)N * sizeof(float), st>>>(
           theta, ZT, C_out, sigma_out, rank_out, img_status, N, N, q, D.rank_tol, 1, nullptr); note_launch(); }
     return TC_OK;
   }
@@ -2589,7 +2606,7 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
     mm(Br, YTk, N, k, nullptr, PT, KC_GEMM);
     if (err != TC_OK) return err;
     Scope scope_(KC_ICS, st);
-    { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
+    { ics_kernel<<<dim3((N + 63) / 64, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
           theta, PT, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0, G); note_launch(); }
     return TC_OK;
   }
@@ -2628,7 +2645,7 @@ tc_status launch_ics(const Dims& D, const Plan& P, char* ws, int b0, const void*
   // 5. eigenvectors of G restricted to the subspace:  PT[p][x] = sum_i ZT[p][i] Q1[x][i]
   gemm<float, float, false, true>(ZT, Y2, Y0, k, N, k, k, k, N, sK, sY, sY, B, st);
   Scope scope_(KC_ICS, st);
-  { ics_kernel<<<dim3((N + 255) / 256, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
+  { ics_kernel<<<dim3((N + 63) / 64, B), 256, 2 * (size_t)k * sizeof(float), st>>>(
         theta, Y0, C_out, sigma_out, rank_out, img_status, N, k, q, D.rank_tol, 0, G); note_launch(); }
   return TC_OK;
 }
