@@ -267,7 +267,8 @@ static tc_status enqueue_score(const Ctx& c, const void* O, const void* A, float
     // before it: groups that all sit in the same phase of the chain compete for the same unit
     // (the tensor pipes in the products, 64 of 148 SMs in the single-block kernels) while the
     // others idle.  Measured at 64 images: 1.35 ms per carve in one wave, 1.29 ms in four.
-    const int waves = ng >= 8 ? 4 : (ng >= 4 ? 2 : 1);
+    // (Under 32 images the kernels of different groups hardly compete and a wave only waits.)
+    const int waves = D.B < 32 ? 1 : (ng >= 8 ? 4 : (ng >= 4 ? 2 : 1));
     const int per_wave = (ng + waves - 1) / waves;
     const bool late = (waves > 1) && (g >= per_wave) && !D.full;
     if (late) cudaStreamWaitEvent(st, gs->gram_done[g - per_wave], 0);
