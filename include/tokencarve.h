@@ -340,8 +340,9 @@ tc_status tc_rope_tables(const int32_t* pos, int64_t n_rows, int32_t head_dim, f
  * eigen-solve -> scores, and in tc_carve the selection and gather as well) are enqueued on
  * internal streams forked from `stream` and joined back into it, so that the
  * one-block-per-image solver kernels of one group overlap the products of another.  With four
- * or more groups and 32 or more images they start in waves (two; four from eight groups on), a wave's Gram products
- * behind the previous wave's, so that the groups are not all in the same phase of the chain.
+ * or more groups and 32 or more images they start in waves (two; four from eight groups on), a
+ * wave's Gram products behind the previous wave's, so that the groups are not all in the same
+ * phase of the chain.
  * Results do not depend on the setting.  The setting is process-wide state (one value for all
  * threads and devices), and calls that use groups are serialised on a lock while they enqueue.
  * Each group costs the host a few dozen launches per call: more than four groups pay only when
