@@ -513,6 +513,37 @@ def test_image_groups_and_graph_replay_do_not_change_results():
     assert not outs[0][4].any()
 
 
+def test_start_waves_and_group_tails_do_not_change_results():
+    # 32 images or more with eight or more groups: the groups start in four waves and every
+    # group runs its own selection and gather; ragged group sizes (34 = 3,3,2,2,...)
+    cfg = inputs.CONFIGS["cfg5_sweep_f16"].with_(batch=34, n_heads=4, n_query=16)
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    d = {k: dev(v) for k, v in batch.items()}
+    ws = tcb.workspace(p)
+    outs = []
+    try:
+        for groups in (1, 4, 16):
+            tcb.tc_set_groups(groups)
+            o = tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)
+            torch.cuda.synchronize()
+            outs.append([host(t) for t in o])
+    finally:
+        tcb.tc_set_groups(4)
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert np.array_equal(a, b)
+    assert not outs[0][4].any()
+    # ... and the staged calls (whole batch, no groups in their selection and gather) agree with
+    # the fused ones bit for bit and with the oracle
+    res = run_staged(p, batch, True)
+    assert np.array_equal(res["kept"], outs[2][3]) and np.array_equal(res["Xo"], outs[2][0])
+    assert np.array_equal(res["Ko"], outs[2][1]) and np.array_equal(res["Vo"], outs[2][2])
+    for bi in (0, 17, 33):
+        f = pu.check_image(cfgp_of(p), {k: batch[k][bi] for k in batch}, image_slice(res, bi))
+        assert f["flips_sets"] + f["flips_merge"] <= 2, f
+
+
 def test_host_entry_point_matches_the_device_one():
     cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=6)       # chunks of 2, 2, 1, 1 images
     p = params_of(cfg)
