@@ -1086,7 +1086,8 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
   const int PW = k;                       // row length of P (k is a multiple of 16)
   float* P = fsm;                          // [16][PW] block row, later [<= k][16] the product T
   float* Dinv = P + CNB * PW;              // [nblk][16][16] inverses of the diagonal blocks
-  float* A = Dinv + nblk * CNB * CNB;      // [k][ld]
+  float* TB = Dinv + nblk * CNB * CNB;     // [k][16] the product T = R[0:j0, J] D_J of the inverse
+  float* A = TB + CNB * k;                 // [k][ld]
   const size_t kk = (size_t)k * k;
   const float* Sb = S + (size_t)b * nparts * kk;  // S arrives as nparts parts to be added up
 
@@ -1219,6 +1220,76 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
     for (int xx = 0; xx < 4; ++xx)
       if (on && r0 + xx < m && cl >= r0 + xx) A[(j1 + r0 + xx) * ld + j1 + cl] -= acc[xx];
   };
+  // ---- the inverse X = R^{-1}, in place, one block column J per step of the factorisation:
+  //        X[0:j0, J] = -X[0:j0, 0:j0] (R[0:j0, J] D_J),   X_JJ = D_J.
+  //      Step J reads rows of R above block row J (final since step J - 1), D_J (from the
+  //      look-ahead of step J - 1) and the block columns of X before J, and writes only above
+  //      block row J, where the factorisation no longer looks: it runs inside step J of the
+  //      factorisation, on the warps that the shrinking trailing update leaves idle.
+  // T = R[0:j0, J] D_J, all threads
+  auto inv_T = [&](int j0, const float* Dj) {
+    for (int rb = 0; rb < j0; rb += 128) {
+      const int r = rb + (tid >> 2), cg = tid & 3;
+      if (r < j0) {
+        float out[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int mm = 0; mm < CNB; ++mm) {
+          const float rv = A[r * ld + j0 + mm];
+          const float4 d4 = *reinterpret_cast<const float4*>(Dj + mm * CNB + 4 * cg);
+          out[0] = fmaf(rv, d4.x, out[0]);
+          out[1] = fmaf(rv, d4.y, out[1]);
+          out[2] = fmaf(rv, d4.z, out[2]);
+          out[3] = fmaf(rv, d4.w, out[3]);
+        }
+        *reinterpret_cast<float4*>(TB + r * CNB + 4 * cg) = make_float4(out[0], out[1], out[2], out[3]);
+      }
+    }
+  };
+  // X[r][J] = - sum_{mm = r}^{j0 - 1} X[r][mm] T[mm][:] and X_JJ = D_J, warps 1 .. 15
+  auto inv_X = [&](int j0, const float* Dj) {
+    const int t2 = tid - 32;  // 0 .. 479
+    for (int rb = 0; rb < j0; rb += 120) {
+      const int r = rb + (t2 >> 2), cg = t2 & 3;
+      if (r < j0) {
+        float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
+        const float* xr = A + r * ld;
+        const float* tb = TB + 4 * cg;
+        // the eight rows of a warp walk the same mm (from the first of them on, entries left
+        // of a row's diagonal counting as zero), so that lanes with the same columns read the
+        // same 16 bytes of T
+        int mm = r & ~7;
+        for (; mm + 3 < j0; mm += 4) {
+          const float x0 = (mm >= r) ? xr[mm] : 0.f, x1 = (mm + 1 >= r) ? xr[mm + 1] : 0.f;
+          const float x2 = (mm + 2 >= r) ? xr[mm + 2] : 0.f, x3 = (mm + 3 >= r) ? xr[mm + 3] : 0.f;
+          const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
+          const float4 t1 = *reinterpret_cast<const float4*>(tb + (mm + 1) * CNB);
+          const float4 t2v = *reinterpret_cast<const float4*>(tb + (mm + 2) * CNB);
+          const float4 t3 = *reinterpret_cast<const float4*>(tb + (mm + 3) * CNB);
+          o0[0] = fmaf(x0, t0.x, o0[0]); o0[1] = fmaf(x0, t0.y, o0[1]);
+          o0[2] = fmaf(x0, t0.z, o0[2]); o0[3] = fmaf(x0, t0.w, o0[3]);
+          o1[0] = fmaf(x1, t1.x, o1[0]); o1[1] = fmaf(x1, t1.y, o1[1]);
+          o1[2] = fmaf(x1, t1.z, o1[2]); o1[3] = fmaf(x1, t1.w, o1[3]);
+          o0[0] = fmaf(x2, t2v.x, o0[0]); o0[1] = fmaf(x2, t2v.y, o0[1]);
+          o0[2] = fmaf(x2, t2v.z, o0[2]); o0[3] = fmaf(x2, t2v.w, o0[3]);
+          o1[0] = fmaf(x3, t3.x, o1[0]); o1[1] = fmaf(x3, t3.y, o1[1]);
+          o1[2] = fmaf(x3, t3.z, o1[2]); o1[3] = fmaf(x3, t3.w, o1[3]);
+        }
+        for (; mm < j0; ++mm) {
+          const float x0 = (mm >= r) ? xr[mm] : 0.f;
+          const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
+          o0[0] = fmaf(x0, t0.x, o0[0]); o0[1] = fmaf(x0, t0.y, o0[1]);
+          o0[2] = fmaf(x0, t0.z, o0[2]); o0[3] = fmaf(x0, t0.w, o0[3]);
+        }
+        // columns J of these rows are read by nobody in this part of the step
+#pragma unroll
+        for (int u = 0; u < 4; ++u) A[r * ld + j0 + 4 * cg + u] = -(o0[u] + o1[u]);
+      }
+    }
+    if (t2 < CNB * CNB) {
+      const int i = t2 >> 4, c = t2 & 15;
+      A[(j0 + i) * ld + j0 + c] = Dj[i * CNB + c];
+    }
+  };
   if (warp == 0) diag(0);
   __syncthreads();
   for (int jb = 0; jb < nblk; ++jb) {
@@ -1264,87 +1335,19 @@ __global__ void __launch_bounds__(512) chol_inv_fast_kernel(const float* __restr
         if (u >= ((4 * s4) >> 5)) trail_unit(j1, m, 4 * s4, u);
       }
     }
+    inv_T(j0, Dj);
     __syncthreads();
     if (warp == 0) {
       if (jb + 1 < nblk) diag(jb + 1);
     } else {
       for (int s4 = 4 + (warp - 1); s4 * 4 < m; s4 += 15)
         for (int u = (4 * s4) >> 5; u * 32 < m; ++u) trail_unit(j1, m, 4 * s4, u);
+      inv_X(j0, Dj);
     }
     __syncthreads();
   }
   if (tid == 0 && s_bad) atomicMax(&status[b], (int)TC_ERR_BREAKDOWN);
 
-  // ---------------- phase 2: X = R^{-1}, in place ----------------
-  float* TB = P;  // [j0][16]
-  for (int jb = 0; jb < nblk; ++jb) {
-    const int j0 = jb * CNB;
-    const float* Dj = Dinv + jb * CNB * CNB;
-    if (j0 > 0) {
-      // T = R[0:j0, J] D_J
-      for (int rb = 0; rb < j0; rb += 128) {
-        const int r = rb + (tid >> 2), cg = tid & 3;
-        if (r < j0) {
-          float out[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-          for (int mm = 0; mm < CNB; ++mm) {
-            const float rv = A[r * ld + j0 + mm];
-            const float4 d4 = *reinterpret_cast<const float4*>(Dj + mm * CNB + 4 * cg);
-            out[0] = fmaf(rv, d4.x, out[0]);
-            out[1] = fmaf(rv, d4.y, out[1]);
-            out[2] = fmaf(rv, d4.z, out[2]);
-            out[3] = fmaf(rv, d4.w, out[3]);
-          }
-          *reinterpret_cast<float4*>(TB + r * CNB + 4 * cg) = make_float4(out[0], out[1], out[2], out[3]);
-        }
-      }
-      __syncthreads();
-      // X[r][J] = - sum_{mm = r}^{j0 - 1} X[r][mm] T[mm][:]
-      for (int rb = 0; rb < j0; rb += 128) {
-        const int r = rb + (tid >> 2), cg = tid & 3;
-        if (r < j0) {
-          float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
-          const float* xr = A + r * ld;
-          const float* tb = TB + 4 * cg;
-          // the eight rows of a warp walk the same mm (from the first of them on, entries left
-          // of a row's diagonal counting as zero), so that lanes with the same columns read the
-          // same 16 bytes of T
-          int mm = r & ~7;
-          for (; mm + 3 < j0; mm += 4) {
-            const float x0 = (mm >= r) ? xr[mm] : 0.f, x1 = (mm + 1 >= r) ? xr[mm + 1] : 0.f;
-            const float x2 = (mm + 2 >= r) ? xr[mm + 2] : 0.f, x3 = (mm + 3 >= r) ? xr[mm + 3] : 0.f;
-            const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
-            const float4 t1 = *reinterpret_cast<const float4*>(tb + (mm + 1) * CNB);
-            const float4 t2 = *reinterpret_cast<const float4*>(tb + (mm + 2) * CNB);
-            const float4 t3 = *reinterpret_cast<const float4*>(tb + (mm + 3) * CNB);
-            o0[0] = fmaf(x0, t0.x, o0[0]); o0[1] = fmaf(x0, t0.y, o0[1]);
-            o0[2] = fmaf(x0, t0.z, o0[2]); o0[3] = fmaf(x0, t0.w, o0[3]);
-            o1[0] = fmaf(x1, t1.x, o1[0]); o1[1] = fmaf(x1, t1.y, o1[1]);
-            o1[2] = fmaf(x1, t1.z, o1[2]); o1[3] = fmaf(x1, t1.w, o1[3]);
-            o0[0] = fmaf(x2, t2.x, o0[0]); o0[1] = fmaf(x2, t2.y, o0[1]);
-            o0[2] = fmaf(x2, t2.z, o0[2]); o0[3] = fmaf(x2, t2.w, o0[3]);
-            o1[0] = fmaf(x3, t3.x, o1[0]); o1[1] = fmaf(x3, t3.y, o1[1]);
-            o1[2] = fmaf(x3, t3.z, o1[2]); o1[3] = fmaf(x3, t3.w, o1[3]);
-          }
-          for (; mm < j0; ++mm) {
-            const float x0 = (mm >= r) ? xr[mm] : 0.f;
-            const float4 t0 = *reinterpret_cast<const float4*>(tb + mm * CNB);
-            o0[0] = fmaf(x0, t0.x, o0[0]); o0[1] = fmaf(x0, t0.y, o0[1]);
-            o0[2] = fmaf(x0, t0.z, o0[2]); o0[3] = fmaf(x0, t0.w, o0[3]);
-          }
-          // columns J of A are not read in this step: the results can go straight in
-#pragma unroll
-          for (int u = 0; u < 4; ++u) A[r * ld + j0 + 4 * cg + u] = -(o0[u] + o1[u]);
-        }
-      }
-    }
-    // X_JJ = D_J
-    if (tid < CNB * CNB) {
-      const int i = tid >> 4, c = tid & 15;
-      A[(j0 + i) * ld + j0 + c] = Dj[i * CNB + c];
-    }
-    __syncthreads();
-  }
   // RinvT[c][m] = X[m][c] for m <= c, zero otherwise
   float* out = RinvT + b * kk;
   for (int e = tid; e < (int)kk; e += 512) {
@@ -2322,7 +2325,7 @@ static void launch_jacobi(const float* H, float* W, float* ZT, float* theta, int
 static void launch_chol_inv(const float* S, float* RinvT, float* Rwork, int k, int batch,
                             float shift_rel, int32_t* status, cudaStream_t st, int nparts) {
   Scope scope_(KC_CHOL, st);
-  const size_t fast = ((size_t)k * (k | 1) + (size_t)CNB * k + (size_t)(k / CNB) * CNB * CNB) * sizeof(float);
+  const size_t fast = ((size_t)k * (k | 1) + 2 * (size_t)CNB * k + (size_t)(k / CNB) * CNB * CNB) * sizeof(float);
   if (k % CNB == 0 && k >= CNB && fast <= SMEM_LIMIT) {
     auto go = [&](auto kernel) {
       cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast);
