@@ -39,7 +39,8 @@ constexpr int DH = 128;          // head dimension the kernel is built for
 constexpr uint32_t ATOM = 128 * 128;        // bytes of one 128-row x 64-element swizzle atom
 constexpr uint32_t TILE_B = 2 * ATOM;       // a 128 x 128 tile of 16-bit elements
 constexpr uint32_t SMEM_O = 5 * TILE_B + 1024;   // Q, K, P, two tiles of V^T
-constexpr uint32_t SMEM_A = 2 * TILE_B + 1024;   // Q, K
+constexpr uint32_t STG_ROW = 2 * KB + 16;         // bytes of a row of the staging tile (padded: no bank is hit twice by a quarter warp)
+constexpr uint32_t SMEM_A = 2 * TILE_B + QT * STG_ROW + 1024;   // Q, K, staging tile of the probabilities
 constexpr uint32_t TMEM_COLS_O = 512;            // two score accumulators and the block's P V
 constexpr uint32_t TMEM_COLS_A = 256;            // two score accumulators
 
@@ -84,6 +85,13 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// 2^x on the special-function unit (relative error 2^-22: far inside the 16-bit outputs)
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 template <typename T>
@@ -276,7 +284,7 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
         pair_sync();
         bm = fmaxf(bm, s_xm[it & 1][half ^ 1][row]);
         const float m_new = fmaxf(m, bm * pa.scale2);
-        alpha = (m_new == -INFINITY) ? 1.f : exp2f(m - m_new);
+        alpha = (m_new == -INFINITY) ? 1.f : ex2(m - m_new);
         m = m_new;
         l *= alpha;
       }
@@ -291,7 +299,7 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
           float pr[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float e = exp2f(fmaf(__uint_as_float(r[j]), pa.scale2, -m));
+            const float e = ex2(fmaf(__uint_as_float(r[j]), pa.scale2, -m));
             pr[j] = (c * 32 + j <= jmax && m != -INFINITY) ? e : 0.f;
             ls += pr[j];
           }
@@ -314,21 +322,45 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
         }
         l += ls;
       } else {
-        // second pass of the probe rows: normalised probabilities of the visual columns
+        // second pass of the probe rows: normalised probabilities of the block's columns into a
+        // staging tile (row-major, 16-bit), from which whole rows leave in runs of 32
+        // neighbouring elements per store (a thread owns a row, so storing from the registers
+        // would put every lane of a store into a sector of its own)
+        uint8_t* stg = smem_gen + 2 * TILE_B;
+        if (it > nkb) pair_sync();   // the rows of the block before have left the tile
 #pragma unroll
         for (int c = 0; c < HC / 32; ++c) {
           uint32_t r[32];
           tmem_ld32_issue(ts + (uint32_t)(c * 32), r);
           tmem_wait_ld();
-          if (live) {
-            T* dst = out + (((size_t)bh * pa.n_rows + (qpos - pa.row0)) * pa.n_vis);
+          float pr[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int key = kb * KB + (int)col0 + c * 32 + j, x = key - pa.n_sys;
-              if (x >= 0 && x < pa.n_vis) {
-                const float e = exp2f(fmaf(__uint_as_float(r[j]), pa.scale2, -m)) * inv_l;
-                dst[x] = (T)((c * 32 + j <= jmax) ? e : 0.f);
-              }
+          for (int j = 0; j < 32; ++j) {
+            const float e = ex2(fmaf(__uint_as_float(r[j]), pa.scale2, -m)) * inv_l;
+            pr[j] = (c * 32 + j <= jmax) ? e : 0.f;
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint4 v;
+            v.x = pack2<T>(pr[q * 8], pr[q * 8 + 1]);
+            v.y = pack2<T>(pr[q * 8 + 2], pr[q * 8 + 3]);
+            v.z = pack2<T>(pr[q * 8 + 4], pr[q * 8 + 5]);
+            v.w = pack2<T>(pr[q * 8 + 6], pr[q * 8 + 7]);
+            *reinterpret_cast<uint4*>(stg + (uint32_t)row * STG_ROW + (col0 + (uint32_t)(c * 32 + q * 8)) * 2u) = v;
+          }
+        }
+        pair_sync();
+        {
+          const int x0 = kb * KB - pa.n_sys;   // visual index of the block's first column
+          for (int rr = warp; rr < QT; rr += 8) {
+            const int qp = q0 + rr;
+            if (qp > q_last) break;
+            T* drow = out + (((size_t)bh * pa.n_rows + (qp - pa.row0)) * pa.n_vis);
+            const T* srow = reinterpret_cast<const T*>(stg + (uint32_t)rr * STG_ROW);
+#pragma unroll
+            for (int j = 0; j < KB / 32; ++j) {
+              const int col = lane + 32 * j, x = x0 + col;
+              if (x >= 0 && x < pa.n_vis) drow[x] = srow[col];
             }
           }
         }
