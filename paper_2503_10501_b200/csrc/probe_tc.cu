@@ -38,10 +38,10 @@ constexpr int KB = 128;          // keys per block
 constexpr int DH = 128;          // head dimension the kernel is built for
 constexpr uint32_t ATOM = 128 * 128;        // bytes of one 128-row x 64-element swizzle atom
 constexpr uint32_t TILE_B = 2 * ATOM;       // a 128 x 128 tile of 16-bit elements
-constexpr uint32_t SMEM_O = 5 * TILE_B + 1024;   // Q, K, P, two tiles of V^T
+constexpr uint32_t SMEM_O = 6 * TILE_B + 1024;   // Q, K, two tiles of P, two tiles of V^T
 constexpr uint32_t STG_ROW = 2 * KB + 16;         // bytes of a row of the staging tile (padded: no bank is hit twice by a quarter warp)
 constexpr uint32_t SMEM_A = 2 * TILE_B + QT * STG_ROW + 1024;   // Q, K, staging tile of the probabilities
-constexpr uint32_t TMEM_COLS_O = 512;            // two score accumulators and the block's P V
+constexpr uint32_t TMEM_COLS_O = 512;            // two score accumulators and two for the blocks' P V
 constexpr uint32_t TMEM_COLS_A = 256;            // two score accumulators
 
 // D float32, A and B float16 (bf = 0) or bfloat16 (bf = 1), both K-major, M = N = 128
@@ -125,10 +125,12 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
   extern __shared__ uint8_t smem_raw[];
   // bar_k: key tile landed; bar_kfree: its scores are formed (the tile may be reloaded);
   // bar_v[2]: V^T tile landed; bar_s[2]: scores ready in accumulator 0 / 1; bar_sfree[2]: the
-  // softmax warps are done with that accumulator; bar_p: P written; bar_pv: P V done (O_blk
-  // ready, P free); bar_vfree[2]: the same event per V^T tile (so that no waiter can fall two
-  // completions behind)
-  __shared__ __align__(8) uint64_t bar_q, bar_k, bar_kfree, bar_v[2], bar_vfree[2], bar_s[2], bar_sfree[2], bar_p, bar_pv;
+  // softmax warps are done with that accumulator; bar_p[2]: tile of P written; bar_pv[2]: its
+  // P V done (O_blk ready, that tile of P free); bar_vfree[2]: the same event for the loader of
+  // the V^T tiles (every waiter has a barrier of its own, so none can fall two completions
+  // behind); bar_ofree[2]: the softmax warps have folded that O_blk into their rows
+  __shared__ __align__(8) uint64_t bar_q, bar_k, bar_kfree, bar_v[2], bar_vfree[2], bar_s[2], bar_sfree[2],
+      bar_p[2], bar_pv[2], bar_ofree[2];
   constexpr uint32_t TMEM_COLS = WANT_O ? TMEM_COLS_O : TMEM_COLS_A;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
@@ -143,8 +145,9 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
   const int nkb = q_last / KB + 1;                        // causal: keys up to the last row's position
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t sQ = smem_base, sK = smem_base + TILE_B, sP = smem_base + 2 * TILE_B;
-  auto sV = [&](int i) { return smem_base + (uint32_t)(3 + (i & 1)) * TILE_B; };
+  const uint32_t sQ = smem_base, sK = smem_base + TILE_B;
+  auto sP = [&](int i) { return smem_base + (uint32_t)(2 + (i & 1)) * TILE_B; };
+  auto sV = [&](int i) { return smem_base + (uint32_t)(4 + (i & 1)) * TILE_B; };
   const uint32_t id = idesc(pa.bf);
 
   if (threadIdx.x == 0) {
@@ -156,9 +159,10 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
       mbar_init(smem_u32(&bar_vfree[i]), 1);
       mbar_init(smem_u32(&bar_s[i]), 1);
       mbar_init(smem_u32(&bar_sfree[i]), 8);
+      mbar_init(smem_u32(&bar_p[i]), 8);
+      mbar_init(smem_u32(&bar_pv[i]), 1);
+      mbar_init(smem_u32(&bar_ofree[i]), 8);
     }
-    mbar_init(smem_u32(&bar_p), 8);
-    mbar_init(smem_u32(&bar_pv), 1);
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -173,7 +177,7 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   auto tmem_s = [&](int i) { return s_tmem + (uint32_t)(i & 1) * 128u; };
-  const uint32_t tmem_o = s_tmem + 256u;
+  auto tmem_o = [&](int i) { return s_tmem + 256u + (uint32_t)(i & 1) * 128u; };
 
   // key blocks in the order they are walked: all of them once (WANT_O), or all of them for the
   // row statistics and then those that hold visual columns once more
@@ -222,12 +226,16 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
       for (int it = 0; it < n_iter && ok; ++it) {
         if (it + 1 < n_iter) ok = scores(it + 1);
         if (WANT_O && ok) {
-          if (!mbar_wait(smem_u32(&bar_p), (uint32_t)it & 1u) ||
-              !mbar_wait(smem_u32(&bar_v[it & 1]), ((uint32_t)it >> 1) & 1u)) { ok = false; break; }
+          const uint32_t par = ((uint32_t)it >> 1) & 1u;
+          if (!mbar_wait(smem_u32(&bar_p[it & 1]), par) || !mbar_wait(smem_u32(&bar_v[it & 1]), par) ||
+              (it >= 2 && !mbar_wait(smem_u32(&bar_ofree[it & 1]), ((uint32_t)(it - 2) >> 1) & 1u))) {
+            ok = false;
+            break;
+          }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          mma_tile(tmem_o, sP, sV(it), id);             // O_blk = P V
+          mma_tile(tmem_o(it), sP(it), sV(it), id);     // O_blk = P V
           umma_commit(smem_u32(&bar_vfree[it & 1]));
-          umma_commit(smem_u32(&bar_pv));
+          umma_commit(smem_u32(&bar_pv[it & 1]));
         }
       }
       if (!ok) s_fail = 1;
@@ -249,8 +257,26 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
     auto pair_sync = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };
     bool ok = true;
     float inv_l = 0.f;
+    float alpha_prev = 1.f;
+    // o = o * alpha_j + (P V of block j); alpha_j = 2^(m_{j-1} - m_j) is the factor block j's new
+    // maximum put on everything before it
+    auto fold = [&](int j, float alpha_j) {
+      if (ok && !mbar_wait(smem_u32(&bar_pv[j & 1]), ((uint32_t)j >> 1) & 1u)) ok = false;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+      for (int c = 0; c < HC / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32_issue(tmem_o(j) + lane_addr + col0 + (uint32_t)(c * 32), r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) o[c * 32 + jj] = fmaf(o[c * 32 + jj], alpha_j, __uint_as_float(r[jj]));
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_ofree[j & 1])) : "memory");
+    };
     for (int it = 0; it < n_iter; ++it) {
-      const uint32_t ph = (uint32_t)it & 1u;
       const int kb = block_of(it);
       const bool second = it >= nkb;
       const uint32_t ts = tmem_s(it) + lane_addr + col0;
@@ -315,7 +341,7 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
               v.y = pack2<T>(pr[q * 8 + 2], pr[q * 8 + 3]);
               v.z = pack2<T>(pr[q * 8 + 4], pr[q * 8 + 5]);
               v.w = pack2<T>(pr[q * 8 + 6], pr[q * 8 + 7]);
-              *reinterpret_cast<uint4*>(smem_gen + 2 * TILE_B + (uint32_t)half * ATOM + (uint32_t)row * 128u +
+              *reinterpret_cast<uint4*>(smem_gen + (uint32_t)(2 + (it & 1)) * TILE_B + (uint32_t)half * ATOM + (uint32_t)row * 128u +
                                         ((ch ^ ((uint32_t)row & 7u)) << 4)) = v;
             }
           }
@@ -371,24 +397,18 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
       if (lane == 0)
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_sfree[it & 1])) : "memory");
       if (WANT_O) {
-        // hand P to the tensor core, then fold the block's P V into the own half of the row of Z
+        // hand this block's P to the tensor core, then fold the P V of the block BEFORE into the
+        // own half of the row of Z: that product ran while this block's probabilities were
+        // formed (two tiles of P, two accumulators for P V), so the wait below is short
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0)
-          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_p)) : "memory");
-        if (ok && !mbar_wait(smem_u32(&bar_pv), ph)) ok = false;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-        for (int c = 0; c < HC / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32_issue(tmem_o + lane_addr + col0 + (uint32_t)(c * 32), r);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[c * 32 + j] = fmaf(o[c * 32 + j], alpha, __uint_as_float(r[j]));
-        }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_p[it & 1])) : "memory");
+        if (it > 0) fold(it - 1, alpha_prev);
+        alpha_prev = alpha;
       }
     }
+    if (WANT_O && n_iter > 0) fold(n_iter - 1, alpha_prev);
     if (WANT_O) {
       // the whole row sum (every thread of the team comes here, whatever happened above)
       s_xl[half][row] = l;
