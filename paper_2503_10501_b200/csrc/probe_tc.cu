@@ -446,24 +446,31 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
   }
 }
 
-// Vt [BH][dh][Lp] = V [BH][L][dh]^T, columns L .. Lp - 1 zero.  32 x 32 tiles; grid (Lp / 32
-// rounded up, dh / 32, BH), block (32, 8).
+// Vt [BH][dh][Lp] = V [BH][L][dh]^T, columns L .. Lp - 1 zero (Lp and dh even).  64 x 64 tiles,
+// two elements per access: a warp reads and writes 128 contiguous bytes.  grid (Lp / 64 rounded
+// up, dh / 64 rounded up, BH), block (32, 8).
 template <typename T>
 __global__ void __launch_bounds__(256) transpose_v_kernel(const T* __restrict__ V, T* __restrict__ Vt,
                                                          int L, int Lp, int dh) {
-  __shared__ T t[32][33];
+  __shared__ T t[64][66];
   const size_t bh = blockIdx.z;
-  const int l0 = blockIdx.x * 32, d0 = blockIdx.y * 32;
+  const int l0 = blockIdx.x * 64, d0 = blockIdx.y * 64;
+  const int tx = threadIdx.x, ty = threadIdx.y;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int l = l0 + threadIdx.y + 8 * i, d = d0 + threadIdx.x;
-    t[threadIdx.y + 8 * i][threadIdx.x] = (l < L && d < dh) ? V[(bh * L + l) * dh + d] : (T)0.f;
+  for (int i = 0; i < 8; ++i) {
+    const int l = l0 + ty + 8 * i, d = d0 + 2 * tx;
+    uint32_t v = 0u;
+    if (l < L && d < dh) v = *reinterpret_cast<const uint32_t*>(V + (bh * L + l) * dh + d);
+    *reinterpret_cast<uint32_t*>(&t[ty + 8 * i][2 * tx]) = v;
   }
   __syncthreads();
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int d = d0 + threadIdx.y + 8 * i, l = l0 + threadIdx.x;
-    if (d < dh && l < Lp) Vt[(bh * dh + d) * Lp + l] = t[threadIdx.x][threadIdx.y + 8 * i];
+  for (int i = 0; i < 8; ++i) {
+    const int dd = ty + 8 * i, d = d0 + dd, l = l0 + 2 * tx;
+    if (d < dh && l < Lp) {
+      T pair[2] = {t[2 * tx][dd], t[2 * tx + 1][dd]};
+      *reinterpret_cast<uint32_t*>(Vt + (bh * dh + d) * Lp + l) = *reinterpret_cast<uint32_t*>(pair);
+    }
   }
 }
 
@@ -500,7 +507,7 @@ tc_status run_probe(int B, int H, int L, int n_sys, int n_vis, int probe_start, 
   pa.bf = bf;
   if (O != nullptr) {
     Scope scope_(KC_GRAM, st);
-    dim3 tg((Lp + 31) / 32, DH / 32, B * H), tb(32, 8);
+    dim3 tg((Lp + 63) / 64, (DH + 63) / 64, B * H), tb(32, 8);
     transpose_v_kernel<T><<<tg, tb, 0, st>>>((const T*)V, (T*)Vt, L, Lp, DH);
     note_launch();
     pa.row0 = n_sys; pa.n_rows = n_vis;
