@@ -352,6 +352,16 @@ tc_status tc_rope_tables(const int32_t* pos, int64_t n_rows, int32_t head_dim, f
 tc_status tc_set_groups(int32_t groups);
 
 /*
+ * Test hook, not part of the method: while `on` is non-zero every launcher that needs a TMA
+ * tensor map is refused on the host (as if the driver's encode entry point were missing), so
+ * that the calls' error paths can be exercised without faulting a GPU: tc_score / tc_carve /
+ * tc_gram / tc_matmul_f32x3 / tc_probe then return TC_ERR_CUDA, leave no kernel of the refused
+ * step enqueued, join their internal streams, and tc_score / tc_carve set img_status of the
+ * images they did not reach.  Process-wide; returns TC_OK.
+ */
+tc_status tc_test_fail_tensor_maps(int32_t on);
+
+/*
  * Optional event profile (diagnostics; the paper has no counterpart).  Between
  * tc_profile_begin() and tc_profile_end() every kernel launch of the library is bracketed by
  * CUDA events on its stream.  tc_profile_end() waits for those events and returns, per kernel

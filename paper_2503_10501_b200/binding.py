@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "TC_OK", 1: "TC_ERR_INVALID_ARG", 2: "TC_ERR_UNSUPPORTED", 3:
 EXPORTS = ("tc_counts", "tc_workspace_bytes", "tc_score", "tc_prune", "tc_merge", "tc_compact",
            "tc_carve", "tc_workspace_bytes_host", "tc_carve_host", "tc_gram", "tc_status_string",
            "tc_version", "tc_launch_count", "tc_profile_begin", "tc_profile_end",
-           "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_rank",
+           "tc_kernel_class_name", "tc_attn_score_noalloc", "tc_set_groups", "tc_test_fail_tensor_maps", "tc_rank",
            "tc_rank_workspace_bytes", "tc_reassemble", "tc_matmul_f32x3", "tc_stage_status", "tc_rope_tables",
            "tc_compact_weighted", "tc_probe", "tc_probe_workspace_bytes")
 
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
         L.tc_probe.argtypes = [pp, C.c_int32, C.c_int32, C.c_int32] + [vp] * 7 + [sz, vp]
         L.tc_matmul_f32x3.argtypes = [vp, vp, vp, vp] + [C.c_int32] * 4 + [vp, vp]
         L.tc_set_groups.argtypes = [C.c_int32]
+        L.tc_test_fail_tensor_maps.argtypes = [C.c_int32]
         L.tc_attn_score_noalloc.argtypes = [pp, vp, vp, vp]
         L.tc_status_string.argtypes = [C.c_int32]
         L.tc_status_string.restype = C.c_char_p
@@ -403,6 +404,11 @@ def tc_status_string(status: int) -> str:
 
 def tc_set_groups(groups: int) -> None:
     _check("tc_set_groups", lib().tc_set_groups(C.c_int32(groups)))
+
+
+def tc_test_fail_tensor_maps(on: bool) -> None:
+    """Test hook: refuse every tensor-map encode on the host while set."""
+    _check("tc_test_fail_tensor_maps", lib().tc_test_fail_tensor_maps(C.c_int32(1 if on else 0)))
 
 
 def tc_version() -> int:

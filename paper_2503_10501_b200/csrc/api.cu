@@ -818,6 +818,11 @@ const char* tc_status_string(int32_t status) {
 
 int32_t tc_version(void) { return 100; }
 
+tc_status tc_test_fail_tensor_maps(int32_t on) {
+  tc::g_refuse_encode.store(on ? 1 : 0);
+  return TC_OK;
+}
+
 tc_status tc_set_groups(int32_t groups) {
   if (groups < 1 || groups > tc::kMaxGroups) return TC_ERR_INVALID_ARG;
   tc::g_n_groups.store(groups);

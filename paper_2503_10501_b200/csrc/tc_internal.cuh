@@ -8,7 +8,14 @@
 
 #include "tokencarve.h"
 
+#include <atomic>
+
 namespace tc {
+
+// test hook (tc_test_fail_tensor_maps): while set, every tensor-map encode is refused, which is
+// how a launcher's refusal after the group streams were forked is exercised without a GPU fault
+inline std::atomic<int> g_refuse_encode{0};
+
 
 // Counts of Sec. 3.3.1 / Eq. 3-9 plus everything the launchers derive from tc_params.
 struct Dims {

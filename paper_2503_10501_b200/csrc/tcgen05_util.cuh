@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "tc_internal.cuh"
+
 namespace tc {
 namespace t5 {
 
@@ -105,6 +107,7 @@ typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
                               CUtensorMapFloatOOBfill);
 
 inline encode_fn get_encode() {
+  if (g_refuse_encode.load()) return nullptr;
   static encode_fn fn = nullptr;
   static bool tried = false;
   if (!tried) {

@@ -544,6 +544,35 @@ def test_start_waves_and_group_tails_do_not_change_results():
         assert f["flips_sets"] + f["flips_merge"] <= 2, f
 
 
+def test_refused_launcher_returns_a_status_and_leaves_the_library_usable():
+    # a launcher that cannot get its tensor map (host-side refusal, injected through the test
+    # hook: nothing faults on the device) must surface as a status from the call, with the
+    # internal streams joined, and the next call must work and give the usual results
+    cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=6)
+    p = params_of(cfg)
+    batch = inputs.make_batch(cfg)
+    d = {k: dev(v) for k, v in batch.items()}
+    ws = tcb.workspace(p)
+    ref = [host(t) for t in tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)]
+    try:
+        for groups in (1, 4):
+            tcb.tc_set_groups(groups)
+            tcb.tc_test_fail_tensor_maps(True)
+            with pytest.raises(tcb.TokenCarveError) as e:
+                tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)
+            assert e.value.status == 5                  # TC_ERR_CUDA
+            with pytest.raises(tcb.TokenCarveError):
+                tcb.tc_score(p, d["O"], d["A"], ws)
+            torch.cuda.synchronize()                    # nothing is left running or waiting
+            tcb.tc_test_fail_tensor_maps(False)
+            out = [host(t) for t in tcb.tc_carve(p, d["O"], d["A"], d["X"], d["K"], d["V"], ws)]
+            for a, b in zip(ref, out):
+                assert np.array_equal(a, b)
+    finally:
+        tcb.tc_test_fail_tensor_maps(False)
+        tcb.tc_set_groups(4)
+
+
 def test_host_entry_point_matches_the_device_one():
     cfg = inputs.CONFIGS["cfg2_llava7b_f16"].with_(batch=6)       # chunks of 2, 2, 1, 1 images
     p = params_of(cfg)
