@@ -264,26 +264,46 @@ __global__ void __launch_bounds__(THREADS) gemm_f32x3_kernel(const __grid_consta
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_acc_empty[buf]))
                      : "memory");
     }
-    if (ok && s_fail == 0) {
+    // The row-major form leaves through shared memory (the operand ring is free: every MMA that
+    // read it has completed): a thread owns a row of the tile, so stores straight from its
+    // registers would put every lane into a sector of its own; from the staging tile a warp
+    // writes whole rows.  All eight warps come to the barrier whatever their waits returned.
+    constexpr int SROW = NN + 4;   // floats per staged row: 16-byte aligned, no bank hit twice by a quarter warp
+    float* stg = reinterpret_cast<float*>(smem_gen);
+    if (!ok) s_fail = 1;
+    if (out.plain != nullptr) {
+      float* srow = stg + (quad * 32 + lane) * SROW;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        const int chunk = 2 * c + half;
+        if (chunk >= NCHUNK) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          *reinterpret_cast<float4*>(srow + chunk * 16 + 4 * j) =
+              make_float4(acc[c][4 * j], acc[c][4 * j + 1], acc[c][4 * j + 2], acc[c][4 * j + 3]);
+      }
+    }
+    asm volatile("bar.sync 2, 256;" ::: "memory");
+    if (s_fail == 0) {
+      const size_t MN = (size_t)M * NN;
+      if (out.plain != nullptr) {
+        for (int rl = warp; rl < BM; rl += EPI_WARPS) {
+          const int grow = mt * BM + rl;
+          if (grow >= M) break;
+          const float4* src = reinterpret_cast<const float4*>(stg + rl * SROW);
+          float4* dst = reinterpret_cast<float4*>(out.plain + (size_t)b * MN + (size_t)grow * NN);
+          for (int v = lane; v < NN / 4; v += 32) dst[v] = src[v];
+        }
+      }
       const int row = mt * BM + quad * 32 + lane;
-      if (row < M) {
-        const size_t MN = (size_t)M * NN;
+      if (row < M && out.plainT != nullptr) {
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int chunk = 2 * c + half;
           if (chunk >= NCHUNK) continue;
-          const int col0 = chunk * 16;
-          if (out.plain != nullptr) {
-            float4* dst = reinterpret_cast<float4*>(out.plain + (size_t)b * MN + (size_t)row * NN + col0);
+          float* dst = out.plainT + (size_t)b * MN + (size_t)(chunk * 16) * M + row;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              dst[j] = make_float4(acc[c][4 * j], acc[c][4 * j + 1], acc[c][4 * j + 2], acc[c][4 * j + 3]);
-          }
-          if (out.plainT != nullptr) {
-            float* dst = out.plainT + (size_t)b * MN + (size_t)col0 * M + row;
-#pragma unroll
-            for (int j = 0; j < 16; ++j) dst[(size_t)j * M] = acc[c][j];
-          }
+          for (int j = 0; j < 16; ++j) dst[(size_t)j * M] = acc[c][j];
         }
       }
     } else if (status != nullptr && threadIdx.x == 0) {
