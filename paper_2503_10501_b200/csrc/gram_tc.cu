@@ -180,29 +180,47 @@ __global__ void __launch_bounds__(192) gram_tc_kernel(const __grid_constant__ CU
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_acc_empty[buf]))
                      : "memory");
     }
-    if (ok && s_fail == 0) {
+    // The tile leaves row-major through shared memory (the operand ring is free: every MMA has
+    // completed): a thread owns a row, so stores from its registers would put each lane of a
+    // store into a sector of its own; from the staging tile a warp writes a whole row per store.
+    // The mirror image goes out from the registers (there the lanes are neighbours).
+    // All four warps come to the barrier whatever their waits returned.
+    constexpr int SROW = TILE + 4;   // floats per staged row
+    float* stg = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
+    if (!ok) s_fail = 1;
+    {
+      float* srow = stg + (warp * 32 + lane) * SROW;
+#pragma unroll
+      for (int j = 0; j < TILE / 4; ++j)
+        *reinterpret_cast<float4*>(srow + 4 * j) =
+            make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (s_fail == 0) {
       float* Gb = G + (size_t)b * N * N;
+      for (int rl = warp; rl < TILE; rl += 4) {
+        const int grow = ti * TILE + rl;
+        if (grow >= N) break;
+        const int col = tj * TILE + 4 * lane;
+        const float4 v = *reinterpret_cast<const float4*>(stg + rl * SROW + 4 * lane);
+        float* dst = Gb + (size_t)grow * N + col;
+        if (col + 3 < N && (N & 3) == 0) {
+          *reinterpret_cast<float4*>(dst) = v;
+        } else {
+          if (col < N) dst[0] = v.x;
+          if (col + 1 < N) dst[1] = v.y;
+          if (col + 2 < N) dst[2] = v.z;
+          if (col + 3 < N) dst[3] = v.w;
+        }
+      }
       const int row = ti * TILE + warp * 32 + lane;
-      if (row < N) {
+      if (row < N && !diag) {
 #pragma unroll
         for (int q = 0; q < TILE / 32; ++q) {
           const int col0 = tj * TILE + q * 32;
-          if (col0 + 32 <= N && (N & 3) == 0) {
-            float4* dst = reinterpret_cast<float4*>(Gb + (size_t)row * N + col0);
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              dst[j] = make_float4(acc[q * 32 + 4 * j], acc[q * 32 + 4 * j + 1],
-                                   acc[q * 32 + 4 * j + 2], acc[q * 32 + 4 * j + 3]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < N) Gb[(size_t)row * N + col0 + j] = acc[q * 32 + j];
-          }
-          if (!diag) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < N) Gb[(size_t)(col0 + j) * N + row] = acc[q * 32 + j];
-          }
+          for (int j = 0; j < 32; ++j)
+            if (col0 + j < N) Gb[(size_t)(col0 + j) * N + row] = acc[q * 32 + j];
         }
       }
     } else if (status != nullptr) {
