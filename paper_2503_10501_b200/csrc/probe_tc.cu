@@ -417,20 +417,31 @@ __global__ void __launch_bounds__(320, 1) probe_kernel(
       inv_l = (lt > 0.f) ? 1.0f / lt : 0.f;
     }
     if (!ok) s_fail = 1;
+    if (WANT_O) {
+      // The rows of Z leave through a row-major staging tile in the first tile of P (every P V
+      // has completed): a thread owns half a row, so stores from its registers would put each
+      // lane of a store into a sector of its own; from the tile a warp writes a row per store.
+      uint8_t* stg = smem_gen + 2 * TILE_B;
+#pragma unroll
+      for (int q = 0; q < HC / 8; ++q) {
+        uint4 v;
+        v.x = pack2<T>(o[q * 8] * inv_l, o[q * 8 + 1] * inv_l);
+        v.y = pack2<T>(o[q * 8 + 2] * inv_l, o[q * 8 + 3] * inv_l);
+        v.z = pack2<T>(o[q * 8 + 4] * inv_l, o[q * 8 + 5] * inv_l);
+        v.w = pack2<T>(o[q * 8 + 6] * inv_l, o[q * 8 + 7] * inv_l);
+        *reinterpret_cast<uint4*>(stg + (uint32_t)row * STG_ROW + (uint32_t)(half * HC + q * 8) * 2u) = v;
+      }
+    }
     pair_sync();
     if (s_fail == 0) {
-      if (WANT_O && live) {
-        // row qpos - n_sys of O, columns h * dh + 64 half ..
-        uint4* dst = reinterpret_cast<uint4*>(
-            out + (((size_t)b * pa.n_vis + (qpos - pa.n_sys)) * pa.H + h) * DH + half * HC);
-#pragma unroll
-        for (int q = 0; q < HC / 8; ++q) {
-          uint4 v;
-          v.x = pack2<T>(o[q * 8] * inv_l, o[q * 8 + 1] * inv_l);
-          v.y = pack2<T>(o[q * 8 + 2] * inv_l, o[q * 8 + 3] * inv_l);
-          v.z = pack2<T>(o[q * 8 + 4] * inv_l, o[q * 8 + 5] * inv_l);
-          v.w = pack2<T>(o[q * 8 + 6] * inv_l, o[q * 8 + 7] * inv_l);
-          dst[q] = v;
+      if (WANT_O) {
+        uint8_t* stg = smem_gen + 2 * TILE_B;
+        for (int rr = warp; rr < QT; rr += 8) {
+          const int qp = q0 + rr;
+          if (qp > q_last) break;
+          // row qp - n_sys of O, columns h * dh ..: 256 bytes, 8 per lane
+          uint2* dst = reinterpret_cast<uint2*>(out + (((size_t)b * pa.n_vis + (qp - pa.n_sys)) * pa.H + h) * DH);
+          dst[lane] = *reinterpret_cast<const uint2*>(stg + (uint32_t)rr * STG_ROW + (uint32_t)lane * 8u);
         }
       }
     } else if (status != nullptr && threadIdx.x == 0) {
