@@ -284,6 +284,52 @@ def run_ours(args):
         for _ in range(min(args.warmup, 2)):
             step_host()
         ms_host, _ = timed(step_host, args.steps)
+
+        # Extra figure, not the headline: the same K steps with two of them in flight (two
+        # graphs with a workspace and outputs each, replayed on alternating streams), as a
+        # server with a queue of batches would run them.  One carve of 64 images is bound by
+        # the latency of its dependent chain; the second batch fills the SMs it leaves idle.
+        pipelined = None
+        nfl = args.inflight
+        if use_graph and world == 1 and nfl >= 2 and args.steps >= nfl:
+            sA = torch.cuda.current_stream()
+            lanes = [(graph, sA, out)]
+            for _ in range(nfl - 1):
+                wsx = tcb.workspace(p, host=True)
+                outx = tuple(torch.empty_like(t) for t in out)
+                sx = torch.cuda.Stream()
+                sx.wait_stream(sA)
+                with torch.cuda.stream(sx):   # warm-up outside capture
+                    tcb.tc_carve(p, devin["O"], devin["A"], devin["X"], devin["K"], devin["V"], wsx, outx)
+                sA.wait_stream(sx)
+                torch.cuda.synchronize()
+                gx = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gx):
+                    tcb.tc_carve(p, devin["O"], devin["A"], devin["X"], devin["K"], devin["V"], wsx, outx)
+                lanes.append((gx, sx, outx, wsx))
+
+            def run_lanes(n):
+                e0 = torch.cuda.Event(enable_timing=True)
+                ends = [torch.cuda.Event(enable_timing=True) for _ in lanes]
+                torch.cuda.synchronize()
+                e0.record(sA)
+                for ln in lanes[1:]:
+                    ln[1].wait_event(e0)
+                for i in range(n):
+                    g_, s_ = lanes[i % nfl][0], lanes[i % nfl][1]
+                    with torch.cuda.stream(s_):
+                        g_.replay()
+                for ln, e in zip(lanes, ends):
+                    e.record(ln[1])
+                torch.cuda.synchronize()
+                return max(e0.elapsed_time(e) for e in ends)
+
+            run_lanes(2 * nfl)
+            ms2 = run_lanes(args.steps)
+            same = all(torch.equal(a_, b_) for ln in lanes[1:] for a_, b_ in zip(out, ln[2]))
+            pipelined = {"steps_in_flight": nfl, "value": cfg.batch * args.steps / (ms2 * 1e-3),
+                         "unit": "images/s", "ms_per_step": ms2 / args.steps,
+                         "outputs_equal_single": bool(same)}
     clocks = cs.summary()
 
     images = cfg.batch * world * args.steps
@@ -353,6 +399,8 @@ def run_ours(args):
                 "kernel_ms_per_step": {k_: round(v[0] / args.steps, 4) for k_, v in prof.items() if v[1]},
                 "kernel_roofline": kfr,
                 "cpu_baseline": cpu}
+        if pipelined is not None:
+            line["steps_in_flight"] = pipelined
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -626,6 +674,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true",
                     help="time plain tc_carve calls instead of the replay of a CUDA graph of one call")
     ap.add_argument("--groups", type=int, default=0, help="concurrent image groups (0 = library default)")
+    ap.add_argument("--inflight", type=int, default=2,
+                    help="extra figure: the timed steps again with this many of them in flight (0 = skip)")
     ap.add_argument("--cpu-images", type=int, default=12,
                     help="images the CPU oracle is timed on (0 = skip)")
     ap.add_argument("--sweep", action="store_true",
